@@ -1,0 +1,183 @@
+"""CPU oracle for the RCP W2A4 decode hot path -- TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+
+Thin ctypes wrapper over ``rcp_oracle.cpp`` (plain single-threaded C++, written from the
+paper's definitions: Appendix A.2 for the Hadamard matrix, Section 4.4 and Appendix A.7 for
+the tensor formats and the LUT product).  Only the tests, the smoke check and the benchmark's
+CPU-baseline leg may import this package; the CUDA library never does, and the two share no
+code.
+"""
+import ctypes as C
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "rcp_oracle.cpp")
+_LIB = os.path.join(_HERE, "librcp_oracle.so")
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ (no fast-math, no FMA contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.check_call(
+            ["g++", "-std=c++17", "-O2", "-fPIC", "-shared", "-ffp-contract=off", "-fno-fast-math",
+             "-o", _LIB, _SRC])
+    return _LIB
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.orc_f16_to_f32.restype = C.c_float
+        _lib.orc_f16_to_f32.argtypes = [C.c_uint16]
+        _lib.orc_f32_to_f16.restype = C.c_uint16
+        _lib.orc_f32_to_f16.argtypes = [C.c_float]
+    return _lib
+
+
+def _p(a):
+    return a.ctypes.data_as(C.c_void_p) if a is not None else None
+
+
+def _c(a, dtype):
+    a = np.ascontiguousarray(a)
+    assert a.dtype == dtype, (a.dtype, dtype)
+    return a
+
+
+def f16_to_f32(bits: int) -> float:
+    return float(lib().orc_f16_to_f32(int(bits)))
+
+
+def f32_to_f16(x: float) -> int:
+    return int(lib().orc_f32_to_f16(C.c_float(x)))
+
+
+def hadamard_matrix(n: int) -> np.ndarray:
+    """Normalized Sylvester Hadamard matrix H_n (Appendix A.2), dense float64."""
+    H = np.empty((n, n), dtype=np.float64)
+    rc = lib().orc_hadamard_matrix(C.c_int(n), _p(H))
+    if rc:
+        raise ValueError("n must be a power of two")
+    return H
+
+
+def rotate_exact_f64(x_f16_bits: np.ndarray, B: int) -> np.ndarray:
+    x = _c(x_f16_bits, np.uint16)
+    y = np.empty(x.shape, dtype=np.float64)
+    K = x.shape[-1]
+    for m in range(x.reshape(-1, K).shape[0]):
+        rc = lib().orc_rotate_exact_f64(_p(x.reshape(-1, K)[m]), C.c_int(K), C.c_int(B), _p(y.reshape(-1, K)[m]))
+        if rc:
+            raise ValueError("bad block")
+    return y
+
+
+def rotate_f32(x_f16_bits: np.ndarray, B: int) -> np.ndarray:
+    x = _c(x_f16_bits, np.uint16).reshape(-1)
+    v = np.empty(x.shape, dtype=np.float32)
+    rc = lib().orc_rotate_f32(_p(x), C.c_int(x.size), C.c_int(B), _p(v))
+    if rc:
+        raise ValueError("bad block")
+    return v
+
+
+def quantize_act(x_f16_bits: np.ndarray, had_block: int, clip_ratio: float = 1.0):
+    """x: uint16 [M][K] (fp16 bit patterns). Returns dict(xq u8 [M][K/2], scale u16 [M], q i8 [M][K], v f32 [M][K])."""
+    x = _c(x_f16_bits, np.uint16)
+    M, K = x.shape
+    xq = np.empty((M, K // 2), dtype=np.uint8)
+    scale = np.empty((M,), dtype=np.uint16)
+    q = np.empty((M, K), dtype=np.int8)
+    v = np.empty((M, K), dtype=np.float32)
+    rc = lib().orc_quantize_act(_p(x), C.c_int(M), C.c_int(K), C.c_int(had_block), C.c_float(clip_ratio),
+                                _p(xq), _p(scale), _p(q), _p(v))
+    if rc:
+        raise ValueError(f"orc_quantize_act failed: {rc}")
+    return dict(xq=xq, scale=scale, q=q, v=v)
+
+
+def unpack_act(xq: np.ndarray) -> np.ndarray:
+    xq = _c(xq, np.uint8)
+    q = np.empty(xq.shape[:-1] + (xq.shape[-1] * 2,), dtype=np.int8)
+    lib().orc_unpack_act(_p(xq), C.c_size_t(xq.size), _p(q))
+    return q
+
+
+def pack_weights(codes: np.ndarray) -> np.ndarray:
+    codes = _c(codes, np.uint8)
+    N, K = codes.shape
+    words = np.empty((N, K // 16), dtype=np.uint32)
+    rc = lib().orc_pack_weights(_p(codes), C.c_int(N), C.c_int(K), _p(words))
+    if rc:
+        raise ValueError(f"orc_pack_weights failed: {rc}")
+    return words
+
+
+def unpack_weights(words: np.ndarray) -> np.ndarray:
+    words = _c(words, np.uint32)
+    N, W = words.shape
+    codes = np.empty((N, W * 16), dtype=np.uint8)
+    lib().orc_unpack_weights(_p(words), C.c_int(N), C.c_int(W * 16), _p(codes))
+    return codes
+
+
+def gemv_w2a4(words, lut_bits, xq, scale_bits):
+    """Returns dict(S int32 [M][N][4], y float64 [M][N], tol float64 [M][N])."""
+    words = _c(words, np.uint32)
+    lut = _c(lut_bits, np.uint16)
+    xq = _c(xq, np.uint8)
+    scale = _c(scale_bits, np.uint16)
+    N, W = words.shape
+    K = W * 16
+    M = xq.shape[0]
+    assert xq.shape == (M, K // 2) and lut.shape == (N, 4) and scale.shape == (M,)
+    S = np.empty((M, N, 4), dtype=np.int32)
+    y = np.empty((M, N), dtype=np.float64)
+    tol = np.empty((M, N), dtype=np.float64)
+    rc = lib().orc_gemv_w2a4(_p(words), _p(lut), _p(xq), _p(scale), C.c_int(M), C.c_int(N), C.c_int(K),
+                             _p(S), _p(y), _p(tol))
+    if rc:
+        raise ValueError(f"orc_gemv_w2a4 failed: {rc}")
+    return dict(S=S, y=y, tol=tol)
+
+
+def gemv_direct(words, lut_bits, xq, scale_bits):
+    """Direct sum over k. Returns dict(y float64 [M][N], acc_int int64 [M][N])."""
+    words = _c(words, np.uint32)
+    lut = _c(lut_bits, np.uint16)
+    xq = _c(xq, np.uint8)
+    scale = _c(scale_bits, np.uint16)
+    N, W = words.shape
+    K = W * 16
+    M = xq.shape[0]
+    y = np.empty((M, N), dtype=np.float64)
+    ai = np.empty((M, N), dtype=np.int64)
+    rc = lib().orc_gemv_direct(_p(words), _p(lut), _p(xq), _p(scale), C.c_int(M), C.c_int(N), C.c_int(K),
+                               _p(y), _p(ai))
+    if rc:
+        raise ValueError(f"orc_gemv_direct failed: {rc}")
+    return dict(y=y, acc_int=ai)
+
+
+def percode_int(lut_bits, S):
+    lut = _c(lut_bits, np.uint16)
+    S = _c(S, np.int32)
+    M, N, _ = S.shape
+    ai = np.empty((M, N), dtype=np.int64)
+    lib().orc_percode_int(_p(lut), _p(S), C.c_int(M), C.c_int(N), _p(ai))
+    return ai
+
+
+def dequant_weights(words, lut_bits):
+    words = _c(words, np.uint32)
+    lut = _c(lut_bits, np.uint16)
+    N, W = words.shape
+    Wd = np.empty((N, W * 16), dtype=np.float64)
+    lib().orc_dequant_weights(_p(words), _p(lut), C.c_int(N), C.c_int(W * 16), _p(Wd))
+    return Wd

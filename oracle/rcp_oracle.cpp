@@ -1,0 +1,373 @@
+// rcp_oracle.cpp -- TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+//
+// Plain, slow, single-threaded CPU oracle for the decode-time W2A4 hot path of RCP
+// (Rotate, Clip, Partition; arXiv 2502.15779):
+//   * block-Hadamard rotation of the activation (Appendix A.2, definition of the
+//     normalized Hadamard matrix H_n = H'_n / sqrt(n), Sylvester recursion),
+//   * per-token symmetric absmax int4 quantization and nibble packing (Section 4.4
+//     "Fast GEMV via Latency Hiding": X_q is 1 x C/2 INT8 holding two INT4 each, scale is
+//     one FP16 scalar; Table "Quantization configurations": activations symmetric,
+//     per-token),
+//   * 2-bit weight-code packing (Section 4.4: W_q packed sub-byte along the input channel),
+//   * the look-up-table GEMV  O = s * X_q * LUT[W_q]  (Section 4.4, Eq. "deqgrid": the
+//     four-entry dequantization grid W^_0..W^_3 per quantization unit).
+//
+// Only tests, the smoke check and the benchmark's CPU-baseline leg may call this file.
+// It shares no code, header, table or helper with the CUDA library, and the CUDA library
+// never calls it. No SIMD intrinsics, no threads, no blocking or reordering beyond what the
+// definitions state.
+//
+// Pins (all in tests marked "not gpu"): H H^T = I and FWHT == explicit Sylvester matrix
+// product; library fp16 conversion; hand-computed rounding cases; brute-force 8x8 and
+// 16x32 GEMV; exact integer equality of the per-code-sum form and the direct form;
+// LUT lookup of unpacked codes == dequantized weight matrix; affine/constant LUT special
+// cases reducing to a plain integer GEMV.
+// fp16 output y: the paper prints no worked numeric GEMV example, so y is pinned only by the
+// mathematical identities above, not by a printed value.
+#include <cstdint>
+#include <cstring>
+#include <cmath>
+#include <cstdlib>
+
+extern "C" {
+
+// ---------------------------------------------------------------------------------------
+// IEEE binary16 <-> binary32, written at the bit level (round-to-nearest-even, subnormals,
+// infinities and NaN handled). No compiler half type is used.
+// ---------------------------------------------------------------------------------------
+float orc_f16_to_f32(uint16_t h) {
+  uint32_t sign = (uint32_t)(h >> 15) & 1u;
+  uint32_t exp = (uint32_t)(h >> 10) & 0x1Fu;
+  uint32_t man = (uint32_t)h & 0x3FFu;
+  uint32_t out;
+  if (exp == 0) {
+    if (man == 0) {
+      out = sign << 31;
+    } else {
+      // subnormal: value = man * 2^-24; normalise
+      int e = -1;
+      do { man <<= 1; e++; } while ((man & 0x400u) == 0);
+      man &= 0x3FFu;
+      out = (sign << 31) | ((uint32_t)(127 - 15 - e) << 23) | (man << 13);
+    }
+  } else if (exp == 31) {
+    out = (sign << 31) | 0x7F800000u | (man << 13);
+  } else {
+    out = (sign << 31) | ((exp - 15 + 127) << 23) | (man << 13);
+  }
+  float f;
+  std::memcpy(&f, &out, 4);
+  return f;
+}
+
+uint16_t orc_f32_to_f16(float f) {
+  uint32_t x;
+  std::memcpy(&x, &f, 4);
+  uint32_t sign = (x >> 16) & 0x8000u;
+  uint32_t exp = (x >> 23) & 0xFFu;
+  uint32_t man = x & 0x7FFFFFu;
+  if (exp == 255) {  // inf / nan
+    return (uint16_t)(sign | 0x7C00u | (man ? (0x200u | (man >> 13)) : 0u));
+  }
+  int e = (int)exp - 127 + 15;  // biased half exponent
+  if (e >= 31) return (uint16_t)(sign | 0x7C00u);  // overflow -> inf
+  if (e <= 0) {
+    // result is subnormal or zero: value = 1.man * 2^(e-15), unit 2^-24
+    if (e < -10) return (uint16_t)sign;  // below half of the smallest subnormal
+    uint32_t m = man | 0x800000u;         // 24-bit significand
+    int shift = 14 - e;                   // bits to drop (14..24)
+    uint32_t q = m >> shift;
+    uint32_t rem = m & ((1u << shift) - 1u);
+    uint32_t half = 1u << (shift - 1);
+    if (rem > half || (rem == half && (q & 1u))) q++;
+    return (uint16_t)(sign | q);  // a carry into bit 10 yields the smallest normal: correct
+  }
+  uint32_t q = man >> 13;
+  uint32_t rem = man & 0x1FFFu;
+  uint32_t h = (uint32_t)e << 10 | q;
+  if (rem > 0x1000u || (rem == 0x1000u && (q & 1u))) h++;  // carry may bump exponent; inf if needed
+  return (uint16_t)(sign | h);
+}
+
+// ---------------------------------------------------------------------------------------
+// Appendix A.2: unnormalised Hadamard matrix by the Sylvester recursion
+//   H'_1 = [1],  H'_{2n} = [[H'_n, H'_n], [H'_n, -H'_n]],   H_n = H'_n / sqrt(n).
+// Written out as a dense matrix (row-major n x n doubles) for the identity checks.
+// ---------------------------------------------------------------------------------------
+int orc_hadamard_matrix(int n, double* H) {
+  if (n < 1 || (n & (n - 1))) return -1;
+  H[0] = 1.0;
+  for (int m = 1; m < n; m *= 2) {
+    // grow the m x m block in the top-left corner (stride n) to 2m x 2m
+    for (int i = 0; i < m; i++)
+      for (int j = 0; j < m; j++) {
+        double v = H[(size_t)i * n + j];
+        H[(size_t)i * n + (j + m)] = v;
+        H[(size_t)(i + m) * n + j] = v;
+        H[(size_t)(i + m) * n + (j + m)] = -v;
+      }
+  }
+  double c = 1.0 / std::sqrt((double)n);
+  for (size_t i = 0; i < (size_t)n * n; i++) H[i] *= c;
+  return 0;
+}
+
+// Exact block rotation in double: y = blockdiag(H_B,...,H_B) x  by the dense definition
+// (O(K*B) work). Every fp16 is a multiple of 2^-24 with magnitude < 2^16, so the +-1 sums are
+// exact in double for B <= 8192; only the final division by sqrt(B) rounds.
+int orc_rotate_exact_f64(const uint16_t* x_f16, int K, int B, double* y) {
+  if (B <= 1) { for (int k = 0; k < K; k++) y[k] = (double)orc_f16_to_f32(x_f16[k]); return 0; }
+  if ((B & (B - 1)) || K % B) return -1;
+  double c = std::sqrt((double)B);
+  for (int b0 = 0; b0 < K; b0 += B) {
+    for (int i = 0; i < B; i++) {
+      double acc = 0.0;
+      for (int j = 0; j < B; j++) {
+        // entry (i,j) of H'_B in Sylvester (natural) order is (-1)^{popcount(i & j)}
+        int p = __builtin_popcount((unsigned)(i & j)) & 1;
+        double xv = (double)orc_f16_to_f32(x_f16[b0 + j]);
+        acc += p ? -xv : xv;
+      }
+      y[b0 + i] = acc / c;
+    }
+  }
+  return 0;
+}
+
+// ---------------------------------------------------------------------------------------
+// Rotation as the quantizer performs it: fp32 fast Walsh-Hadamard butterflies with ascending
+// strides (each add/sub one fp32 round-to-nearest operation), then one fp32 multiply by
+// (float)(1/sqrt(B)). This fixes the rounding order so that the int4 decision below is
+// reproducible bit for bit (the paper's latency table lists an FP32 Hadamard variant; the
+// butterfly order is this build's reading, the paper gives none).
+// ---------------------------------------------------------------------------------------
+static void fwht_f32(float* v, int B) {
+  for (int h = 1; h < B; h *= 2) {
+    for (int i = 0; i < B; i++) {
+      if ((i & h) == 0) {
+        float u = v[i];
+        float w = v[i + h];
+        v[i] = u + w;
+        v[i + h] = u - w;
+      }
+    }
+  }
+  float c = (float)(1.0 / std::sqrt((double)B));
+  for (int i = 0; i < B; i++) v[i] = v[i] * c;
+}
+
+int orc_rotate_f32(const uint16_t* x_f16, int K, int B, float* v) {
+  for (int k = 0; k < K; k++) v[k] = orc_f16_to_f32(x_f16[k]);
+  if (B <= 1) return 0;
+  if ((B & (B - 1)) || K % B) return -1;
+  for (int b0 = 0; b0 < K; b0 += B) fwht_f32(v + b0, B);
+  return 0;
+}
+
+// round half to even of a finite float, as an int
+static int rint_half_even(float r) {
+  double d = (double)r;  // exact
+  double fl = std::floor(d);
+  double diff = d - fl;  // exact for |d| < 2^52
+  long long n = (long long)fl;
+  if (diff > 0.5) n += 1;
+  else if (diff == 0.5 && (n & 1)) n += 1;
+  return (int)n;
+}
+
+// ---------------------------------------------------------------------------------------
+// Per-token symmetric int4 quantization (Section 4.4; Table "Quantization configurations").
+//   v      = rotated token (fp32, above)
+//   amax   = max_k |v_k| over the whole token
+//   s32    = (amax * clip_ratio) / 7        (fp32 multiply, then fp32 IEEE division)
+//   s16    = fp16(s32)  -- the FP16 scalar the paper stores; s = (float)s16 is what divides
+//   q_k    = clamp(round_half_even(v_k / s), -8, 7)      (fp32 IEEE division)
+//   xq[j]  = (q_{2j} & 0xF) | ((q_{2j+1} & 0xF) << 4)    -- low nibble = even index
+// s == 0 (all-zero token, or scale underflow) gives q = 0 everywhere and scale 0.
+// Compile with -ffp-contract=off and without fast-math: every operation is one IEEE fp32 op.
+// q_out (optional, int8 [M][K]) and v_out (optional, float [M][K]) expose intermediates.
+// Returns 0, or -1 on a bad shape, -2 on a non-finite input.
+// ---------------------------------------------------------------------------------------
+int orc_quantize_act(const uint16_t* x_f16, int M, int K, int had_block, float clip_ratio,
+                     uint8_t* xq, uint16_t* scale_f16, int8_t* q_out, float* v_out) {
+  if (M < 1 || K < 2 || (K & 1)) return -1;
+  int B = had_block <= 1 ? 1 : had_block;
+  if ((B & (B - 1)) || K % B) return -1;
+  float* v = (float*)std::malloc(sizeof(float) * (size_t)K);
+  int8_t* q = (int8_t*)std::malloc((size_t)K);
+  for (int m = 0; m < M; m++) {
+    const uint16_t* xm = x_f16 + (size_t)m * K;
+    for (int k = 0; k < K; k++) {
+      float f = orc_f16_to_f32(xm[k]);
+      if (!(f - f == 0.0f)) { std::free(v); std::free(q); return -2; }
+    }
+    orc_rotate_f32(xm, K, B, v);
+    float amax = 0.0f;
+    for (int k = 0; k < K; k++) { float a = std::fabs(v[k]); if (a > amax) amax = a; }
+    float num = amax * clip_ratio;
+    float s32 = num / 7.0f;
+    uint16_t s16 = orc_f32_to_f16(s32);
+    float s = orc_f16_to_f32(s16);
+    for (int k = 0; k < K; k++) {
+      int qi = 0;
+      if (s != 0.0f) {
+        float r = v[k] / s;  // s = +inf (scale overflowed fp16) gives r = 0
+        qi = rint_half_even(r);
+        if (qi < -8) qi = -8;
+        if (qi > 7) qi = 7;
+      }
+      q[k] = (int8_t)qi;
+    }
+    for (int j = 0; j < K / 2; j++)
+      xq[(size_t)m * (K / 2) + j] = (uint8_t)((q[2 * j] & 0xF) | ((q[2 * j + 1] & 0xF) << 4));
+    scale_f16[m] = s16;
+    if (q_out) std::memcpy(q_out + (size_t)m * K, q, (size_t)K);
+    if (v_out) std::memcpy(v_out + (size_t)m * K, v, sizeof(float) * (size_t)K);
+  }
+  std::free(v);
+  std::free(q);
+  return 0;
+}
+
+// Decode packed int4 pairs the way Appendix A.7 ("Online Dequantization") describes:
+// high element by an arithmetic right shift of the signed byte by 4; low element by a left
+// shift by 4 (sign bit of the low nibble to the MSB) then an arithmetic right shift by 4.
+void orc_unpack_act(const uint8_t* xq, size_t nbytes, int8_t* q) {
+  for (size_t j = 0; j < nbytes; j++) {
+    int8_t b = (int8_t)xq[j];
+    int8_t hi = (int8_t)(b >> 4);
+    int8_t lo = (int8_t)((int8_t)(b << 4) >> 4);
+    q[2 * j] = lo;
+    q[2 * j + 1] = hi;
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Weight-code packing: 16 two-bit codes per 32-bit word along the input channel K,
+// code 16w+j in bits [2j, 2j+1] (least-significant first). Returns -3 if a code exceeds 3.
+// ---------------------------------------------------------------------------------------
+int orc_pack_weights(const uint8_t* codes, int N, int K, uint32_t* words) {
+  if (N < 1 || K < 16 || K % 16) return -1;
+  for (size_t i = 0; i < (size_t)N * K; i++) if (codes[i] > 3) return -3;
+  for (int n = 0; n < N; n++)
+    for (int w = 0; w < K / 16; w++) {
+      uint32_t acc = 0;
+      for (int j = 0; j < 16; j++) acc += (uint32_t)codes[(size_t)n * K + 16 * w + j] << (2 * j);
+      words[(size_t)n * (K / 16) + w] = acc;
+    }
+  return 0;
+}
+
+// Independent unpack (division/modulo, not the pack routine's shifts).
+void orc_unpack_weights(const uint32_t* words, int N, int K, uint8_t* codes) {
+  for (int n = 0; n < N; n++)
+    for (int k = 0; k < K; k++) {
+      uint32_t w = words[(size_t)n * (K / 16) + k / 16];
+      uint32_t div = 1;
+      for (int t = 0; t < k % 16; t++) div *= 4;
+      codes[(size_t)n * K + k] = (uint8_t)((w / div) % 4);
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// LUT GEMV (Section 4.4). For token m and output row n:
+//   S_c[m][n] = sum over k with code[n][k] == c of q[m][k]            (exact integers)
+//   y_ref     = s_m * sum_c LUT[n][c] * S_c                          (double)
+//   tol       = 2e-3 * ( s_m * sum_c |LUT[n][c]| * |S_c| ) + 1e-5
+// Outputs: S int32 [M][N][4] (may be NULL), y_ref double [M][N], tol double [M][N] (may be
+// NULL). Returns 0; -1 bad shape; -4 if an S_c does not fit int32.
+// ---------------------------------------------------------------------------------------
+int orc_gemv_w2a4(const uint32_t* words, const uint16_t* lut_f16, const uint8_t* xq,
+                  const uint16_t* scale_f16, int M, int N, int K,
+                  int32_t* S, double* y_ref, double* tol) {
+  if (M < 1 || N < 1 || K < 16 || K % 16) return -1;
+  uint8_t* codes = (uint8_t*)std::malloc((size_t)K);
+  int8_t* q = (int8_t*)std::malloc((size_t)M * K);
+  orc_unpack_act(xq, (size_t)M * (K / 2), q);
+  int rc = 0;
+  for (int n = 0; n < N; n++) {
+    orc_unpack_weights(words + (size_t)n * (K / 16), 1, K, codes);
+    double L[4];
+    for (int c = 0; c < 4; c++) L[c] = (double)orc_f16_to_f32(lut_f16[(size_t)n * 4 + c]);
+    for (int m = 0; m < M; m++) {
+      long long Sc[4] = {0, 0, 0, 0};
+      for (int k = 0; k < K; k++) Sc[codes[k]] += (long long)q[(size_t)m * K + k];
+      double s = (double)orc_f16_to_f32(scale_f16[m]);
+      double acc = 0.0, mag = 0.0;
+      for (int c = 0; c < 4; c++) {
+        if (Sc[c] > 2147483647LL || Sc[c] < -2147483648LL) rc = -4;
+        if (S) S[((size_t)m * N + n) * 4 + c] = (int32_t)Sc[c];
+        acc += L[c] * (double)Sc[c];
+        mag += std::fabs(L[c]) * std::fabs((double)Sc[c]);
+      }
+      y_ref[(size_t)m * N + n] = s * acc;
+      if (tol) tol[(size_t)m * N + n] = 2e-3 * (s * mag) + 1e-5;
+    }
+  }
+  std::free(codes);
+  std::free(q);
+  return rc;
+}
+
+// Direct form of the same product: y = s_m * sum_k LUT[n][code[n][k]] * q[m][k], the sum
+// taken over k in order, in double. Also returns the exact integer value of the sum with
+// every fp16 level scaled by 2^24 (each level is then an integer below 2^41 in magnitude, and
+// the K-term sum stays below 2^60): acc_int[m][n] = sum_k Lint[code]*q.
+int orc_gemv_direct(const uint32_t* words, const uint16_t* lut_f16, const uint8_t* xq,
+                    const uint16_t* scale_f16, int M, int N, int K,
+                    double* y_direct, long long* acc_int) {
+  if (M < 1 || N < 1 || K < 16 || K % 16) return -1;
+  uint8_t* codes = (uint8_t*)std::malloc((size_t)N * K);
+  int8_t* q = (int8_t*)std::malloc((size_t)M * K);
+  orc_unpack_weights(words, N, K, codes);
+  orc_unpack_act(xq, (size_t)M * (K / 2), q);
+  for (int n = 0; n < N; n++) {
+    double L[4];
+    long long Li[4];
+    for (int c = 0; c < 4; c++) {
+      L[c] = (double)orc_f16_to_f32(lut_f16[(size_t)n * 4 + c]);
+      Li[c] = (long long)std::ldexp(L[c], 24);  // exact: fp16 values are multiples of 2^-24
+    }
+    for (int m = 0; m < M; m++) {
+      double acc = 0.0;
+      long long ai = 0;
+      for (int k = 0; k < K; k++) {
+        int c = codes[(size_t)n * K + k];
+        int qq = q[(size_t)m * K + k];
+        acc += L[c] * (double)qq;
+        ai += Li[c] * (long long)qq;
+      }
+      y_direct[(size_t)m * N + n] = (double)orc_f16_to_f32(scale_f16[m]) * acc;
+      if (acc_int) acc_int[(size_t)m * N + n] = ai;
+    }
+  }
+  std::free(codes);
+  std::free(q);
+  return 0;
+}
+
+// Same exact integer, from the per-code sums: sum_c Lint[c] * S_c.
+void orc_percode_int(const uint16_t* lut_f16, const int32_t* S, int M, int N, long long* acc_int) {
+  for (int m = 0; m < M; m++)
+    for (int n = 0; n < N; n++) {
+      long long ai = 0;
+      for (int c = 0; c < 4; c++) {
+        long long Li = (long long)std::ldexp((double)orc_f16_to_f32(lut_f16[(size_t)n * 4 + c]), 24);
+        ai += Li * (long long)S[((size_t)m * N + n) * 4 + c];
+      }
+      acc_int[(size_t)m * N + n] = ai;
+    }
+}
+
+// Dequantized weight matrix (Eq. "deqgrid"): W^[n][k] = LUT[n][code[n][k]], as double.
+void orc_dequant_weights(const uint32_t* words, const uint16_t* lut_f16, int N, int K, double* W) {
+  uint8_t* codes = (uint8_t*)std::malloc((size_t)K);
+  for (int n = 0; n < N; n++) {
+    orc_unpack_weights(words + (size_t)n * (K / 16), 1, K, codes);
+    for (int k = 0; k < K; k++)
+      W[(size_t)n * K + k] = (double)orc_f16_to_f32(lut_f16[(size_t)n * 4 + codes[k]]);
+  }
+  std::free(codes);
+}
+
+}  // extern "C"

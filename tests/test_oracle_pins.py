@@ -1,0 +1,364 @@
+"""Pins for the CPU oracle: every check here compares the oracle with something other than
+itself -- a library routine, a closed form, a hand-written fixture or a brute-force loop."""
+import itertools
+import os
+
+import numpy as np
+import pytest
+import scipy.linalg
+import torch
+
+import oracle
+from paper_2502_15779_b200 import synth
+from helpers import f16_bits
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ----------------------------------------------------------------------------- fp16 <-> fp32
+def test_f16_to_f32_all_patterns_match_numpy():
+    bits = np.arange(65536, dtype=np.uint16)
+    ref = bits.view(np.float16).astype(np.float32)
+    got = np.array([oracle.f16_to_f32(int(b)) for b in bits], dtype=np.float32)
+    both_nan = np.isnan(ref) & np.isnan(got)
+    assert np.array_equal(ref.view(np.uint32)[~both_nan], got.view(np.uint32)[~both_nan])
+
+
+def test_f32_to_f16_matches_numpy_including_ties_and_subnormals():
+    rng = np.random.default_rng(0)
+    vals = [rng.standard_normal(20000).astype(np.float32) * s for s in (1e-7, 1e-4, 1.0, 300.0, 7e4)]
+    # every exact halfway point between neighbouring fp16 values (ties), and +-1 ulp(fp32) around them
+    h = np.arange(0, 0x7C00, dtype=np.uint16).view(np.float16).astype(np.float64)
+    mid = ((h[:-1] + h[1:]) / 2).astype(np.float32)
+    vals += [mid, np.nextafter(mid, np.float32(np.inf)), np.nextafter(mid, np.float32(-np.inf)), -mid]
+    vals += [np.array([0.0, -0.0, 65504.0, 65519.9, 65520.0, 1e9, -1e9, np.inf, -np.inf], dtype=np.float32)]
+    v = np.concatenate(vals).astype(np.float32)
+    with np.errstate(over="ignore"):
+        ref = v.astype(np.float16).view(np.uint16)
+    got = np.array([oracle.f32_to_f16(float(x)) for x in v], dtype=np.uint16)
+    assert np.array_equal(ref, got)
+
+
+# ----------------------------------------------------------------------------- Hadamard
+def test_hadamard4_matches_handwritten_fixture():
+    Hp = np.loadtxt(os.path.join(GOLD, "hadamard4.txt"))
+    assert np.array_equal(oracle.hadamard_matrix(4) * 2.0, Hp)
+
+
+@pytest.mark.parametrize("n", [1, 2, 4, 8, 16, 32, 64])
+def test_hadamard_orthogonal_and_matches_library(n):
+    H = oracle.hadamard_matrix(n)
+    assert np.allclose(H @ H.T, np.eye(n), atol=1e-14)
+    assert np.array_equal(np.sign(H), scipy.linalg.hadamard(n).astype(np.float64))
+    assert np.allclose(np.abs(H), 1.0 / np.sqrt(n))
+    # first row all ones, every other row balanced
+    assert np.all(H[0] > 0)
+    for i in range(1, n):
+        assert (H[i] > 0).sum() == n // 2
+
+
+@pytest.mark.parametrize("B,K", [(2, 8), (4, 16), (16, 64), (64, 128), (128, 384), (256, 256)])
+def test_fwht_equals_matrix_product_bit_exact_on_small_integers(B, K):
+    # integer inputs: every butterfly sum is exact in fp32, so the result must equal the dense
+    # product with the library's Sylvester matrix, then one fp32 multiply by (float)(1/sqrt(B))
+    rng = np.random.default_rng(B)
+    xi = rng.integers(-8, 9, size=K)
+    x = xi.astype(np.float16).view(np.uint16)
+    got = oracle.rotate_f32(x, B)
+    Hp = scipy.linalg.hadamard(B).astype(np.int64)
+    ref_int = np.concatenate([Hp @ xi[b:b + B] for b in range(0, K, B)])
+    ref = ref_int.astype(np.float32) * np.float32(1.0 / np.sqrt(float(B)))
+    assert np.array_equal(got.view(np.uint32), ref.view(np.uint32))
+
+
+def test_fwht_unit_vectors_give_columns():
+    B = 32
+    Hp = scipy.linalg.hadamard(B)
+    for j in (0, 1, 5, 31):
+        e = np.zeros(B, dtype=np.float16)
+        e[j] = 1.0
+        got = oracle.rotate_f32(e.view(np.uint16), B)
+        assert np.array_equal(got, Hp[:, j].astype(np.float32) * np.float32(1 / np.sqrt(32.0)))
+
+
+@pytest.mark.parametrize("B", [4, 16, 64, 256])
+def test_rotation_is_involution_when_scale_is_a_power_of_two(B):
+    # sqrt(B) is a power of two here and inputs are small integers, so both passes are exact
+    rng = np.random.default_rng(1)
+    xi = rng.integers(-4, 5, size=B)
+    once = oracle.rotate_f32(xi.astype(np.float16).view(np.uint16), B)
+    once16 = once.astype(np.float16)
+    assert np.array_equal(once16.astype(np.float32), once)  # representable in fp16
+    twice = oracle.rotate_f32(once16.view(np.uint16), B)
+    assert np.array_equal(twice, xi.astype(np.float32))
+
+
+@pytest.mark.parametrize("B,K", [(128, 1280), (2048, 2048), (8192, 8192)])
+def test_fp32_butterflies_stay_within_rounding_bound_of_exact_rotation(B, K):
+    x = synth.make_activations(1, K, seed=11)
+    xb = f16_bits(x)[0]
+    v32 = oracle.rotate_f32(xb, B).astype(np.float64)
+    exact = oracle.rotate_exact_f64(xb.reshape(1, K), B)[0]
+    # independent of both: dense product with the library matrix in float64
+    Hp = scipy.linalg.hadamard(B).astype(np.float64) if B <= 2048 else None
+    if Hp is not None:
+        xd = xb.view(np.float16).astype(np.float64)
+        lib = np.concatenate([Hp @ xd[b:b + B] for b in range(0, K, B)]) / np.sqrt(B)
+        assert np.allclose(exact, lib, rtol=0, atol=1e-9)
+    # error of log2(B) fp32 additions + 1 multiply, each <= 2^-24 relative to running magnitude
+    l1 = np.abs(xb.view(np.float16).astype(np.float64)).reshape(-1, B).sum(axis=1).repeat(B) / np.sqrt(B)
+    bound = (np.log2(B) + 2) * 2.0 ** -24 * l1
+    assert np.all(np.abs(v32 - exact) <= bound)
+    # Parseval: the rotation preserves the Euclidean norm
+    assert np.isclose(np.linalg.norm(exact), np.linalg.norm(xb.view(np.float16).astype(np.float64)), rtol=1e-12)
+
+
+# ----------------------------------------------------------------------------- quantizer
+def _load_hand_cases():
+    xs, qs = [], []
+    for line in open(os.path.join(GOLD, "quant_hand_cases.txt")):
+        if line.startswith("#") or "->" not in line:
+            continue
+        a, b = line.split("->")
+        xs.append(float(a))
+        qs.append(int(b))
+    return np.array(xs), np.array(qs)
+
+
+def test_quantizer_hand_cases_from_fixture():
+    xs, qs = _load_hand_cases()
+    K = 32
+    x = np.zeros((1, K), dtype=np.float16)
+    x[0, :len(xs)] = xs
+    assert np.array_equal(x[0, :len(xs)].astype(np.float64), xs)  # fixture values are exact fp16
+    r = oracle.quantize_act(x.view(np.uint16), had_block=1, clip_ratio=1.0)
+    assert r["scale"][0] == np.float16(1.0).view(np.uint16)
+    assert np.array_equal(r["q"][0, :len(xs)], qs)
+    assert np.all(r["q"][0, len(xs):] == 0)
+
+
+def test_quantizer_scale_matches_library_arithmetic_and_absmax_maps_to_7():
+    for seed in range(5):
+        x = synth.make_activations(3, 256, seed=seed)
+        r = oracle.quantize_act(f16_bits(x), had_block=1, clip_ratio=1.0)
+        xf = x.numpy().astype(np.float32)
+        amax = np.abs(xf).max(axis=1)
+        s16 = (amax / np.float32(7.0)).astype(np.float16)
+        assert np.array_equal(r["scale"], s16.view(np.uint16))
+        q = r["q"]
+        assert np.all(np.abs(q).max(axis=1) == 7)
+        idx = np.abs(xf).argmax(axis=1)
+        assert np.all(np.abs(q[np.arange(3), idx]) == 7)
+        # library restatement: numpy float32 division + rint (round half to even)
+        ref = np.clip(np.rint(xf / s16.astype(np.float32)[:, None]), -8, 7).astype(np.int8)
+        assert np.array_equal(q, ref)
+
+
+def test_quantizer_clip_ratio_below_one_reaches_minus8_never_plus8():
+    x = np.zeros((2, 16), dtype=np.float16)
+    x[0, 0], x[0, 1] = -7.0, 7.0
+    x[1, 0], x[1, 1] = 7.0, -6.0
+    r = oracle.quantize_act(x.view(np.uint16), had_block=1, clip_ratio=0.9)
+    assert r["q"][0, 0] == -8 and r["q"][0, 1] == 7
+    assert r["q"][1, 0] == 7 and r["q"][1, 1] == -7  # -6/0.9 = -6.67 -> -7
+    assert r["q"].min() >= -8 and r["q"].max() <= 7
+
+
+def test_quantizer_zero_token_and_nibble_layout():
+    x = np.zeros((2, 32), dtype=np.float16)
+    x[1, :] = np.arange(32) % 15 - 7
+    r = oracle.quantize_act(x.view(np.uint16), had_block=1, clip_ratio=1.0)
+    assert r["scale"][0] == 0 and np.all(r["xq"][0] == 0) and np.all(r["q"][0] == 0)
+    q = r["q"][1].astype(np.int32)
+    assert np.array_equal(q, np.arange(32) % 15 - 7)  # scale is exactly 1
+    # low nibble = even index, high nibble = odd index, two's complement
+    expect = ((q[0::2] & 0xF) | ((q[1::2] & 0xF) << 4)).astype(np.uint8)
+    assert np.array_equal(r["xq"][1], expect)
+    # decode with a different formula than the oracle's shift recipe: ((n ^ 8) - 8)
+    lo = ((r["xq"][1].astype(np.int32) & 0xF) ^ 8) - 8
+    hi = ((r["xq"][1].astype(np.int32) >> 4) ^ 8) - 8
+    dec = oracle.unpack_act(r["xq"][1:2])[0]
+    assert np.array_equal(dec[0::2], lo) and np.array_equal(dec[1::2], hi)
+
+
+def test_quantizer_identity_rotation_vs_hadamard_and_exact_rotation_agree_on_codes():
+    # with rotation: quantizing the oracle's rotated vector by numpy must give the same codes
+    K, B = 512, 128
+    x = synth.make_activations(2, K, seed=3)
+    r = oracle.quantize_act(f16_bits(x), had_block=B, clip_ratio=1.0)
+    v = r["v"]
+    amax = np.abs(v).max(axis=1)
+    s16 = (amax / np.float32(7.0)).astype(np.float16)
+    assert np.array_equal(r["scale"], s16.view(np.uint16))
+    ref = np.clip(np.rint(v / s16.astype(np.float32)[:, None]), -8, 7).astype(np.int8)
+    assert np.array_equal(r["q"], ref)
+    # and the rotated vector is close to the exact one (so codes differ from the exact-rotation
+    # codes only where the exact value sits within rounding distance of a decision boundary)
+    exact = oracle.rotate_exact_f64(f16_bits(x), B)
+    qe = np.clip(np.rint(exact / s16.astype(np.float64)[:, None]), -8, 7)
+    frac = np.abs(exact / s16.astype(np.float64)[:, None] - np.floor(exact / s16.astype(np.float64)[:, None]) - 0.5)
+    differs = qe != r["q"]
+    assert np.all(frac[differs] < 1e-4)
+    assert differs.mean() < 1e-3
+
+
+def test_quantizer_rejects_nonfinite():
+    x = np.zeros((1, 16), dtype=np.float16)
+    x[0, 3] = np.inf
+    with pytest.raises(ValueError):
+        oracle.quantize_act(x.view(np.uint16), 1, 1.0)
+
+
+# ----------------------------------------------------------------------------- packing
+def test_pack_single_code_words_and_roundtrip():
+    for j in range(16):
+        codes = np.zeros((1, 16), dtype=np.uint8)
+        codes[0, j] = 3
+        assert oracle.pack_weights(codes)[0, 0] == np.uint32(3 << (2 * j))
+    rng = np.random.default_rng(5)
+    codes = rng.integers(0, 4, size=(7, 96), dtype=np.uint8)
+    words = oracle.pack_weights(codes)
+    # independent numpy restatement of the layout
+    ref = (codes.reshape(7, 6, 16).astype(np.uint64) << (2 * np.arange(16, dtype=np.uint64))).sum(axis=2)
+    assert np.array_equal(words, ref.astype(np.uint32))
+    assert np.array_equal(oracle.unpack_weights(words), codes)
+
+
+def test_pack_bytes_decode_with_shift_and_mask_recipe():
+    # Appendix A.7 decodes four codes per byte with shifts and the mask 0x03; in this layout the
+    # first code sits in the LOW two bits (shifts 0,2,4,6), bytes in little-endian order.
+    rng = np.random.default_rng(6)
+    codes = rng.integers(0, 4, size=(3, 64), dtype=np.uint8)
+    by = oracle.pack_weights(codes).view(np.uint8).reshape(3, 16)
+    dec = np.stack([(by >> s) & 0x03 for s in (0, 2, 4, 6)], axis=2).reshape(3, 64)
+    assert np.array_equal(dec, codes)
+
+
+def test_pack_rejects_codes_above_3():
+    codes = np.zeros((2, 16), dtype=np.uint8)
+    codes[1, 7] = 4
+    with pytest.raises(ValueError):
+        oracle.pack_weights(codes)
+
+
+def test_lut_lookup_of_unpacked_codes_reproduces_dequantized_weights():
+    codes, lut = synth.make_layer(24, 256, 128, "rotated_laplace", seed=9)
+    words = oracle.pack_weights(codes.numpy())
+    Wd = oracle.dequant_weights(words, f16_bits(lut))
+    ref = np.take_along_axis(lut.numpy().astype(np.float64), codes.numpy().astype(np.int64), axis=1)
+    assert np.array_equal(Wd, ref)
+    # the generator assigned every weight to a level: all dequantized values are LUT levels
+    assert set(np.unique(Wd[0])) <= set(lut.numpy()[0].astype(np.float64))
+
+
+# ----------------------------------------------------------------------------- GEMV
+def _problem(N, K, M, seed, kind="uniform", B=1):
+    codes, lut = synth.make_layer(N, K, B, kind, seed)
+    x = synth.make_activations(M, K, seed)
+    qa = oracle.quantize_act(f16_bits(x), B, 1.0)
+    words = oracle.pack_weights(codes.numpy())
+    return codes.numpy(), lut, words, qa
+
+
+def _brute(codes, lut, q, scale_bits):
+    """Pure-Python triple loop straight from the definition."""
+    M, K = q.shape
+    N = codes.shape[0]
+    S = np.zeros((M, N, 4), dtype=np.int64)
+    y = np.zeros((M, N))
+    lutf = lut.numpy().astype(np.float64)
+    for m in range(M):
+        s = float(scale_bits[m:m + 1].view(np.float16)[0])
+        for n in range(N):
+            acc = 0.0
+            for k in range(K):
+                c = int(codes[n, k])
+                S[m, n, c] += int(q[m, k])
+            for c in range(4):
+                acc += lutf[n, c] * float(S[m, n, c])
+            y[m, n] = s * acc
+    return S, y
+
+
+@pytest.mark.parametrize("N,K,M,zero_from", [(8, 16, 1, 8), (16, 32, 1, None), (16, 32, 3, None)])
+def test_gemv_brute_force_small(N, K, M, zero_from):
+    # the 8x8 case is embedded in one packed word: codes beyond k=8 meet zero activations
+    codes, lut, words, qa = _problem(N, K, M, seed=N + K)
+    xq, q = qa["xq"].copy(), qa["q"].copy()
+    if zero_from is not None:
+        q[:, zero_from:] = 0
+        xq[:, zero_from // 2:] = 0
+    r = oracle.gemv_w2a4(words, f16_bits(lut), xq, qa["scale"])
+    S, y = _brute(codes, lut, q, qa["scale"])
+    assert np.array_equal(r["S"], S)
+    assert np.allclose(r["y"], y, rtol=1e-14, atol=0)
+    if zero_from is not None:
+        S8, y8 = _brute(codes[:, :zero_from], lut, q[:, :zero_from], qa["scale"])
+        assert np.array_equal(S[..., 1:], S8[..., 1:]) and np.allclose(y, y8)
+
+
+def test_gemv_percode_sums_add_up_and_equal_codes_rows():
+    codes, lut, words, qa = _problem(32, 256, 2, seed=4)
+    codes[5, :] = 2
+    codes[6, :] = 0
+    words = oracle.pack_weights(codes)
+    r = oracle.gemv_w2a4(words, f16_bits(lut), qa["xq"], qa["scale"])
+    tot = qa["q"].astype(np.int64).sum(axis=1)
+    assert np.array_equal(r["S"].sum(axis=2), np.repeat(tot[:, None], 32, axis=1))
+    assert np.array_equal(r["S"][:, 5, 2], tot) and np.all(r["S"][:, 5, [0, 1, 3]] == 0)
+    assert np.array_equal(r["S"][:, 6, 0], tot)
+
+
+@pytest.mark.parametrize("N,K,M,B,kind", [(64, 512, 1, 128, "rotated_laplace"), (40, 2048, 2, 2048, "rotated_laplace"),
+                                          (33, 192, 3, 64, "uniform")])
+def test_direct_form_equals_percode_form_as_exact_integers(N, K, M, B, kind):
+    codes, lut, words, qa = _problem(N, K, M, seed=7, kind=kind, B=B)
+    lb = f16_bits(lut)
+    r = oracle.gemv_w2a4(words, lb, qa["xq"], qa["scale"])
+    d = oracle.gemv_direct(words, lb, qa["xq"], qa["scale"])
+    assert np.array_equal(d["acc_int"], oracle.percode_int(lb, r["S"]))
+    # numpy restatement of the scaled-integer direct sum (fp16 levels times 2^24 are integers)
+    Li = np.round(np.ldexp(lut.numpy().astype(np.float64), 24)).astype(np.int64)
+    Wi = np.take_along_axis(Li, codes.astype(np.int64), axis=1)
+    assert np.array_equal(d["acc_int"], qa["q"].astype(np.int64) @ Wi.T)
+    assert np.allclose(d["y"], r["y"], rtol=1e-12, atol=1e-300)
+
+
+def test_affine_and_constant_lut_reduce_to_plain_integer_gemv():
+    N, K, M = 48, 320, 2
+    codes, lut, words, qa = _problem(N, K, M, seed=12, kind="uniform", B=64)
+    a, d = 0.125, 0.03125  # exactly representable
+    lut_aff = torch.tensor([[a + c * d for c in range(4)]] * N, dtype=torch.float16)
+    r = oracle.gemv_w2a4(words, f16_bits(lut_aff), qa["xq"], qa["scale"])
+    q = qa["q"].astype(np.int64)
+    s = qa["scale"].view(np.float16).astype(np.float64)
+    ref = s[:, None] * (a * q.sum(axis=1)[:, None] + d * (q @ codes.astype(np.int64).T))
+    assert np.allclose(r["y"], ref, rtol=1e-13, atol=0)
+    lut_c = torch.full((N, 4), 0.5, dtype=torch.float16)
+    r2 = oracle.gemv_w2a4(words, f16_bits(lut_c), qa["xq"], qa["scale"])
+    assert np.allclose(r2["y"], s[:, None] * 0.5 * q.sum(axis=1)[:, None] * np.ones((1, N)), rtol=1e-13)
+
+
+def test_gemv_equals_dense_matmul_with_dequantized_weights():
+    N, K, M = 64, 1024, 3
+    codes, lut, words, qa = _problem(N, K, M, seed=21, kind="rotated_laplace", B=128)
+    r = oracle.gemv_w2a4(words, f16_bits(lut), qa["xq"], qa["scale"])
+    Wd = np.take_along_axis(lut.numpy().astype(np.float64), codes.astype(np.int64), axis=1)  # [N][K]
+    s = qa["scale"].view(np.float16).astype(np.float64)
+    ref = (qa["q"].astype(np.float64) * s[:, None]) @ Wd.T
+    assert np.allclose(r["y"], ref, rtol=1e-11, atol=1e-15)
+    mag = s[:, None] * (np.abs(lut.numpy().astype(np.float64))[None] * np.abs(r["S"])).sum(axis=2)
+    assert np.allclose(r["tol"], 2e-3 * mag + 1e-5, rtol=1e-12)
+
+
+def test_planted_mistakes_are_caught_by_the_brute_force_pin():
+    # a transposed nibble order or a reversed code order in the inputs changes the result: the pin
+    # is sensitive to exactly the mistakes a wrong index would make
+    codes, lut, words, qa = _problem(16, 32, 1, seed=3)
+    r = oracle.gemv_w2a4(words, f16_bits(lut), qa["xq"], qa["scale"])
+    swapped = ((qa["xq"] >> 4) | (qa["xq"] << 4)).astype(np.uint8)
+    r_sw = oracle.gemv_w2a4(words, f16_bits(lut), swapped, qa["scale"])
+    assert not np.array_equal(r["S"], r_sw["S"])
+    rev = oracle.pack_weights(np.ascontiguousarray(codes.reshape(16, 2, 16)[:, :, ::-1].reshape(16, 32)))
+    r_rev = oracle.gemv_w2a4(rev, f16_bits(lut), qa["xq"], qa["scale"])
+    assert not np.array_equal(r["S"], r_rev["S"])
