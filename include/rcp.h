@@ -1,0 +1,114 @@
+/*
+ * rcp.h -- C ABI of the B200 (sm_100a) library for the decode-time W2A4 hot path of RCP
+ * ("Rotate, Clip, and Partition", arXiv 2502.15779).
+ *
+ * Notation (Section 4.4 of the paper calls the input channels C and the output channels H):
+ *   K = input channels, N = output rows, M = tokens (1..16, the decode / skinny regime).
+ *
+ * Tensor formats (Section 4.4 "Fast GEMV via Latency Hiding", Appendix A.7):
+ *   words  uint32 [N][K/16]  2-bit weight codes W_q, 16 per word along K, code 16w+j in bits
+ *                            [2j, 2j+1] (least significant first).
+ *   lut    fp16   [N][4]     dequantization grid W^_0..W^_3 of Eq. "deqgrid", one per output row.
+ *   xq     uint8  [M][K/2]   int4 activations X_q, two per byte: low nibble = even k, high
+ *                            nibble = odd k, two's complement.
+ *   scale  fp16   [M]        per-token activation scale S.
+ *   y      fp16   [M][N]     output O = S * X_q * LUT[W_q].
+ *
+ * Unless a function says otherwise every pointer is a DEVICE pointer owned by the caller, 16-byte
+ * aligned, valid on the current device; `stream` is a cudaStream_t passed as void* (NULL = the
+ * default stream). Calls are asynchronous on that stream and allocate no device memory.
+ * Every function returns RCP_OK or a negative status; nothing is thrown across this boundary.
+ */
+#ifndef RCP_H_
+#define RCP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  RCP_OK = 0,
+  RCP_ERR_NULL = -1,      /* a required pointer is NULL */
+  RCP_ERR_SHAPE = -2,     /* K % 64 != 0, N < 1, M outside 1..16, bad had_block, ... */
+  RCP_ERR_ALIGN = -3,     /* a pointer is not 16-byte aligned */
+  RCP_ERR_CODE = -4,      /* rcp_pack_weights met a code above 3 */
+  RCP_ERR_WORKSPACE = -5, /* workspace missing */
+  RCP_ERR_CUDA = -6,      /* a CUDA call failed; see rcp_last_cuda_error() */
+  RCP_ERR_VARIANT = -7,   /* unknown kernel variant, or the variant does not support the shape */
+  RCP_ERR_LIMIT = -8      /* size beyond a fixed capacity of the entry point */
+};
+
+/* Text for a status code. Never NULL. */
+const char* rcp_status_str(int status);
+
+/* cudaError_t (as int) of the last failed CUDA call made by this library on this thread. */
+int rcp_last_cuda_error(void);
+
+/*
+ * Weight packing (Section 4.4: W_q is pre-computed offline and stored sub-byte packed along the
+ * input channel). codes: uint8 [N][K], each in {0,1,2,3}. words: uint32 [N][K/16].
+ * K % 64 == 0. Synchronizes the stream before returning so that RCP_ERR_CODE can be reported;
+ * on RCP_ERR_CODE the contents of `words` are unspecified.
+ */
+int rcp_pack_weights(const uint8_t* codes, int N, int K, uint32_t* words, void* stream);
+
+/*
+ * Per-token activation quantization with the online rotation fused in front
+ * (rotation: Section 2.1 / Fig. "rotation", R4 and R_H'; Hadamard matrix: Appendix A.2;
+ *  quantizer: Section 4.4 tensor formats, Table "Quantization configurations": symmetric,
+ *  per-token, 4 bit).
+ *   x_f16      fp16 [M][K] row-major, finite values.
+ *   had_block  0 or 1: no rotation. Otherwise a power of two <= 8192 dividing K: every block of
+ *              had_block consecutive elements is multiplied by the normalized Sylvester Hadamard
+ *              matrix, computed as fp32 butterflies with ascending strides and one final fp32
+ *              multiply by 1/sqrt(had_block).
+ *   clip_ratio scale = fp16( (max_k |x_rot| * clip_ratio) / 7 ); q = clamp(rne(x_rot/scale),-8,7).
+ *              The paper's table uses 0.9; the benchmark configurations use 1.0.
+ *   xq, scale  outputs as described at the top. An all-zero token gives scale 0 and q = 0.
+ * Constraints: 1 <= M <= 65535, K % 64 == 0, 64 <= K <= 65536.
+ */
+int rcp_quantize_act(const void* x_f16, int M, int K, int had_block, float clip_ratio,
+                     uint8_t* xq, void* scale_f16, void* stream);
+
+/*
+ * Kernel variants of the LUT GEMV (all compute the same result).
+ *   RCP_GEMV_AUTO    library picks.
+ *   RCP_GEMV_SIMPLE  one warp per output row, scalar decode; also the variant behind S_dbg.
+ *   RCP_GEMV_DP4A    CUDA-core path: masked code planes times int8 activations with dp4a.
+ *   RCP_GEMV_MMA     masked code planes as the A operand of int8 mma.sync, weights streamed
+ *                    through a TMA/mbarrier shared-memory ring, work split evenly over the SMs.
+ */
+enum { RCP_GEMV_AUTO = 0, RCP_GEMV_SIMPLE = 1, RCP_GEMV_DP4A = 2, RCP_GEMV_MMA = 3 };
+
+/*
+ * Bytes of caller-provided scratch rcp_gemv_w2a4 needs for this shape (0 if none). The scratch
+ * must be zero-filled once after allocation; every call leaves it zero-filled again, so one
+ * buffer can serve any sequence of calls that do not overlap in time. Returns 0 on bad shapes.
+ */
+size_t rcp_gemv_workspace_bytes(int M, int N, int K);
+
+/*
+ * LUT GEMV / skinny GEMM (Section 4.4, Eq. "deqgrid"):
+ *   S_c[m][n] = sum over k with code[n][k] == c of q[m][k]       (exact integers)
+ *   y[m][n]   = fp16( scale[m] * sum_c lut[n][c] * S_c[m][n] )   (fp32 arithmetic)
+ * Constraints: 1 <= M <= 16, N >= 1, K % 64 == 0, 64 <= K <= 65536.
+ *   workspace  rcp_gemv_workspace_bytes(M,N,K) bytes, see above; may be NULL if that is 0.
+ *   S_dbg      NULL in production. Otherwise int32 [M][N][4] receives S_c (runs the SIMPLE variant).
+ * Never synchronizes.
+ */
+int rcp_gemv_w2a4(const uint32_t* words, const void* lut_f16, const uint8_t* xq,
+                  const void* scale_f16, int M, int N, int K, void* y_f16, void* workspace,
+                  int32_t* S_dbg, void* stream);
+
+/* Same, with the kernel variant chosen by the caller (for benchmarks and profiles). */
+int rcp_gemv_w2a4_variant(int variant, const uint32_t* words, const void* lut_f16,
+                          const uint8_t* xq, const void* scale_f16, int M, int N, int K,
+                          void* y_f16, void* workspace, int32_t* S_dbg, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RCP_H_ */

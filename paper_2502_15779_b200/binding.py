@@ -1,0 +1,129 @@
+"""Thin Python binding over the C ABI declared in include/rcp.h.
+
+Argument marshalling only: tensors are allocated by torch (device memory and streams), every
+computation runs in the library's CUDA kernels.  There is no fallback: if the shared library
+is missing or a call fails, an exception is raised.
+"""
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "librcp_w2a4.so")
+
+GEMV_AUTO, GEMV_SIMPLE, GEMV_DP4A, GEMV_MMA = 0, 1, 2, 3
+VARIANTS = {"auto": GEMV_AUTO, "simple": GEMV_SIMPLE, "dp4a": GEMV_DP4A, "mma": GEMV_MMA}
+
+_lib = None
+
+
+class RcpError(RuntimeError):
+    def __init__(self, fn, status, text, cuda_error):
+        super().__init__(f"{fn} failed: {text} (status {status}, cuda error {cuda_error})")
+        self.status = status
+
+
+def lib():
+    """Loads the shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} not found: build it with `python -m paper_2502_15779_b200.build` "
+                "(there is no CPU or PyTorch fallback)")
+        L = C.CDLL(LIB_PATH)
+        vp, i, u64 = C.c_void_p, C.c_int, C.c_size_t
+        L.rcp_status_str.restype = C.c_char_p
+        L.rcp_status_str.argtypes = [i]
+        L.rcp_last_cuda_error.restype = i
+        L.rcp_pack_weights.restype = i
+        L.rcp_pack_weights.argtypes = [vp, i, i, vp, vp]
+        L.rcp_quantize_act.restype = i
+        L.rcp_quantize_act.argtypes = [vp, i, i, i, C.c_float, vp, vp, vp]
+        L.rcp_gemv_workspace_bytes.restype = u64
+        L.rcp_gemv_workspace_bytes.argtypes = [i, i, i]
+        L.rcp_gemv_w2a4.restype = i
+        L.rcp_gemv_w2a4.argtypes = [vp, vp, vp, vp, i, i, i, vp, vp, vp, vp]
+        L.rcp_gemv_w2a4_variant.restype = i
+        L.rcp_gemv_w2a4_variant.argtypes = [i, vp, vp, vp, vp, i, i, i, vp, vp, vp, vp]
+        _lib = L
+    return _lib
+
+
+def _check(fn, status):
+    if status != 0:
+        L = lib()
+        raise RcpError(fn, status, L.rcp_status_str(status).decode(), L.rcp_last_cuda_error())
+
+
+def _ptr(t):
+    return C.c_void_p(t.data_ptr()) if t is not None else None
+
+
+def _stream(t):
+    return C.c_void_p(torch.cuda.current_stream(t.device).cuda_stream)
+
+
+def _dev(t, dtype, name):
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError(f"{name}: expected a contiguous CUDA tensor of dtype {dtype}")
+    return t
+
+
+def rcp_pack_weights(codes: torch.Tensor, out: torch.Tensor = None) -> torch.Tensor:
+    """codes uint8 [N][K] in {0..3} -> words int32 [N][K/16] (bit pattern of the uint32 words)."""
+    _dev(codes, torch.uint8, "codes")
+    N, K = codes.shape
+    words = out if out is not None else torch.empty((N, K // 16), dtype=torch.int32, device=codes.device)
+    with torch.cuda.device(codes.device):
+        _check("rcp_pack_weights", lib().rcp_pack_weights(_ptr(codes), N, K, _ptr(words), _stream(codes)))
+    return words
+
+
+def rcp_quantize_act(x: torch.Tensor, had_block: int, clip_ratio: float = 1.0, xq=None, scale=None):
+    """x fp16 [M][K] -> (xq uint8 [M][K/2], scale fp16 [M])."""
+    _dev(x, torch.float16, "x")
+    M, K = x.shape
+    if xq is None:
+        xq = torch.empty((M, K // 2), dtype=torch.uint8, device=x.device)
+    if scale is None:
+        scale = torch.empty((M,), dtype=torch.float16, device=x.device)
+    with torch.cuda.device(x.device):
+        _check("rcp_quantize_act",
+               lib().rcp_quantize_act(_ptr(x), M, K, int(had_block), float(clip_ratio), _ptr(xq), _ptr(scale),
+                                      _stream(x)))
+    return xq, scale
+
+
+def rcp_gemv_workspace_bytes(M: int, N: int, K: int) -> int:
+    return int(lib().rcp_gemv_workspace_bytes(M, N, K))
+
+
+def make_workspace(M: int, N: int, K: int, device) -> torch.Tensor:
+    """Zero-filled scratch for rcp_gemv_w2a4 (at least 16 bytes so that a pointer always exists)."""
+    n = max(16, rcp_gemv_workspace_bytes(M, N, K))
+    return torch.zeros((n + 3) // 4, dtype=torch.int32, device=device)
+
+
+def rcp_gemv_w2a4(words, lut, xq, scale, y=None, workspace=None, S_dbg=None, variant="auto"):
+    """words int32 [N][K/16], lut fp16 [N][4], xq uint8 [M][K/2], scale fp16 [M] -> y fp16 [M][N]."""
+    _dev(words, torch.int32, "words")
+    _dev(lut, torch.float16, "lut")
+    _dev(xq, torch.uint8, "xq")
+    _dev(scale, torch.float16, "scale")
+    N, W = words.shape
+    K = W * 16
+    M = xq.shape[0]
+    if xq.shape != (M, K // 2) or lut.shape != (N, 4) or scale.shape != (M,):
+        raise ValueError("shape mismatch between words, lut, xq and scale")
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.float16, device=words.device)
+    if workspace is None and rcp_gemv_workspace_bytes(M, N, K) > 0:
+        workspace = make_workspace(M, N, K, words.device)
+    v = VARIANTS[variant] if isinstance(variant, str) else int(variant)
+    with torch.cuda.device(words.device):
+        _check("rcp_gemv_w2a4",
+               lib().rcp_gemv_w2a4_variant(v, _ptr(words), _ptr(lut), _ptr(xq), _ptr(scale), M, N, K, _ptr(y),
+                                           _ptr(workspace), _ptr(S_dbg), _stream(words)))
+    return y
