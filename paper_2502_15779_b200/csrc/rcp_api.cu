@@ -1,10 +1,12 @@
 // C ABI of the RCP W2A4 library: argument validation, launch configuration, status codes.
 #include "../../include/rcp.h"
 
+#include <algorithm>
 #include <cmath>
 
 #include "common.cuh"
 #include "gemv_simple.cuh"
+#include "gemv_stream.cuh"
 #include "pack.cuh"
 #include "quantize_act.cuh"
 
@@ -28,6 +30,113 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 bool k_ok(int K) { return K >= 64 && K <= rcp::kMaxK && K % 64 == 0; }
 
 __device__ int g_pack_bad;  // set by pack_weights_kernel when it meets a code above 3
+
+// ---------------------------------------------------------------------------------------------
+// Streaming GEMV: launch plan shared by rcp_gemv_workspace_bytes and the launcher.
+struct StreamPlan {
+  int ntiles, nchunks, ncol, supers, ch_per_super, stages;
+  size_t smem, ws_count_off, ws_sum_off, ws_bytes;
+};
+
+constexpr size_t kSmemMax = 232448;          // 227 KB of dynamic shared memory per CTA on sm_100
+constexpr size_t kExpandBudget = 64 * 1024;  // expanded activations kept resident per CTA
+
+StreamPlan make_plan(int M, int N, int K) {
+  StreamPlan pl;
+  pl.ntiles = (N + rcp::kTileRows - 1) / rcp::kTileRows;
+  pl.nchunks = (K / 16 + rcp::kChunkWords - 1) / rcp::kChunkWords;
+  pl.ncol = 1;
+  while (pl.ncol < M) pl.ncol *= 2;
+  const int per_chunk = rcp::kChunkWords * 16 * pl.ncol;  // bytes of expanded activations per K chunk
+  const int max_ch = (int)std::max<size_t>(1, kExpandBudget / per_chunk);
+  pl.supers = (pl.nchunks + max_ch - 1) / max_ch;
+  pl.ch_per_super = (pl.nchunks + pl.supers - 1) / pl.supers;
+  pl.supers = (pl.nchunks + pl.ch_per_super - 1) / pl.ch_per_super;
+  const size_t bs = (size_t)pl.ch_per_super * per_chunk;
+  const size_t fixed = 1024 + 512 + bs;
+  pl.stages = (int)std::min<size_t>(rcp::kMaxStages, (kSmemMax - fixed) / rcp::kStageBytes);
+  pl.smem = fixed + (size_t)pl.stages * rcp::kStageBytes;
+  pl.ws_count_off = 16;
+  const size_t cnt = (size_t)pl.ntiles * rcp::kConsumerWarps * 4;
+  pl.ws_sum_off = pl.ws_count_off + ((cnt + 15) / 16) * 16;
+  pl.ws_bytes = pl.ws_sum_off + (size_t)pl.ntiles * rcp::kTileRows * M * 3 * 4;
+  return pl;
+}
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+      n = 148;
+  }
+  return n;
+}
+
+template <int MT, int MODE>
+int launch_stream_t(const CUtensorMap& map, const rcp::StreamParams& sp, const StreamPlan& pl, cudaStream_t st) {
+  static bool attr_set = false;
+  auto kern = rcp::gemv_stream_kernel<MT, MODE>;
+  if (!attr_set) {
+    RCP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax));
+    attr_set = true;
+  }
+  const int gx = std::max(1, sm_count() / pl.supers);
+  kern<<<dim3(gx, pl.supers), rcp::kStreamThreads, pl.smem, st>>>(map, sp);
+  RCP_CUDA(cudaGetLastError());
+  return RCP_OK;
+}
+
+int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const uint8_t* xq, const void* scale_f16,
+                  int M, int N, int K, void* y_f16, void* workspace, cudaStream_t st) {
+  if (!workspace) return RCP_ERR_WORKSPACE;
+  if (!aligned16(workspace)) return RCP_ERR_ALIGN;
+  if (mode != rcp::kModeMma && M > 2) return RCP_ERR_VARIANT;
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (!enc) return cuda_fail(cudaErrorNotSupported);
+  const StreamPlan pl = make_plan(M, N, K);
+  CUtensorMap map;
+  const cuuint64_t gdim[2] = {(cuuint64_t)(K / 16), (cuuint64_t)N};
+  const cuuint64_t gstride[1] = {(cuuint64_t)(K / 4)};
+  const cuuint32_t box[2] = {(cuuint32_t)rcp::kChunkWords, (cuuint32_t)rcp::kTileRows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = enc(&map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t*>(words), gdim, gstride, box,
+                         estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue);
+  rcp::StreamParams sp;
+  sp.lut = static_cast<const uint2*>(lut_f16);
+  sp.xq = xq;
+  sp.scale = static_cast<const __half*>(scale_f16);
+  sp.y = static_cast<__half*>(y_f16);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  sp.ws_status = reinterpret_cast<int32_t*>(ws);
+  sp.ws_count = reinterpret_cast<uint32_t*>(ws + pl.ws_count_off);
+  sp.ws_sum = reinterpret_cast<int32_t*>(ws + pl.ws_sum_off);
+  sp.M = M; sp.N = N; sp.K = K;
+  sp.ntiles = pl.ntiles; sp.nchunks = pl.nchunks; sp.ch_per_super = pl.ch_per_super;
+  sp.stages = pl.stages; sp.ncol = pl.ncol;
+  if (mode == rcp::kModeHybrid) return launch_stream_t<1, rcp::kModeHybrid>(map, sp, pl, st);
+  if (mode == rcp::kModeDp4a) return launch_stream_t<1, rcp::kModeDp4a>(map, sp, pl, st);
+  if (M <= 8) return launch_stream_t<1, rcp::kModeMma>(map, sp, pl, st);
+  return launch_stream_t<2, rcp::kModeMma>(map, sp, pl, st);
+}
 
 }  // namespace
 
@@ -103,7 +212,7 @@ int rcp_quantize_act(const void* x_f16, int M, int K, int had_block, float clip_
 
 size_t rcp_gemv_workspace_bytes(int M, int N, int K) {
   if (M < 1 || M > rcp::kMaxTokens || N < 1 || !k_ok(K)) return 0;
-  return 0;
+  return make_plan(M, N, K).ws_bytes;
 }
 
 int rcp_gemv_w2a4_variant(int variant, const uint32_t* words, const void* lut_f16, const uint8_t* xq,
@@ -115,10 +224,9 @@ int rcp_gemv_w2a4_variant(int variant, const uint32_t* words, const void* lut_f1
       (reinterpret_cast<uintptr_t>(lut_f16) & 7u) || (reinterpret_cast<uintptr_t>(y_f16) & 1u) ||
       (reinterpret_cast<uintptr_t>(scale_f16) & 1u))
     return RCP_ERR_ALIGN;
-  (void)workspace;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (S_dbg) variant = RCP_GEMV_SIMPLE;
-  if (variant == RCP_GEMV_AUTO) variant = RCP_GEMV_SIMPLE;
+  if (variant == RCP_GEMV_AUTO) variant = RCP_GEMV_MMA;
   switch (variant) {
     case RCP_GEMV_SIMPLE: {
       const int block = 256;
@@ -127,6 +235,22 @@ int rcp_gemv_w2a4_variant(int variant, const uint32_t* words, const void* lut_f1
                                                       static_cast<const __half*>(scale_f16), M, N, K,
                                                       static_cast<__half*>(y_f16), S_dbg);
       break;
+    }
+    case RCP_GEMV_MMA:
+      // tensor-core path; for one or two tokens the b0*b1 plane goes to dp4a (FMA pipe) instead
+      return launch_stream(M <= 2 ? rcp::kModeHybrid : rcp::kModeMma, words, lut_f16, xq, scale_f16, M, N, K, y_f16,
+                           workspace, st);
+    case RCP_GEMV_DP4A: {
+      // CUDA-core path: two tokens per launch
+      for (int m0 = 0; m0 < M; m0 += 2) {
+        const int mm = std::min(2, M - m0);
+        // later token pairs reuse the same scratch: it is left zeroed by the previous launch
+        const int rc = launch_stream(rcp::kModeDp4a, words, lut_f16, xq + (size_t)m0 * (K / 2),
+                                     static_cast<const __half*>(scale_f16) + m0, mm, N, K,
+                                     static_cast<__half*>(y_f16) + (size_t)m0 * N, workspace, st);
+        if (rc != RCP_OK) return rc;
+      }
+      return RCP_OK;
     }
     default:
       return RCP_ERR_VARIANT;
