@@ -1,0 +1,473 @@
+#!/usr/bin/env python
+"""Benchmark of the W2A4 decode hot path on B200.
+
+A step is one decode pass over one LLaMA-shaped layer: for every linear of the layer,
+rcp_quantize_act (block-Hadamard + int4) then rcp_gemv_w2a4 (LUT GEMV), on seeded synthetic
+tensors already resident in HBM. Successive steps use different weight copies (more than twice
+the L2 in total), so every step streams its weights from DRAM.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload KEY] [--tokens M]
+  python bench.py --impl reference ...     # the CPU oracle on a bounded sample, same metric
+
+Prints ONE JSON line (rank 0).
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2502_15779_b200 import configs as cfgs  # noqa: E402
+from paper_2502_15779_b200 import synth  # noqa: E402
+
+METRIC = "w2a4_decode_layer_hbm_gbs"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        return json.load(open(path)), "measured"
+    return {"hbm_gbs": 6650.0}, "fallback"
+
+
+def f16_bits(t):
+    return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+# ------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs (read only)."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100", "-i",
+                 str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------- workload
+class LayerSet:
+    """Packed weights (several distinct copies), LUTs, activations and scratch for one decode layer."""
+
+    def __init__(self, cfg, M, device, copies, rcp):
+        self.cfg, self.M, self.dev, self.rcp = cfg, M, device, rcp
+        self.layers = list(cfg.layers)
+        self.words, self.luts, self.x, self.xq, self.scale, self.y, self.ws = [], [], [], [], [], [], []
+        self.codes_first = []
+        for li, L in enumerate(self.layers):
+            wcopies, lcopies = [], []
+            for c in range(copies):
+                seed = cfgs.BASE_SEED + 101 * li + 7 * c
+                codes, lut = synth.make_layer(L.N, L.K, L.had_block, cfg.codes, seed, device)
+                wcopies.append(rcp.rcp_pack_weights(codes))
+                lcopies.append(lut)
+                if c == 0:
+                    self.codes_first.append(None)  # codes regenerated on demand for the CPU sample
+                del codes
+            self.words.append(wcopies)
+            self.luts.append(lcopies)
+            self.x.append(synth.make_activations(M, L.K, cfgs.BASE_SEED + 13 * li, device))
+            self.xq.append(torch.empty(M, L.K // 2, dtype=torch.uint8, device=device))
+            self.scale.append(torch.empty(M, dtype=torch.float16, device=device))
+            self.y.append(torch.empty(M, L.N, dtype=torch.float16, device=device))
+            self.ws.append(rcp.make_workspace(M, L.N, L.K, device))
+        self.copies = copies
+
+    def step(self, copy, variant="auto"):
+        r = self.rcp
+        for li, L in enumerate(self.layers):
+            r.rcp_quantize_act(self.x[li], L.had_block, 1.0, xq=self.xq[li], scale=self.scale[li])
+            r.rcp_gemv_w2a4(self.words[li][copy], self.luts[li][copy], self.xq[li], self.scale[li], y=self.y[li],
+                            workspace=self.ws[li], variant=variant)
+
+    def gemv_bytes(self):
+        return sum(cfgs.gemv_bytes(self.M, L.N, L.K) for L in self.layers)
+
+    def quant_bytes(self):
+        return sum(cfgs.quant_bytes(self.M, L.K) for L in self.layers)
+
+    def weight_bytes(self):
+        return sum(L.N * L.K // 4 for L in self.layers)
+
+
+def l2_bytes(device):
+    return torch.cuda.get_device_properties(device).L2_cache_size
+
+
+def time_graph_replays(graphs, order, stream):
+    """Replays graphs[order[i]] back to back; returns total milliseconds by CUDA events on `stream`."""
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for i in order:
+            graphs[i].replay()
+        e1.record(stream)
+    e1.synchronize()
+    return e0.elapsed_time(e1)
+
+
+def capture(fn, stream):
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=stream):
+        fn()
+    return g
+
+
+def per_shape_table(cfg, M, device, rcp, stream, variant, reps=3):
+    """us/call and GB/s for every GEMV shape of a config: graphs of back-to-back launches cycling
+    through distinct weight copies (cold L2), timed with CUDA events."""
+    rows = []
+    L2 = l2_bytes(device)
+    seen = set()
+    for li, L in enumerate(cfg.layers):
+        if (L.N, L.K) in seen:
+            continue
+        seen.add((L.N, L.K))
+        wbytes = L.N * L.K // 4
+        copies = max(2, -(-2 * L2 // wbytes) + 1)
+        copies = min(copies, 1200)
+        seed = cfgs.BASE_SEED + 101 * li
+        codes, lut = synth.make_layer(L.N, L.K, L.had_block, cfg.codes, seed, device)
+        base = rcp.rcp_pack_weights(codes)
+        del codes
+        # distinct copies: rows rotated so contents differ but the value distribution is the same
+        words = [torch.roll(base, shifts=c, dims=0).contiguous() if c else base for c in range(copies)]
+        luts = [torch.roll(lut, shifts=c, dims=0).contiguous() if c else lut for c in range(copies)]
+        x = synth.make_activations(M, L.K, cfgs.BASE_SEED + 13 * li, device)
+        xq, scale = rcp.rcp_quantize_act(x, L.had_block, 1.0)
+        y = torch.empty(M, L.N, dtype=torch.float16, device=device)
+        ws = rcp.make_workspace(M, L.N, L.K, device)
+        launches = copies * max(1, 64 // copies)
+
+        def body():
+            for i in range(launches):
+                c = i % copies
+                rcp.rcp_gemv_w2a4(words[c], luts[c], xq, scale, y=y, workspace=ws, variant=variant)
+
+        with torch.cuda.stream(stream):
+            body()
+        stream.synchronize()
+        g = capture(body, stream)
+        for _ in range(3):
+            g.replay()
+        stream.synchronize()
+        best = min(time_graph_replays([g], [0], stream) for _ in range(reps))
+        us = best * 1e3 / launches
+        nbytes = cfgs.gemv_bytes(M, L.N, L.K)
+        # isolated single launch (includes launch latency)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        iso = []
+        for c in range(min(copies, 5)):
+            with torch.cuda.stream(stream):
+                e0.record(stream)
+                rcp.rcp_gemv_w2a4(words[c], luts[c], xq, scale, y=y, workspace=ws, variant=variant)
+                e1.record(stream)
+            e1.synchronize()
+            iso.append(e0.elapsed_time(e1) * 1e3)
+        # the quantizer alone
+        gq = capture(lambda: [rcp.rcp_quantize_act(x, L.had_block, 1.0, xq=xq, scale=scale) for _ in range(32)], stream)
+        gq.replay()
+        stream.synchronize()
+        q_us = min(time_graph_replays([gq], [0], stream) for _ in range(reps)) * 1e3 / 32
+        rows.append({"layer": L.name, "N": L.N, "K": L.K, "M": M, "bytes": nbytes, "us_per_call": round(us, 3),
+                     "gbs": round(nbytes / us / 1e3, 1), "frac_of_8TBs": round(nbytes / us / 1e3 / NOMINAL_HBM_GBS, 4),
+                     "isolated_us": round(min(iso), 2), "quantize_us": round(q_us, 2), "copies": copies})
+        del words, luts, base
+        torch.cuda.empty_cache()
+    return rows
+
+
+# ------------------------------------------------------------------------------- CPU oracle leg
+def cpu_oracle_sample(cfg, M, target_seconds=12.0):
+    """Times the oracle (as it stands, one thread) on a bounded sample of the workload: the full
+    activation quantization of every linear of the layer plus the GEMV on the first `rows` output
+    rows of each. Returns (value in the benchmark's unit, description, seconds)."""
+    import oracle
+    layers = list(cfg.layers)
+    # calibration on a tiny slice
+    L0 = layers[0]
+    codes, lut = synth.make_layer(16, L0.K, L0.had_block, cfg.codes, 1)
+    x = synth.make_activations(M, L0.K, 1)
+    t = time.perf_counter()
+    qa = oracle.quantize_act(f16_bits(x), L0.had_block, 1.0)
+    oracle.gemv_w2a4(oracle.pack_weights(codes.numpy()), f16_bits(lut), qa["xq"], qa["scale"])
+    per_code = (time.perf_counter() - t) / (16 * L0.K * M)
+    total_codes = sum(L.N * L.K for L in layers) * M
+    frac = min(1.0, target_seconds / max(1e-9, per_code * total_codes))
+    nbytes, secs, desc = 0, 0.0, []
+    for li, L in enumerate(layers):
+        rows = max(16, int(L.N * frac))
+        rows = min(rows, L.N)
+        seed = cfgs.BASE_SEED + 101 * li
+        codes, lut = synth.make_layer(rows, L.K, L.had_block, cfg.codes, seed)
+        x = synth.make_activations(M, L.K, cfgs.BASE_SEED + 13 * li)
+        xb, cb, lb = f16_bits(x), codes.numpy(), f16_bits(lut)
+        words = oracle.pack_weights(cb)  # offline step, not timed
+        t = time.perf_counter()
+        qa = oracle.quantize_act(xb, L.had_block, 1.0)
+        oracle.gemv_w2a4(words, lb, qa["xq"], qa["scale"])
+        secs += time.perf_counter() - t
+        nbytes += cfgs.gemv_bytes(M, rows, L.K) + cfgs.quant_bytes(M, L.K)
+        desc.append(f"{L.name}:{rows}/{L.N} rows")
+    return nbytes / secs / 1e9, "quantize_act + gemv on " + ", ".join(desc), secs
+
+
+def run_reference(args, cfg, M):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    budget = 60.0 / max(1, args.steps + args.warmup)
+    vals, secs = [], []
+    desc = ""
+    for i in range(args.warmup + args.steps):
+        v, desc, s = cpu_oracle_sample(cfg, M, target_seconds=min(12.0, budget))
+        if i >= args.warmup:
+            vals.append(v)
+            secs.append(s)
+    value = statistics.mean(vals)
+    out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": 1e3 * statistics.mean(secs), "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+           "config": {"workload": f"{cfg.key} M={M}", "note": "CPU oracle on a bounded sample of each step"},
+           "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+           "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out), flush=True)
+
+
+# ------------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama2_70b", choices=list(cfgs.BY_KEY))
+    ap.add_argument("--tokens", type=int, default=1)
+    ap.add_argument("--variant", default="auto", choices=["auto", "simple", "dp4a", "mma", "mma_only"])
+    ap.add_argument("--no-table", action="store_true", help="skip the per-shape table of the other configs")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle leg")
+    args = ap.parse_args()
+    cfg = cfgs.BY_KEY[args.workload]
+    M = args.tokens
+    if args.warmup < 3:
+        args.warmup = 3
+
+    if args.impl == "reference":
+        run_reference(args, cfg, M)
+        return
+
+    import paper_2502_15779_b200 as rcp
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    torch.cuda.set_device(local_rank)
+    device = torch.device(f"cuda:{local_rank}")
+    rcp.lib()  # fail loudly if the CUDA library is missing
+
+    L2 = l2_bytes(device)
+    wbytes = sum(L.N * L.K // 4 for L in cfg.layers)
+    copies = max(2, -(-2 * L2 // wbytes) + 1)
+    layer = LayerSet(cfg, M, device, copies, rcp)
+    stream = torch.cuda.Stream(device=device)
+
+    # eager warm-up (sets kernel attributes), then one CUDA graph per weight copy
+    with torch.cuda.stream(stream):
+        for c in range(copies):
+            layer.step(c, args.variant)
+    stream.synchronize()
+    graphs = [capture(lambda c=c: layer.step(c, args.variant), stream) for c in range(copies)]
+    order = [i % copies for i in range(args.warmup)]
+    time_graph_replays(graphs, order, stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    barrier()
+    if sampler:
+        sampler.start()
+    order = [i % copies for i in range(args.steps)]
+    ms = time_graph_replays(graphs, order, stream)
+    # keep the GPU under the same load a little longer so that the clock sampler sees it
+    t_end = time.time() + 0.6
+    while time.time() < t_end:
+        time_graph_replays(graphs, order[:max(1, len(order) // 4)], stream)
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    if dist is not None:
+        tmax = torch.tensor([ms], device=device)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        ms = float(tmax.item())
+    step_bytes = layer.gemv_bytes() + layer.quant_bytes()
+    ms_per_step = ms / args.steps
+    value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+    launches = args.steps * 2 * len(layer.layers)
+
+    # ---- dominant kernel alone: the GEMV launches of the layer, back to back, cold L2
+    def gemv_only(c):
+        for li, L in enumerate(layer.layers):
+            rcp.rcp_gemv_w2a4(layer.words[li][c], layer.luts[li][c], layer.xq[li], layer.scale[li], y=layer.y[li],
+                              workspace=layer.ws[li], variant=args.variant)
+    ggraphs = [capture(lambda c=c: gemv_only(c), stream) for c in range(copies)]
+    time_graph_replays(ggraphs, order[:8], stream)
+    gms = min(time_graph_replays(ggraphs, order, stream) for _ in range(3))
+    g_launches = args.steps * len(layer.layers)
+    g_bytes_per_launch = layer.gemv_bytes() / len(layer.layers)
+    g_us = gms * 1e3 / g_launches
+    achieved = g_bytes_per_launch / g_us / 1e3
+    peaks, peak_kind = measured_peaks()
+    roofline = {"bound": "hbm", "kernel": "gemv_stream_kernel", "achieved": round(achieved, 1),
+                "peak": peaks["hbm_gbs"], "peak_kind": peak_kind, "unit": "GB/s",
+                "frac": round(achieved / peaks["hbm_gbs"], 4), "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
+                "avg_launch_us": round(g_us, 3), "bytes_per_launch": int(g_bytes_per_launch), "traffic": None}
+    prof = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(prof):
+        try:
+            roofline["traffic"] = json.load(open(prof)).get(f"{cfg.key}_M{M}")
+        except Exception:
+            pass
+
+    # ---- end to end through the C ABI with host buffers
+    xh = [layer.x[li].cpu().pin_memory() for li in range(len(layer.layers))]
+    yh = [torch.empty(M, L.N, dtype=torch.float16).pin_memory() for L in layer.layers]
+
+    def e2e_step(c):
+        for li, L in enumerate(layer.layers):
+            rcp.rcp_linear_w2a4_host(xh[li], L.had_block, 1.0, layer.words[li][c], layer.luts[li][c], yh[li],
+                                     layer.x[li], layer.xq[li], layer.scale[li], layer.y[li], layer.ws[li])
+    e2e_steps = min(args.steps, 100)
+    with torch.cuda.stream(stream):
+        for i in range(3):
+            e2e_step(i % copies)
+            stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for i in range(e2e_steps):
+            e2e_step(i % copies)
+            stream.synchronize()  # the host reads y before the next decode step
+        e1.record(stream)
+    e1.synchronize()
+    e2e_ms = e0.elapsed_time(e1)
+    if dist is not None:
+        tmax = torch.tensor([e2e_ms], device=device)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tmax.item())
+    e2e = {"value": round(world * step_bytes / (e2e_ms / e2e_steps * 1e-3) / 1e9, 2), "unit": UNIT,
+           "ms_per_step": round(e2e_ms / e2e_steps, 4),
+           "h2d_bytes_per_step": sum(2 * M * L.K for L in layer.layers),
+           "d2h_bytes_per_step": sum(2 * M * L.N for L in layer.layers)}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    shapes = []
+    if not args.no_table:
+        del graphs, ggraphs
+        wl_rows = per_shape_table(cfg, M, device, rcp, stream, args.variant)
+        shapes.append({"config": cfg.key, "rows": wl_rows})
+        for other in cfgs.CONFIGS:
+            if other.key != cfg.key:
+                shapes.append({"config": other.key, "rows": per_shape_table(other, 1, device, rcp, stream, args.variant)})
+
+    # offline step: weight packing throughput (not part of the decode step)
+    Lp = cfg.layers[0]
+    codes = synth.make_codes_uniform(Lp.N, Lp.K, 1, device)
+    outw = torch.empty(Lp.N, Lp.K // 16, dtype=torch.int32, device=device)
+    rcp.rcp_pack_weights(codes, out=outw)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    rcp.rcp_pack_weights(codes, out=outw)
+    e1.record()
+    e1.synchronize()
+    pack_ms = e0.elapsed_time(e1)
+    pack = {"N": Lp.N, "K": Lp.K, "ms": round(pack_ms, 4),
+            "gbs": round((Lp.N * Lp.K * 1.25) / pack_ms / 1e6, 1), "note": "offline step, includes the status read-back"}
+
+    cpu = None
+    if not args.no_cpu:
+        v, desc, secs = cpu_oracle_sample(cfg, M)
+        cpu = {"value": round(v, 4), "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc, "seconds": round(secs, 2)}
+
+    out = {"metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+           "config": {"workload": f"{cfg.key} ({cfg.title}), M={M}: " +
+                      ", ".join(f"{L.name} {L.N}x{L.K}" for L in cfg.layers),
+                      "step": "per linear: rcp_quantize_act + rcp_gemv_w2a4, replayed from a CUDA graph",
+                      "cold_l2": f"{copies} distinct weight copies in rotation ({copies * wbytes / 1e6:.0f} MB > 2x L2 "
+                                 f"of {L2 / 1e6:.0f} MB)",
+                      "variant": args.variant, "parallelism": "replicas only" if world > 1 else "single GPU",
+                      "bytes_per_step": step_bytes},
+           "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
+           "us_per_gemv_call": round(g_us, 3), "pack": pack, "shapes": shapes}
+    print(json.dumps(out), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

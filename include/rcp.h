@@ -79,9 +79,11 @@ int rcp_quantize_act(const void* x_f16, int M, int K, int had_block, float clip_
  *   RCP_GEMV_SIMPLE  one warp per output row, scalar decode; also the variant behind S_dbg.
  *   RCP_GEMV_DP4A    CUDA-core path: masked code planes times int8 activations with dp4a.
  *   RCP_GEMV_MMA     masked code planes as the A operand of int8 mma.sync, weights streamed
- *                    through a TMA/mbarrier shared-memory ring, work split evenly over the SMs.
+ *                    through a TMA/mbarrier shared-memory ring, work split evenly over the SMs;
+ *                    for M <= 2 the b0*b1 plane is computed with dp4a beside the tensor cores.
+ *   RCP_GEMV_MMA_ONLY  as RCP_GEMV_MMA with all three planes on the tensor cores for every M.
  */
-enum { RCP_GEMV_AUTO = 0, RCP_GEMV_SIMPLE = 1, RCP_GEMV_DP4A = 2, RCP_GEMV_MMA = 3 };
+enum { RCP_GEMV_AUTO = 0, RCP_GEMV_SIMPLE = 1, RCP_GEMV_DP4A = 2, RCP_GEMV_MMA = 3, RCP_GEMV_MMA_ONLY = 4 };
 
 /*
  * Bytes of caller-provided scratch rcp_gemv_w2a4 needs for this shape (0 if none). The scratch
@@ -107,6 +109,21 @@ int rcp_gemv_w2a4(const uint32_t* words, const void* lut_f16, const uint8_t* xq,
 int rcp_gemv_w2a4_variant(int variant, const uint32_t* words, const void* lut_f16,
                           const uint8_t* xq, const void* scale_f16, int M, int N, int K,
                           void* y_f16, void* workspace, int32_t* S_dbg, void* stream);
+
+/*
+ * One decode linear layer end to end with HOST activations (Section 4.4 data path: rotate and
+ * quantize the token, then the LUT GEMV): copies x from host memory, runs rcp_quantize_act and
+ * rcp_gemv_w2a4, copies y back. All on `stream`, no synchronization: y_host is valid after the
+ * caller synchronizes the stream. Pinned host memory makes the copies asynchronous.
+ *   x_host_f16  HOST fp16 [M][K];  y_host_f16  HOST fp16 [M][N].
+ *   words, lut_f16             DEVICE, the resident packed layer.
+ *   x_dev [M][K] fp16, xq_dev [M][K/2], scale_dev [M] fp16, y_dev [M][N] fp16, workspace:
+ *                              DEVICE staging owned by the caller (same rules as above).
+ */
+int rcp_linear_w2a4_host(const void* x_host_f16, int M, int K, int had_block, float clip_ratio,
+                         const uint32_t* words, const void* lut_f16, int N, void* y_host_f16,
+                         void* x_dev, uint8_t* xq_dev, void* scale_dev, void* y_dev, void* workspace,
+                         void* stream);
 
 #ifdef __cplusplus
 }

@@ -12,8 +12,8 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "librcp_w2a4.so")
 
-GEMV_AUTO, GEMV_SIMPLE, GEMV_DP4A, GEMV_MMA = 0, 1, 2, 3
-VARIANTS = {"auto": GEMV_AUTO, "simple": GEMV_SIMPLE, "dp4a": GEMV_DP4A, "mma": GEMV_MMA}
+GEMV_AUTO, GEMV_SIMPLE, GEMV_DP4A, GEMV_MMA, GEMV_MMA_ONLY = 0, 1, 2, 3, 4
+VARIANTS = {"auto": GEMV_AUTO, "simple": GEMV_SIMPLE, "dp4a": GEMV_DP4A, "mma": GEMV_MMA, "mma_only": GEMV_MMA_ONLY}
 
 _lib = None
 
@@ -47,6 +47,8 @@ def lib():
         L.rcp_gemv_w2a4.argtypes = [vp, vp, vp, vp, i, i, i, vp, vp, vp, vp]
         L.rcp_gemv_w2a4_variant.restype = i
         L.rcp_gemv_w2a4_variant.argtypes = [i, vp, vp, vp, vp, i, i, i, vp, vp, vp, vp]
+        L.rcp_linear_w2a4_host.restype = i
+        L.rcp_linear_w2a4_host.argtypes = [vp, i, i, i, C.c_float, vp, vp, i, vp, vp, vp, vp, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -127,3 +129,18 @@ def rcp_gemv_w2a4(words, lut, xq, scale, y=None, workspace=None, S_dbg=None, var
                lib().rcp_gemv_w2a4_variant(v, _ptr(words), _ptr(lut), _ptr(xq), _ptr(scale), M, N, K, _ptr(y),
                                            _ptr(workspace), _ptr(S_dbg), _stream(words)))
     return y
+
+
+def rcp_linear_w2a4_host(x_host, had_block, clip_ratio, words, lut, y_host, x_dev, xq_dev, scale_dev, y_dev, workspace):
+    """x_host fp16 [M][K] (host, ideally pinned) -> y_host fp16 [M][N] (host). Asynchronous on the
+    current stream: synchronize before reading y_host."""
+    M, K = x_host.shape
+    N = words.shape[0]
+    if x_host.is_cuda or y_host.is_cuda or x_host.dtype != torch.float16 or y_host.dtype != torch.float16:
+        raise TypeError("x_host / y_host must be fp16 host tensors")
+    with torch.cuda.device(words.device):
+        _check("rcp_linear_w2a4_host",
+               lib().rcp_linear_w2a4_host(_ptr(x_host), M, K, int(had_block), float(clip_ratio), _ptr(words), _ptr(lut),
+                                          N, _ptr(y_host), _ptr(x_dev), _ptr(xq_dev), _ptr(scale_dev), _ptr(y_dev),
+                                          _ptr(workspace), _stream(words)))
+    return y_host

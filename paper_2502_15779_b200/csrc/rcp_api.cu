@@ -30,16 +30,24 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 bool k_ok(int K) { return K >= 64 && K <= rcp::kMaxK && K % 64 == 0; }
 
 __device__ int g_pack_bad;  // set by pack_weights_kernel when it meets a code above 3
+}  // namespace
+#ifdef RCP_EXPERIMENTS
+extern "C" int rcp_set_experiment(int v) {
+  return (int)cudaMemcpyToSymbol(rcp::g_experiment, &v, sizeof(int));
+}
+#endif
+namespace {
 
 // ---------------------------------------------------------------------------------------------
 // Streaming GEMV: launch plan shared by rcp_gemv_workspace_bytes and the launcher.
 struct StreamPlan {
-  int ntiles, nchunks, ncol, supers, ch_per_super, stages;
+  int ntiles, nchunks, ncol, supers, ch_per_super, stages, ctas_per_sm;
   size_t smem, ws_count_off, ws_sum_off, ws_bytes;
 };
 
 constexpr size_t kSmemMax = 232448;          // 227 KB of dynamic shared memory per CTA on sm_100
-constexpr size_t kExpandBudget = 64 * 1024;  // expanded activations kept resident per CTA
+constexpr size_t kSmemPerSm = 233472;         // 228 KB of shared memory per SM
+constexpr size_t kExpandBudget = 32 * 1024;  // expanded activations kept resident per CTA
 
 StreamPlan make_plan(int M, int N, int K) {
   StreamPlan pl;
@@ -53,11 +61,15 @@ StreamPlan make_plan(int M, int N, int K) {
   pl.ch_per_super = (pl.nchunks + pl.supers - 1) / pl.supers;
   pl.supers = (pl.nchunks + pl.ch_per_super - 1) / pl.ch_per_super;
   const size_t bs = (size_t)pl.ch_per_super * per_chunk;
-  const size_t fixed = 1024 + 512 + bs;
-  pl.stages = (int)std::min<size_t>(rcp::kMaxStages, (kSmemMax - fixed) / rcp::kStageBytes);
+  const size_t fixed = 1024 + 640 + bs;
+  // two CTAs per SM (more warps to hide latency) except for the 16-token kernel, whose
+  // accumulators need the whole register file
+  pl.ctas_per_sm = M <= 8 ? 2 : 1;
+  const size_t per_cta = (kSmemPerSm / pl.ctas_per_sm) - 1024;  // 1 KB per CTA is reserved by the system
+  pl.stages = (int)std::min<size_t>(rcp::kMaxStages, (per_cta - fixed) / rcp::kStageBytes);
   pl.smem = fixed + (size_t)pl.stages * rcp::kStageBytes;
   pl.ws_count_off = 16;
-  const size_t cnt = (size_t)pl.ntiles * rcp::kConsumerWarps * 4;
+  const size_t cnt = (size_t)pl.ntiles * rcp::kWarps * 4;
   pl.ws_sum_off = pl.ws_count_off + ((cnt + 15) / 16) * 16;
   pl.ws_bytes = pl.ws_sum_off + (size_t)pl.ntiles * rcp::kTileRows * M * 3 * 4;
   return pl;
@@ -89,15 +101,15 @@ int sm_count() {
   return n;
 }
 
-template <int MT, int MODE>
+template <int MT, int MODE, int MTOK, int MINB>
 int launch_stream_t(const CUtensorMap& map, const rcp::StreamParams& sp, const StreamPlan& pl, cudaStream_t st) {
   static bool attr_set = false;
-  auto kern = rcp::gemv_stream_kernel<MT, MODE>;
+  auto kern = rcp::gemv_stream_kernel<MT, MODE, MTOK, MINB>;
   if (!attr_set) {
     RCP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax));
     attr_set = true;
   }
-  const int gx = std::max(1, sm_count() / pl.supers);
+  const int gx = std::max(1, sm_count() * pl.ctas_per_sm / pl.supers);
   kern<<<dim3(gx, pl.supers), rcp::kStreamThreads, pl.smem, st>>>(map, sp);
   RCP_CUDA(cudaGetLastError());
   return RCP_OK;
@@ -114,7 +126,7 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   CUtensorMap map;
   const cuuint64_t gdim[2] = {(cuuint64_t)(K / 16), (cuuint64_t)N};
   const cuuint64_t gstride[1] = {(cuuint64_t)(K / 4)};
-  const cuuint32_t box[2] = {(cuuint32_t)rcp::kChunkWords, (cuuint32_t)rcp::kTileRows};
+  const cuuint32_t box[2] = {(cuuint32_t)rcp::kChunkWords, (cuuint32_t)rcp::kWarpRows};
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = enc(&map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t*>(words), gdim, gstride, box,
                          estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -132,10 +144,14 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   sp.M = M; sp.N = N; sp.K = K;
   sp.ntiles = pl.ntiles; sp.nchunks = pl.nchunks; sp.ch_per_super = pl.ch_per_super;
   sp.stages = pl.stages; sp.ncol = pl.ncol;
-  if (mode == rcp::kModeHybrid) return launch_stream_t<1, rcp::kModeHybrid>(map, sp, pl, st);
-  if (mode == rcp::kModeDp4a) return launch_stream_t<1, rcp::kModeDp4a>(map, sp, pl, st);
-  if (M <= 8) return launch_stream_t<1, rcp::kModeMma>(map, sp, pl, st);
-  return launch_stream_t<2, rcp::kModeMma>(map, sp, pl, st);
+  if (mode == rcp::kModeHybrid)
+    return M == 1 ? launch_stream_t<1, rcp::kModeHybrid, 1, 2>(map, sp, pl, st)
+                  : launch_stream_t<1, rcp::kModeHybrid, 2, 2>(map, sp, pl, st);
+  if (mode == rcp::kModeDp4a)
+    return M == 1 ? launch_stream_t<1, rcp::kModeDp4a, 1, 2>(map, sp, pl, st)
+                  : launch_stream_t<1, rcp::kModeDp4a, 2, 2>(map, sp, pl, st);
+  if (M <= 8) return launch_stream_t<1, rcp::kModeMma, 0, 2>(map, sp, pl, st);
+  return launch_stream_t<2, rcp::kModeMma, 0, 1>(map, sp, pl, st);
 }
 
 }  // namespace
@@ -240,6 +256,8 @@ int rcp_gemv_w2a4_variant(int variant, const uint32_t* words, const void* lut_f1
       // tensor-core path; for one or two tokens the b0*b1 plane goes to dp4a (FMA pipe) instead
       return launch_stream(M <= 2 ? rcp::kModeHybrid : rcp::kModeMma, words, lut_f16, xq, scale_f16, M, N, K, y_f16,
                            workspace, st);
+    case RCP_GEMV_MMA_ONLY:
+      return launch_stream(rcp::kModeMma, words, lut_f16, xq, scale_f16, M, N, K, y_f16, workspace, st);
     case RCP_GEMV_DP4A: {
       // CUDA-core path: two tokens per launch
       for (int m0 = 0; m0 < M; m0 += 2) {
@@ -263,6 +281,21 @@ int rcp_gemv_w2a4(const uint32_t* words, const void* lut_f16, const uint8_t* xq,
                   int M, int N, int K, void* y_f16, void* workspace, int32_t* S_dbg, void* stream) {
   return rcp_gemv_w2a4_variant(RCP_GEMV_AUTO, words, lut_f16, xq, scale_f16, M, N, K, y_f16, workspace,
                                S_dbg, stream);
+}
+
+int rcp_linear_w2a4_host(const void* x_host_f16, int M, int K, int had_block, float clip_ratio,
+                         const uint32_t* words, const void* lut_f16, int N, void* y_host_f16, void* x_dev,
+                         uint8_t* xq_dev, void* scale_dev, void* y_dev, void* workspace, void* stream) {
+  if (!x_host_f16 || !y_host_f16 || !x_dev || !y_dev) return RCP_ERR_NULL;
+  if (M < 1 || M > rcp::kMaxTokens || N < 1 || !k_ok(K)) return RCP_ERR_SHAPE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  RCP_CUDA(cudaMemcpyAsync(x_dev, x_host_f16, (size_t)M * K * 2, cudaMemcpyHostToDevice, st));
+  int rc = rcp_quantize_act(x_dev, M, K, had_block, clip_ratio, xq_dev, scale_dev, stream);
+  if (rc != RCP_OK) return rc;
+  rc = rcp_gemv_w2a4(words, lut_f16, xq_dev, scale_dev, M, N, K, y_dev, workspace, nullptr, stream);
+  if (rc != RCP_OK) return rc;
+  RCP_CUDA(cudaMemcpyAsync(y_host_f16, y_dev, (size_t)M * N * 2, cudaMemcpyDeviceToHost, st));
+  return RCP_OK;
 }
 
 }  // extern "C"

@@ -14,7 +14,7 @@ from helpers import f16_bits
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
-VARIANTS = ["simple", "dp4a", "mma", "auto"]
+VARIANTS = ["simple", "dp4a", "mma", "mma_only", "auto"]
 
 
 def words_np(words_t):
