@@ -30,47 +30,43 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 bool k_ok(int K) { return K >= 64 && K <= rcp::kMaxK && K % 64 == 0; }
 
 __device__ int g_pack_bad;  // set by pack_weights_kernel when it meets a code above 3
-}  // namespace
-#ifdef RCP_EXPERIMENTS
-extern "C" int rcp_set_experiment(int v) {
-  return (int)cudaMemcpyToSymbol(rcp::g_experiment, &v, sizeof(int));
-}
-#endif
-namespace {
 
 // ---------------------------------------------------------------------------------------------
 // Streaming GEMV: launch plan shared by rcp_gemv_workspace_bytes and the launcher.
 struct StreamPlan {
-  int ntiles, nchunks, ncol, supers, ch_per_super, stages, ctas_per_sm;
-  size_t smem, ws_count_off, ws_sum_off, ws_bytes;
+  int ntiles, spt_all, sps, supers, stages;
+  int off_bar, off_T0st, off_T0, off_scale, off_bs;
+  size_t smem, ws_count_off, ws_T0_off, ws_sum_off, ws_bytes;
 };
 
-constexpr size_t kSmemMax = 232448;          // 227 KB of dynamic shared memory per CTA on sm_100
-constexpr size_t kSmemPerSm = 233472;         // 228 KB of shared memory per SM
-constexpr size_t kExpandBudget = 32 * 1024;  // expanded activations kept resident per CTA
+constexpr size_t kSmemMax = 232448;           // 227 KB of dynamic shared memory per CTA on sm_100
+constexpr size_t kExpandBudget = 96 * 1024;   // expanded activations kept resident per CTA
 
 StreamPlan make_plan(int M, int N, int K) {
   StreamPlan pl;
   pl.ntiles = (N + rcp::kTileRows - 1) / rcp::kTileRows;
-  pl.nchunks = (K / 16 + rcp::kChunkWords - 1) / rcp::kChunkWords;
-  pl.ncol = 1;
-  while (pl.ncol < M) pl.ncol *= 2;
-  const int per_chunk = rcp::kChunkWords * 16 * pl.ncol;  // bytes of expanded activations per K chunk
-  const int max_ch = (int)std::max<size_t>(1, kExpandBudget / per_chunk);
-  pl.supers = (pl.nchunks + max_ch - 1) / max_ch;
-  pl.ch_per_super = (pl.nchunks + pl.supers - 1) / pl.supers;
-  pl.supers = (pl.nchunks + pl.ch_per_super - 1) / pl.ch_per_super;
-  const size_t bs = (size_t)pl.ch_per_super * per_chunk;
-  const size_t fixed = 1024 + 640 + bs;
-  // two CTAs per SM (more warps to hide latency) except for the 16-token kernel, whose
-  // accumulators need the whole register file
-  pl.ctas_per_sm = M <= 8 ? 2 : 1;
-  const size_t per_cta = (kSmemPerSm / pl.ctas_per_sm) - 1024;  // 1 KB per CTA is reserved by the system
-  pl.stages = (int)std::min<size_t>(rcp::kMaxStages, (per_cta - fixed) / rcp::kStageBytes);
-  pl.smem = fixed + (size_t)pl.stages * rcp::kStageBytes;
+  pl.spt_all = (K / 16 + rcp::kStageWords - 1) / rcp::kStageWords;
+  // expanded activations: one byte per code and token, 512 M bytes per stage; K ranges whose
+  // activations fit in shared memory go to different blockIdx.y
+  const size_t bs_per_stage = (size_t)rcp::kStageWords * 16 * M;
+  int sps = (int)std::min<size_t>(rcp::kMaxSps, std::max<size_t>(1, kExpandBudget / bs_per_stage));
+  sps = std::min(sps, pl.spt_all);
+  pl.supers = (pl.spt_all + sps - 1) / sps;
+  pl.sps = (pl.spt_all + pl.supers - 1) / pl.supers;
+  const size_t bs_bytes = (size_t)pl.sps * bs_per_stage;
+  const size_t misc = 128 + (size_t)M * rcp::kMaxSps * 4 + 64 + 64;
+  pl.stages = (int)std::min<size_t>(rcp::kMaxStages, (kSmemMax - 1024 - misc - bs_bytes) / rcp::kStageBytes);
+  size_t off = (size_t)pl.stages * rcp::kStageBytes;
+  pl.off_bar = (int)off; off += 128;
+  pl.off_T0st = (int)off; off += (size_t)M * rcp::kMaxSps * 4;
+  pl.off_T0 = (int)off; off += 64;
+  pl.off_scale = (int)off; off += 64;
+  pl.off_bs = (int)off; off += bs_bytes;
+  pl.smem = off + 1024;
   pl.ws_count_off = 16;
-  const size_t cnt = (size_t)pl.ntiles * rcp::kWarps * 4;
-  pl.ws_sum_off = pl.ws_count_off + ((cnt + 15) / 16) * 16;
+  const size_t groups = (size_t)pl.ntiles * rcp::kCWarps;
+  pl.ws_T0_off = pl.ws_count_off + ((groups * 4 + 15) / 16) * 16;
+  pl.ws_sum_off = pl.ws_T0_off + ((groups * M * 4 + 15) / 16) * 16;
   pl.ws_bytes = pl.ws_sum_off + (size_t)pl.ntiles * rcp::kTileRows * M * 3 * 4;
   return pl;
 }
@@ -101,16 +97,16 @@ int sm_count() {
   return n;
 }
 
-template <int MT, int MODE, int MTOK, int MINB>
-int launch_stream_t(const CUtensorMap& map, const rcp::StreamParams& sp, const StreamPlan& pl, cudaStream_t st) {
+template <int MT, int MODE, int MTOK>
+int launch_stream_t(const CUtensorMap& map, const rcp::GemvParams& gp, const StreamPlan& pl, cudaStream_t st) {
   static bool attr_set = false;
-  auto kern = rcp::gemv_stream_kernel<MT, MODE, MTOK, MINB>;
+  auto kern = rcp::gemv_stream_kernel<MT, MODE, MTOK>;
   if (!attr_set) {
     RCP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax));
     attr_set = true;
   }
-  const int gx = std::max(1, sm_count() * pl.ctas_per_sm / pl.supers);
-  kern<<<dim3(gx, pl.supers), rcp::kStreamThreads, pl.smem, st>>>(map, sp);
+  const int gx = std::max(1, sm_count() / pl.supers);
+  kern<<<dim3(gx, pl.supers), rcp::kGThreads, pl.smem, st>>>(map, gp);
   RCP_CUDA(cudaGetLastError());
   return RCP_OK;
 }
@@ -123,35 +119,38 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   EncodeTiledFn enc = encode_tiled_fn();
   if (!enc) return cuda_fail(cudaErrorNotSupported);
   const StreamPlan pl = make_plan(M, N, K);
+  if (pl.stages < 2 || pl.smem > kSmemMax) return RCP_ERR_SHAPE;
   CUtensorMap map;
   const cuuint64_t gdim[2] = {(cuuint64_t)(K / 16), (cuuint64_t)N};
   const cuuint64_t gstride[1] = {(cuuint64_t)(K / 4)};
-  const cuuint32_t box[2] = {(cuuint32_t)rcp::kChunkWords, (cuuint32_t)rcp::kWarpRows};
+  const cuuint32_t box[2] = {(cuuint32_t)rcp::kStageWords, (cuuint32_t)rcp::kTileRows};
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = enc(&map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t*>(words), gdim, gstride, box,
                          estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue);
-  rcp::StreamParams sp;
-  sp.lut = static_cast<const uint2*>(lut_f16);
-  sp.xq = xq;
-  sp.scale = static_cast<const __half*>(scale_f16);
-  sp.y = static_cast<__half*>(y_f16);
+  rcp::GemvParams gp;
+  gp.lut = static_cast<const uint2*>(lut_f16);
+  gp.xq = xq;
+  gp.scale = static_cast<const __half*>(scale_f16);
+  gp.y = static_cast<__half*>(y_f16);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
-  sp.ws_status = reinterpret_cast<int32_t*>(ws);
-  sp.ws_count = reinterpret_cast<uint32_t*>(ws + pl.ws_count_off);
-  sp.ws_sum = reinterpret_cast<int32_t*>(ws + pl.ws_sum_off);
-  sp.M = M; sp.N = N; sp.K = K;
-  sp.ntiles = pl.ntiles; sp.nchunks = pl.nchunks; sp.ch_per_super = pl.ch_per_super;
-  sp.stages = pl.stages; sp.ncol = pl.ncol;
+  gp.ws_status = reinterpret_cast<int32_t*>(ws);
+  gp.ws_count = reinterpret_cast<uint32_t*>(ws + pl.ws_count_off);
+  gp.ws_T0 = reinterpret_cast<int32_t*>(ws + pl.ws_T0_off);
+  gp.ws_sum = reinterpret_cast<int32_t*>(ws + pl.ws_sum_off);
+  gp.M = M; gp.N = N; gp.K = K;
+  gp.ntiles = pl.ntiles; gp.spt_all = pl.spt_all; gp.sps = pl.sps; gp.stages = pl.stages;
+  gp.off_bar = pl.off_bar; gp.off_T0st = pl.off_T0st; gp.off_T0 = pl.off_T0; gp.off_scale = pl.off_scale;
+  gp.off_bs = pl.off_bs;
   if (mode == rcp::kModeHybrid)
-    return M == 1 ? launch_stream_t<1, rcp::kModeHybrid, 1, 2>(map, sp, pl, st)
-                  : launch_stream_t<1, rcp::kModeHybrid, 2, 2>(map, sp, pl, st);
+    return M == 1 ? launch_stream_t<1, rcp::kModeHybrid, 1>(map, gp, pl, st)
+                  : launch_stream_t<1, rcp::kModeHybrid, 2>(map, gp, pl, st);
   if (mode == rcp::kModeDp4a)
-    return M == 1 ? launch_stream_t<1, rcp::kModeDp4a, 1, 2>(map, sp, pl, st)
-                  : launch_stream_t<1, rcp::kModeDp4a, 2, 2>(map, sp, pl, st);
-  if (M <= 8) return launch_stream_t<1, rcp::kModeMma, 0, 2>(map, sp, pl, st);
-  return launch_stream_t<2, rcp::kModeMma, 0, 1>(map, sp, pl, st);
+    return M == 1 ? launch_stream_t<1, rcp::kModeDp4a, 1>(map, gp, pl, st)
+                  : launch_stream_t<1, rcp::kModeDp4a, 2>(map, gp, pl, st);
+  if (M <= 8) return launch_stream_t<1, rcp::kModeMma, 0>(map, gp, pl, st);
+  return launch_stream_t<2, rcp::kModeMma, 0>(map, gp, pl, st);
 }
 
 }  // namespace
@@ -228,6 +227,7 @@ int rcp_quantize_act(const void* x_f16, int M, int K, int had_block, float clip_
 
 size_t rcp_gemv_workspace_bytes(int M, int N, int K) {
   if (M < 1 || M > rcp::kMaxTokens || N < 1 || !k_ok(K)) return 0;
+  // the layout grows with M, and the CUDA-core variant runs the tokens in pairs on the same scratch
   return make_plan(M, N, K).ws_bytes;
 }
 
