@@ -18,10 +18,11 @@
 // rows of the box over the whole K range, read their MMA fragments bank-conflict free, keep the
 // partial sums in registers and finish their rows themselves, so the consumers never wait on one
 // another. Tiles (256 rows x K) are dealt round-robin over the CTAs; the tiles left over are split
-// along K between CTAs and their partial sums meet in a caller-provided scratch buffer (integer
-// atomics, order independent, hence deterministic); the last contributor finishes the rows and
-// re-zeroes the scratch. The int4 activations are expanded once per CTA into the B-operand byte
-// layout in shared memory.
+// along K between CTAs and come first. Their partial sums meet in a caller-provided scratch buffer
+// (integer atomics, order independent, hence deterministic); the memory fence, the count of
+// contributions and the finishing of a completed tile are the job of a separate warp, so that
+// their latency stays off the consumers' path; the last contributor re-zeroes the scratch. The
+// int4 activations are expanded once per CTA into the B-operand byte layout in shared memory.
 #pragma once
 #include <cuda.h>
 
@@ -30,7 +31,8 @@
 namespace rcp {
 
 constexpr int kCWarps = 16;                       // consumer warps
-constexpr int kGThreads = (kCWarps + 1) * 32;     // + one producer warp
+constexpr int kGThreads = (kCWarps + 2) * 32;     // + one producer warp + one finishing warp
+constexpr int kPartRing = 8;                      // partial segments in flight between consumers and finisher
 constexpr int kTileRows = 16 * kCWarps;           // rows of a TMA box
 constexpr int kStageWords = 32;                   // 128 bytes of K per row per stage (512 codes)
 constexpr int kStageBytes = kTileRows * kStageWords * 4;
@@ -46,8 +48,8 @@ struct GemvParams {
   const __half* scale;
   __half* y;
   int32_t* ws_status;   // [4]
-  uint32_t* ws_count;   // [ntiles * 16]
-  int32_t* ws_T0;       // [ntiles * 16][M]
+  uint32_t* ws_count;   // [ntiles]
+  int32_t* ws_T0;       // [ntiles][M]
   int32_t* ws_sum;      // [ntiles * 256][M][3]
   int M, N, K;
   int ntiles;           // 256-row tiles
@@ -110,10 +112,10 @@ __device__ __forceinline__ void dp4a_u8s8(int& d, uint32_t a, uint32_t b) {
 // One segment of a CTA's work: stages [sb, se) of a tile (stage indices relative to blockIdx.y's range).
 struct Segment { int tile, sb, se; };
 
-// The work of CTA b of G: rounds of whole tiles dealt round-robin, then an equal share of the
-// stages of the tiles left over (at most two more segments).
+// The work of CTA b of G: first an equal share of the stages of the tiles left over when the tiles
+// are dealt round-robin (at most two segments), then the rounds of whole tiles.
 struct WorkList {
-  int G, b, R, spt, tail_tile, tail_sb, tail_n, nseg;
+  int G, b, R, spt, tail_tile, tail_sb, tail_n, ntail, nseg;
   __device__ __forceinline__ WorkList(int ntiles, int spt_, int G_, int b_) : G(G_), b(b_), spt(spt_) {
     R = ntiles / G;
     const long long rem = (long long)(ntiles - R * G) * spt;
@@ -121,12 +123,13 @@ struct WorkList {
     tail_n = hi - lo;
     tail_sb = tail_n > 0 ? lo % spt : 0;
     tail_tile = R * G + (tail_n > 0 ? lo / spt : 0);
-    nseg = R + (tail_n > 0 ? 1 : 0) + (tail_sb + tail_n > spt ? 1 : 0);
+    ntail = (tail_n > 0 ? 1 : 0) + (tail_sb + tail_n > spt ? 1 : 0);
+    nseg = R + ntail;
   }
   __device__ __forceinline__ Segment get(int i) const {
     Segment s;
-    if (i < R) { s.tile = i * G + b; s.sb = 0; s.se = spt; }
-    else if (i == R) { s.tile = tail_tile; s.sb = tail_sb; s.se = min(spt, tail_sb + tail_n); }
+    if (i >= ntail) { s.tile = (i - ntail) * G + b; s.sb = 0; s.se = spt; }
+    else if (i == 0) { s.tile = tail_tile; s.sb = tail_sb; s.se = min(spt, tail_sb + tail_n); }
     else { s.tile = tail_tile + 1; s.sb = 0; s.se = tail_sb + tail_n - spt; }
     return s;
   }
@@ -157,8 +160,8 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap tmap, const GemvParams p)
   const int ncol = M;
   const int stages = p.stages;
   const uint32_t full0 = base + p.off_bar, empty0 = full0 + 8 * kMaxStages;
+  const uint32_t part0 = empty0 + 8 * kMaxStages, done0 = part0 + 8 * kPartRing;
   int* const s_T0st = reinterpret_cast<int*>(gen + p.off_T0st);         // [M][kMaxSps]
-  int* const s_T0 = reinterpret_cast<int*>(gen + p.off_T0);             // [16]
   float* const s_scale = reinterpret_cast<float*>(gen + p.off_scale);   // [16]
   uint8_t* const bs = gen + p.off_bs;
 
@@ -166,12 +169,8 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap tmap, const GemvParams p)
   const int spt = min(p.sps, p.spt_all - st0);         // stages per tile handled here
   const WorkList work(p.ntiles, spt, gridDim.x, blockIdx.x);
   if (work.nseg == 0) return;
-
-  if (tid == 0) {
-    for (int s = 0; s < stages; s++) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, kCWarps); }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  __syncthreads();
+  const bool one_range = (gridDim.y == 1);
+  auto is_whole = [&](const Segment& sg) { return one_range && sg.sb == 0 && sg.se == p.spt_all; };
 
   // ------------------------------------------------------------------ producer prologue
   // The weights do not depend on the preceding kernel: start streaming at once.
@@ -189,6 +188,10 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap tmap, const GemvParams p)
     if (++pr_slot == stages) { pr_slot = 0; pr_phase ^= 1u; }
   };
   if (tid == kCWarps * 32) {
+    // the producer thread sets up every barrier itself and starts the stream before the CTA meets
+    for (int s = 0; s < stages; s++) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, kCWarps); }
+    for (int s = 0; s < kPartRing; s++) { mbar_init(part0 + 8 * s, kCWarps); mbar_init(done0 + 8 * s, 1); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     for (int i = 0; i < stages && pr_seg < work.nseg; i++) produce();
   }
 
@@ -234,12 +237,6 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap tmap, const GemvParams p)
     if (tid < M) s_scale[tid] = __half2float(p.scale[tid]);
   }
   __syncthreads();
-  if (tid < M) {
-    int a = 0;
-    for (int st = 0; st < spt; st++) a += s_T0st[tid * kMaxSps + st];
-    s_T0[tid] = a;
-  }
-  __syncthreads();
 
   // ------------------------------------------------------------------ producer main loop
   if (warp == kCWarps) {
@@ -249,6 +246,61 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap tmap, const GemvParams p)
         if (!mbar_wait(empty0 + 8 * pr_slot, pr_phase ^ 1u)) { atomicExch(p.ws_status, 2); break; }
         produce();
       }
+    }
+    return;
+  }
+
+  // ------------------------------------------------------------------ finishing warp
+  // For every partial segment, once all consumer warps have added their sums to the scratch:
+  // fence, count the contribution, and if it completes the tile, finish its 256 rows.
+  if (warp == kCWarps + 1) {
+    int pk = 0;
+    for (int si = 0; si < work.nseg; si++) {
+      const Segment sg = work.get(si);
+      if (is_whole(sg)) continue;
+      const int ps = pk & (kPartRing - 1);
+      if (!mbar_wait(part0 + 8 * ps, (uint32_t)(pk / kPartRing) & 1u)) {
+        if (lane == 0) atomicExch(p.ws_status, 4);
+        return;
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(done0 + 8 * ps);   // the ring slot may be used again
+      pk++;
+      if (!one_range && lane < M) {
+        int a = 0;
+        for (int st = sg.sb; st < sg.se; st++) a += s_T0st[lane * kMaxSps + st];
+        atomicAdd(p.ws_T0 + (size_t)sg.tile * M + lane, a);
+      }
+      __threadfence();
+      __syncwarp();
+      uint32_t old = 0;
+      if (lane == 0) old = atomicAdd(p.ws_count + sg.tile, (uint32_t)(sg.se - sg.sb));
+      old = __shfl_sync(0xffffffffu, old, 0);
+      if (old + (uint32_t)(sg.se - sg.sb) != (uint32_t)p.spt_all) continue;
+      __threadfence();
+      const int nout = kTileRows * M;
+      for (int idx = lane; idx < nout; idx += 32) {
+        const int r = idx / M, m = idx - r * M;
+        const int row = sg.tile * kTileRows + r;
+        if (row < p.N) {
+          int32_t* src = p.ws_sum + ((size_t)row * M + m) * 3;
+          const int T1 = __ldcg(src + 0), T2 = __ldcg(src + 1), T3 = __ldcg(src + 2);
+          src[0] = 0; src[1] = 0; src[2] = 0;
+          int T0;
+          if (one_range) {
+            T0 = 0;
+            for (int st = 0; st < spt; st++) T0 += s_T0st[m * kMaxSps + st];
+          } else {
+            T0 = __ldcg(p.ws_T0 + (size_t)sg.tile * M + m);
+          }
+          const int S3 = T3, S1 = T1 - T3, S2 = T2 - T3;
+          const int S0 = T0 - S1 - S2 - S3;
+          p.y[(size_t)m * p.N + row] = lut_finish(s_scale[m], __ldg(p.lut + row), S0, S1, S2, S3);
+        }
+      }
+      __syncwarp();
+      if (!one_range && lane < M) p.ws_T0[(size_t)sg.tile * M + lane] = 0;
+      if (lane == 0) p.ws_count[sg.tile] = 0u;
     }
     return;
   }
@@ -299,6 +351,7 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap tmap, const GemvParams p)
 #pragma unroll
   for (int tok = 0; tok < NTD; tok++) bD_lane[tok] = bs_u32 + (uint32_t)(tok * 64 + t * 16);
 
+  int part_k = 0;  // partial segments handed over so far
   uint2 lut_g[2];  // LUT rows g and g+8 of the current tile, fetched ahead of the epilogue
   auto fetch_lut = [&](int tile) {
 #pragma unroll
@@ -354,13 +407,20 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap tmap, const GemvParams p)
         }
     }
     const int row0 = sg.tile * kTileRows + warp * 16 + g;
-    const bool whole = (gridDim.y == 1) && sg.sb == 0 && sg.se == p.spt_all;
-    bool finish = true;
-    int T0v[NE];
+    if (is_whole(sg)) {
 #pragma unroll
-    for (int e = 0; e < NE; e++) T0v[e] = s_T0[etok[e] & (kMaxTokens - 1)];
-    if (!whole) {
-      // ---- partial rows: add into the scratch sums, the last contributor finishes
+      for (int e = 0; e < NE; e++) {
+        const int row = row0 + 8 * err[e];
+        if (etok[e] < M && row < p.N) {
+          int T0 = 0;
+          for (int st = 0; st < spt; st++) T0 += s_T0st[etok[e] * kMaxSps + st];
+          const int S3 = T3[e], S1 = T1[e] - T3[e], S2 = T2[e] - T3[e];
+          const int S0 = T0 - S1 - S2 - S3;
+          p.y[(size_t)etok[e] * p.N + row] = lut_finish(s_scale[etok[e]], lut_g[err[e]], S0, S1, S2, S3);
+        }
+      }
+    } else {
+      // partial rows: add into the scratch sums and hand the segment to the finishing warp
 #pragma unroll
       for (int e = 0; e < NE; e++) {
         const int row = row0 + 8 * err[e];
@@ -371,46 +431,15 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap tmap, const GemvParams p)
           atomicAdd(dst + 2, T3[e]);
         }
       }
-      const int grp = sg.tile * kCWarps + warp;
-      if (lane < M) {
-        int a = 0;
-        for (int st = sg.sb; st < sg.se; st++) a += s_T0st[lane * kMaxSps + st];
-        atomicAdd(p.ws_T0 + (size_t)grp * M + lane, a);
-      }
-      __threadfence();
+      const int ps = part_k & (kPartRing - 1);
+      bool ok = true;
+      if (part_k >= kPartRing) ok = mbar_wait(done0 + 8 * ps, (uint32_t)(part_k / kPartRing - 1) & 1u);
       __syncwarp();
-      uint32_t old = 0;
-      if (lane == 0) old = atomicAdd(p.ws_count + grp, (uint32_t)(sg.se - sg.sb));
-      old = __shfl_sync(0xffffffffu, old, 0);
-      finish = (old + (uint32_t)(sg.se - sg.sb) == (uint32_t)p.spt_all);
-      if (finish) {
-        __threadfence();
-#pragma unroll
-        for (int e = 0; e < NE; e++) {
-          const int row = row0 + 8 * err[e];
-          if (etok[e] < M && row < p.N) {
-            int32_t* src = p.ws_sum + ((size_t)row * M + etok[e]) * 3;
-            T1[e] = atomicExch(src + 0, 0);
-            T2[e] = atomicExch(src + 1, 0);
-            T3[e] = atomicExch(src + 2, 0);
-            T0v[e] = atomicAdd(p.ws_T0 + (size_t)grp * M + etok[e], 0);
-          }
-        }
-        __syncwarp();
-        if (lane < M) atomicExch(p.ws_T0 + (size_t)grp * M + lane, 0);
-        if (lane == 0) atomicExch(p.ws_count + grp, 0u);
+      if (lane == 0) {
+        if (ok) mbar_arrive(part0 + 8 * ps);
+        else atomicExch(p.ws_status, 5);
       }
-    }
-    if (finish) {
-#pragma unroll
-      for (int e = 0; e < NE; e++) {
-        const int row = row0 + 8 * err[e];
-        if (etok[e] < M && row < p.N) {
-          const int S3 = T3[e], S1 = T1[e] - T3[e], S2 = T2[e] - T3[e];
-          const int S0 = T0v[e] - S1 - S2 - S3;
-          p.y[(size_t)etok[e] * p.N + row] = lut_finish(s_scale[etok[e]], lut_g[err[e]], S0, S1, S2, S3);
-        }
-      }
+      part_k++;
     }
     zero_acc();
   };
@@ -419,7 +448,7 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap tmap, const GemvParams p)
   uint32_t phase = 0;
   for (int si = 0; si < work.nseg; si++) {
     const Segment sg = work.get(si);
-    fetch_lut(sg.tile);
+    if (is_whole(sg)) fetch_lut(sg.tile);
     uint32_t b_stage = (uint32_t)sg.sb * stage_stride;
     for (int st = sg.sb; st < sg.se; st++, b_stage += stage_stride) {
       if (!mbar_wait(full0 + 8 * slot, phase)) {

@@ -54,19 +54,18 @@ StreamPlan make_plan(int M, int N, int K) {
   pl.supers = (pl.spt_all + sps - 1) / sps;
   pl.sps = (pl.spt_all + pl.supers - 1) / pl.supers;
   const size_t bs_bytes = (size_t)pl.sps * bs_per_stage;
-  const size_t misc = 128 + (size_t)M * rcp::kMaxSps * 4 + 64 + 64;
+  const size_t misc = 256 + (size_t)M * rcp::kMaxSps * 4 + 64 + 64;
   pl.stages = (int)std::min<size_t>(rcp::kMaxStages, (kSmemMax - 1024 - misc - bs_bytes) / rcp::kStageBytes);
   size_t off = (size_t)pl.stages * rcp::kStageBytes;
-  pl.off_bar = (int)off; off += 128;
+  pl.off_bar = (int)off; off += 256;
   pl.off_T0st = (int)off; off += (size_t)M * rcp::kMaxSps * 4;
   pl.off_T0 = (int)off; off += 64;
   pl.off_scale = (int)off; off += 64;
   pl.off_bs = (int)off; off += bs_bytes;
   pl.smem = off + 1024;
   pl.ws_count_off = 16;
-  const size_t groups = (size_t)pl.ntiles * rcp::kCWarps;
-  pl.ws_T0_off = pl.ws_count_off + ((groups * 4 + 15) / 16) * 16;
-  pl.ws_sum_off = pl.ws_T0_off + ((groups * M * 4 + 15) / 16) * 16;
+  pl.ws_T0_off = pl.ws_count_off + (((size_t)pl.ntiles * 4 + 15) / 16) * 16;
+  pl.ws_sum_off = pl.ws_T0_off + (((size_t)pl.ntiles * M * 4 + 15) / 16) * 16;
   pl.ws_bytes = pl.ws_sum_off + (size_t)pl.ntiles * rcp::kTileRows * M * 3 * 4;
   return pl;
 }
