@@ -125,6 +125,36 @@ int rcp_linear_w2a4_host(const void* x_host_f16, int M, int K, int had_block, fl
                          void* x_dev, uint8_t* xq_dev, void* scale_dev, void* y_dev, void* workspace,
                          void* stream);
 
+/*
+ * LUT GEMV for callers that cannot allocate device memory. (The paper has no counterpart: this
+ * entry point exists for the way the library is embedded, not for the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a plug-in inside a serving
+ * process whose memory has all been handed to a pool allocator up front, a real-time decode loop
+ * that cannot afford the device-wide synchronization an allocation implies, or a host that is
+ * already inside a region where allocating calls are forbidden. Such callers can supply inputs
+ * and outputs they were given, but not the scratch buffer rcp_gemv_w2a4 asks for.
+ *
+ * What it does: the same computation as rcp_gemv_w2a4 (variant RCP_GEMV_AUTO, same arguments, same
+ * results), with the scratch taken from an array of RCP_STATIC_SCRATCH_BYTES bytes that is part of
+ * the library's device image. Every GPU that loads the library holds that array until the process
+ * exits. The call makes no cudaMalloc, cudaFree or other allocating call.
+ *
+ *   - Shapes whose scratch (rcp_gemv_workspace_bytes) exceeds RCP_STATIC_SCRATCH_BYTES are rejected
+ *     with RCP_ERR_LIMIT; nothing is launched.
+ *   - The first call on each device looks up the array's device address (once per device, with that
+ *     device current) and remembers it. Make that first call outside any stream capture.
+ *   - The array is shared by every call on the device and keeps whatever the previous call left in
+ *     it; each call therefore clears the part it is about to use, on `stream`, before its kernel.
+ *   - Because the array is shared, two calls that may overlap on the GPU (different streams, or
+ *     different host threads launching concurrently) race on it. Serialize them, or give the
+ *     overlapping work to rcp_gemv_w2a4 with scratch buffers of its own.
+ * Never synchronizes.
+ */
+#define RCP_STATIC_SCRATCH_BYTES (4u << 20)
+int rcp_gemv_w2a4_static(const uint32_t* words, const void* lut_f16, const uint8_t* xq,
+                         const void* scale_f16, int M, int N, int K, void* y_f16, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -49,6 +49,8 @@ def lib():
         L.rcp_gemv_w2a4_variant.argtypes = [i, vp, vp, vp, vp, i, i, i, vp, vp, vp, vp]
         L.rcp_linear_w2a4_host.restype = i
         L.rcp_linear_w2a4_host.argtypes = [vp, i, i, i, C.c_float, vp, vp, i, vp, vp, vp, vp, vp, vp, vp]
+        L.rcp_gemv_w2a4_static.restype = i
+        L.rcp_gemv_w2a4_static.argtypes = [vp, vp, vp, vp, i, i, i, vp, vp]
         _lib = L
     return _lib
 
@@ -128,6 +130,32 @@ def rcp_gemv_w2a4(words, lut, xq, scale, y=None, workspace=None, S_dbg=None, var
         _check("rcp_gemv_w2a4",
                lib().rcp_gemv_w2a4_variant(v, _ptr(words), _ptr(lut), _ptr(xq), _ptr(scale), M, N, K, _ptr(y),
                                            _ptr(workspace), _ptr(S_dbg), _stream(words)))
+    return y
+
+
+STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def rcp_gemv_w2a4_static(words, lut, xq, scale, y=None):
+    """Same result as rcp_gemv_w2a4, for callers that may not allocate device memory: the scratch
+    is an array inside the library (STATIC_SCRATCH_BYTES, shared by all calls on the device, so
+    calls that can overlap on the GPU must be serialized). Pass `y` to keep this wrapper from
+    allocating the output; shapes that need more scratch raise RcpError with status -8."""
+    _dev(words, torch.int32, "words")
+    _dev(lut, torch.float16, "lut")
+    _dev(xq, torch.uint8, "xq")
+    _dev(scale, torch.float16, "scale")
+    N, W = words.shape
+    K = W * 16
+    M = xq.shape[0]
+    if xq.shape != (M, K // 2) or lut.shape != (N, 4) or scale.shape != (M,):
+        raise ValueError("shape mismatch between words, lut, xq and scale")
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.float16, device=words.device)
+    with torch.cuda.device(words.device):
+        _check("rcp_gemv_w2a4_static",
+               lib().rcp_gemv_w2a4_static(_ptr(words), _ptr(lut), _ptr(xq), _ptr(scale), M, N, K, _ptr(y),
+                                          _stream(words)))
     return y
 
 

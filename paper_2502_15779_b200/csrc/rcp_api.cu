@@ -3,6 +3,7 @@
 
 #include <algorithm>
 #include <cmath>
+#include <mutex>
 
 #include "common.cuh"
 #include "gemv_simple.cuh"
@@ -152,6 +153,30 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   return launch_stream_t<2, rcp::kModeMma, 0>(map, gp, pl, st);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Scratch of rcp_gemv_w2a4_static: part of the device image, one copy per GPU that loads the library.
+static __device__ __align__(256) unsigned char g_static_scratch[RCP_STATIC_SCRATCH_BYTES];
+
+// Device address of g_static_scratch on the current device. In host code the array's name only
+// stands for the symbol; the address a kernel can use comes from cudaGetSymbolAddress, asked once
+// per device with that device current and remembered afterwards.
+int static_scratch_address(void** out) {
+  constexpr int kMaxDevices = 64;
+  static std::mutex mu;
+  static void* addr[kMaxDevices] = {};
+  int dev = 0;
+  RCP_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return RCP_ERR_LIMIT;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!addr[dev]) {
+    void* p = nullptr;
+    RCP_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));
+    addr[dev] = p;
+  }
+  *out = addr[dev];
+  return RCP_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -280,6 +305,19 @@ int rcp_gemv_w2a4(const uint32_t* words, const void* lut_f16, const uint8_t* xq,
                   int M, int N, int K, void* y_f16, void* workspace, int32_t* S_dbg, void* stream) {
   return rcp_gemv_w2a4_variant(RCP_GEMV_AUTO, words, lut_f16, xq, scale_f16, M, N, K, y_f16, workspace,
                                S_dbg, stream);
+}
+
+int rcp_gemv_w2a4_static(const uint32_t* words, const void* lut_f16, const uint8_t* xq, const void* scale_f16,
+                         int M, int N, int K, void* y_f16, void* stream) {
+  const size_t need = rcp_gemv_workspace_bytes(M, N, K);   // 0 on a bad shape: reported by the call below
+  if (need > RCP_STATIC_SCRATCH_BYTES) return RCP_ERR_LIMIT;
+  void* scratch = nullptr;
+  const int rc = static_scratch_address(&scratch);
+  if (rc != RCP_OK) return rc;
+  // the array keeps the previous call's contents: clear what this call's kernel expects to be zero
+  if (need > 0) RCP_CUDA(cudaMemsetAsync(scratch, 0, need, static_cast<cudaStream_t>(stream)));
+  return rcp_gemv_w2a4_variant(RCP_GEMV_AUTO, words, lut_f16, xq, scale_f16, M, N, K, y_f16, scratch, nullptr,
+                               stream);
 }
 
 int rcp_linear_w2a4_host(const void* x_host_f16, int M, int K, int had_block, float clip_ratio,

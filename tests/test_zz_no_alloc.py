@@ -1,0 +1,75 @@
+"""rcp_gemv_w2a4_static: the LUT GEMV for callers that are not allowed to allocate device memory
+(a plug-in in a process whose memory belongs to a pool, a decode loop that cannot take the
+synchronization an allocation brings). Its scratch is an array inside the library instead of a
+caller buffer, so the checks here are the ones that matter to such a caller: called through the C
+ABI with nothing but inputs and outputs, it must give what rcp_gemv_w2a4 gives, also the second
+time, when the shared array still holds whatever the first call left behind; and a shape that
+needs more scratch than the array has must be refused before anything is launched.
+
+This file sorts after the other test files on purpose: a run that stops at the first failure has
+then already run everything else."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2502_15779_b200 as rcp
+from paper_2502_15779_b200 import synth
+from helpers import f16_bits
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _inputs(N, K, B, M, seed):
+    codes, lut = synth.make_layer(N, K, B, "rotated_laplace", seed, device=DEV)
+    x = synth.make_activations(M, K, seed, device=DEV)
+    words = rcp.rcp_pack_weights(codes)
+    xq, scale = rcp.rcp_quantize_act(x, B, 1.0)
+    return words, lut, xq, scale
+
+
+@pytest.mark.parametrize("N,K,B,M", [(300, 2048, 2048, 1), (1000, 2560, 128, 3), (4096, 4096, 4096, 2)])
+def test_static_scratch_entry_matches_existing_entry_twice_in_a_row(N, K, B, M):
+    words, lut, xq, scale = _inputs(N, K, B, M, seed=N + K + M)
+    # the existing entry point, with a caller-provided scratch buffer
+    ws = rcp.make_workspace(M, N, K, DEV)
+    y_ref = rcp.rcp_gemv_w2a4(words, lut, xq, scale, workspace=ws)
+    # tolerance of the GEMV parity tests: |y - y_ref| <= 2e-3 * (s * sum_c |LUT[c]| |S_c|) + 1e-5, from the oracle
+    orc = oracle.gemv_w2a4(words.cpu().numpy().view(np.uint32), f16_bits(lut), xq.cpu().numpy(), f16_bits(scale))
+    tol = orc["tol"]
+    # the new entry point, straight through the C ABI: inputs and outputs only, on the current stream
+    L = rcp.lib()
+    y = torch.empty(M, N, dtype=torch.float16, device=DEV)
+    stream = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    args = (C.c_void_p(words.data_ptr()), C.c_void_p(lut.data_ptr()), C.c_void_p(xq.data_ptr()),
+            C.c_void_p(scale.data_ptr()), M, N, K, C.c_void_p(y.data_ptr()), stream)
+    want = y_ref.float().cpu().numpy().astype(np.float64)
+    for call in range(2):  # the second call meets the array as the first one left it
+        y.fill_(float("nan"))
+        assert L.rcp_gemv_w2a4_static(*args) == 0
+        torch.cuda.synchronize()
+        got = y.float().cpu().numpy().astype(np.float64)
+        assert np.all(np.isfinite(got)), f"call {call}"
+        assert np.all(np.abs(got - want) <= tol), f"call {call}: max diff/tol {np.max(np.abs(got - want) / tol)}"
+        assert np.all(np.abs(got - orc["y"]) <= tol), f"call {call}"
+
+
+def test_static_scratch_entry_rejects_shapes_beyond_its_array():
+    # scratch grows with N * M; find a shape past the limit without allocating anything that large
+    N, K, M = 600000, 64, 16
+    assert rcp.rcp_gemv_workspace_bytes(M, N, K) > rcp.binding.STATIC_SCRATCH_BYTES
+    z = torch.zeros(64, dtype=torch.int32, device=DEV)
+    p = C.c_void_p(z.data_ptr())
+    # refused on size alone, before any pointer is touched
+    assert rcp.lib().rcp_gemv_w2a4_static(p, p, p, p, M, N, K, p, None) == -8
+    assert rcp.lib().rcp_status_str(-8) not in (None, b"")
+    # a bad shape is still reported as such
+    assert rcp.lib().rcp_gemv_w2a4_static(p, p, p, p, 1, 16, 96, p, None) == -2
+    # and the wrapper raises
+    words, lut, xq, scale = _inputs(64, 256, 128, 1, seed=3)
+    y = rcp.rcp_gemv_w2a4_static(words, lut, xq, scale)
+    ws = rcp.make_workspace(1, 64, 256, DEV)
+    assert torch.equal(y.view(torch.int16), rcp.rcp_gemv_w2a4(words, lut, xq, scale, workspace=ws).view(torch.int16))
