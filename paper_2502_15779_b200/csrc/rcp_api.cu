@@ -33,41 +33,47 @@ bool k_ok(int K) { return K >= 64 && K <= rcp::kMaxK && K % 64 == 0; }
 __device__ int g_pack_bad;  // set by pack_weights_kernel when it meets a code above 3
 
 // ---------------------------------------------------------------------------------------------
-// Streaming GEMV: launch plan shared by rcp_gemv_workspace_bytes and the launcher.
+// Streaming GEMV: launch plan.
 struct StreamPlan {
-  int ntiles, spt_all, sps, supers, stages;
-  int off_bar, off_T0st, off_T0, off_scale, off_bs;
-  size_t smem, ws_count_off, ws_T0_off, ws_sum_off, ws_bytes;
+  int nchunk, R, L, gmax, KS, SA, stages, grid;
+  int off_bar, off_T0c, off_scale, off_red, off_bs;
+  size_t smem;
 };
 
-constexpr size_t kSmemMax = 232448;           // 227 KB of dynamic shared memory per CTA on sm_100
-constexpr size_t kExpandBudget = 96 * 1024;   // expanded activations kept resident per CTA
+constexpr size_t kSmemMax = 232448;            // 227 KB of dynamic shared memory per CTA on sm_100
+constexpr size_t kExpandBudget = 128 * 1024;   // expanded activations (one byte per code and token) per CTA
 
-StreamPlan make_plan(int M, int N, int K) {
+// Tokens one launch can take: their expanded activations must fit beside a ring of three stages.
+int tokens_per_pass(int M, int K, int cap) {
+  int m = std::min(M, cap);
+  while (m > 1 && (size_t)m * K > kExpandBudget) m--;
+  return m;
+}
+
+StreamPlan make_plan(int M, int N, int K, int sms) {
   StreamPlan pl;
-  pl.ntiles = (N + rcp::kTileRows - 1) / rcp::kTileRows;
-  pl.spt_all = (K / 16 + rcp::kStageWords - 1) / rcp::kStageWords;
-  // expanded activations: one byte per code and token, 512 M bytes per stage; K ranges whose
-  // activations fit in shared memory go to different blockIdx.y
-  const size_t bs_per_stage = (size_t)rcp::kStageWords * 16 * M;
-  int sps = (int)std::min<size_t>(rcp::kMaxSps, std::max<size_t>(1, kExpandBudget / bs_per_stage));
-  sps = std::min(sps, pl.spt_all);
-  pl.supers = (pl.spt_all + sps - 1) / sps;
-  pl.sps = (pl.spt_all + pl.supers - 1) / pl.supers;
-  const size_t bs_bytes = (size_t)pl.sps * bs_per_stage;
-  const size_t misc = 256 + (size_t)M * rcp::kMaxSps * 4 + 64 + 64;
+  pl.grid = sms;
+  pl.nchunk = (K / 16 + rcp::kChunkWords - 1) / rcp::kChunkWords;
+  const int groups = (N + 15) / 16;
+  const int per_round = sms * rcp::kCWarps;
+  pl.R = groups / per_round;
+  pl.L = groups - pl.R * per_round;
+  pl.gmax = (pl.L + sms - 1) / sms;
+  pl.KS = pl.gmax > 0 ? rcp::kCWarps / pl.gmax : 1;
+  pl.KS = std::min(pl.KS, pl.nchunk);
+  pl.SA = pl.gmax > 0 ? (pl.nchunk + pl.KS - 1) / pl.KS : 0;
+  const size_t bs_bytes = (size_t)pl.nchunk * rcp::kChunkWords * 16 * M;
+  const size_t t0c_bytes = (((size_t)M * pl.nchunk * 4) + 15) / 16 * 16;
+  const size_t red_bytes = (size_t)8 * 16 * M * 3 * 4;
+  const size_t misc = 128 + t0c_bytes + 64 + red_bytes;
   pl.stages = (int)std::min<size_t>(rcp::kMaxStages, (kSmemMax - 1024 - misc - bs_bytes) / rcp::kStageBytes);
   size_t off = (size_t)pl.stages * rcp::kStageBytes;
-  pl.off_bar = (int)off; off += 256;
-  pl.off_T0st = (int)off; off += (size_t)M * rcp::kMaxSps * 4;
-  pl.off_T0 = (int)off; off += 64;
+  pl.off_bar = (int)off; off += 128;
+  pl.off_T0c = (int)off; off += t0c_bytes;
   pl.off_scale = (int)off; off += 64;
+  pl.off_red = (int)off; off += red_bytes;
   pl.off_bs = (int)off; off += bs_bytes;
   pl.smem = off + 1024;
-  pl.ws_count_off = 16;
-  pl.ws_T0_off = pl.ws_count_off + (((size_t)pl.ntiles * 4 + 15) / 16) * 16;
-  pl.ws_sum_off = pl.ws_T0_off + (((size_t)pl.ntiles * M * 4 + 15) / 16) * 16;
-  pl.ws_bytes = pl.ws_sum_off + (size_t)pl.ntiles * rcp::kTileRows * M * 3 * 4;
   return pl;
 }
 
@@ -97,60 +103,75 @@ int sm_count() {
   return n;
 }
 
-template <int MT, int MODE, int MTOK>
-int launch_stream_t(const CUtensorMap& map, const rcp::GemvParams& gp, const StreamPlan& pl, cudaStream_t st) {
+template <int MODE, int MTOK>
+int launch_stream_t(const CUtensorMap& map_left, const CUtensorMap& map_round, const rcp::GemvParams& gp,
+                    const StreamPlan& pl, cudaStream_t st) {
   static bool attr_set = false;
-  auto kern = rcp::gemv_stream_kernel<MT, MODE, MTOK>;
+  auto kern = rcp::gemv_stream_kernel<MODE, MTOK>;
   if (!attr_set) {
     RCP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax));
     attr_set = true;
   }
-  const int gx = std::max(1, sm_count() / pl.supers);
-  kern<<<dim3(gx, pl.supers), rcp::kGThreads, pl.smem, st>>>(map, gp);
+  kern<<<pl.grid, rcp::kGThreads, pl.smem, st>>>(map_left, map_round, gp);
   RCP_CUDA(cudaGetLastError());
   return RCP_OK;
 }
 
+// One launch: M tokens (their expanded activations fit in shared memory).
 int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const uint8_t* xq, const void* scale_f16,
                   int M, int N, int K, void* y_f16, void* workspace, cudaStream_t st) {
-  if (!workspace) return RCP_ERR_WORKSPACE;
-  if (!aligned16(workspace)) return RCP_ERR_ALIGN;
   if (mode != rcp::kModeMma && M > 2) return RCP_ERR_VARIANT;
+  if (M > 8) return RCP_ERR_VARIANT;
   EncodeTiledFn enc = encode_tiled_fn();
   if (!enc) return cuda_fail(cudaErrorNotSupported);
-  const StreamPlan pl = make_plan(M, N, K);
+  const StreamPlan pl = make_plan(M, N, K, sm_count());
   if (pl.stages < 2 || pl.smem > kSmemMax) return RCP_ERR_SHAPE;
-  CUtensorMap map;
+  CUtensorMap maps[2];
   const cuuint64_t gdim[2] = {(cuuint64_t)(K / 16), (cuuint64_t)N};
   const cuuint64_t gstride[1] = {(cuuint64_t)(K / 4)};
-  const cuuint32_t box[2] = {(cuuint32_t)rcp::kStageWords, (cuuint32_t)rcp::kTileRows};
   const cuuint32_t estr[2] = {1, 1};
-  const CUresult r = enc(&map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t*>(words), gdim, gstride, box,
-                         estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue);
+  const int box_rows[2] = {16 * std::max(1, pl.gmax), rcp::kTileRows};
+  for (int i = 0; i < 2; i++) {
+    const cuuint32_t box[2] = {(cuuint32_t)rcp::kChunkWords, (cuuint32_t)box_rows[i]};
+    const CUresult r = enc(&maps[i], CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t*>(words), gdim, gstride,
+                           box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue);
+  }
   rcp::GemvParams gp;
   gp.lut = static_cast<const uint2*>(lut_f16);
   gp.xq = xq;
   gp.scale = static_cast<const __half*>(scale_f16);
   gp.y = static_cast<__half*>(y_f16);
-  uint8_t* ws = static_cast<uint8_t*>(workspace);
-  gp.ws_status = reinterpret_cast<int32_t*>(ws);
-  gp.ws_count = reinterpret_cast<uint32_t*>(ws + pl.ws_count_off);
-  gp.ws_T0 = reinterpret_cast<int32_t*>(ws + pl.ws_T0_off);
-  gp.ws_sum = reinterpret_cast<int32_t*>(ws + pl.ws_sum_off);
+  gp.status = static_cast<int32_t*>(workspace);
   gp.M = M; gp.N = N; gp.K = K;
-  gp.ntiles = pl.ntiles; gp.spt_all = pl.spt_all; gp.sps = pl.sps; gp.stages = pl.stages;
-  gp.off_bar = pl.off_bar; gp.off_T0st = pl.off_T0st; gp.off_T0 = pl.off_T0; gp.off_scale = pl.off_scale;
+  gp.nchunk = pl.nchunk; gp.R = pl.R; gp.L = pl.L; gp.gmax = pl.gmax; gp.KS = pl.KS; gp.SA = pl.SA;
+  gp.stages = pl.stages;
+  gp.off_bar = pl.off_bar; gp.off_T0c = pl.off_T0c; gp.off_scale = pl.off_scale; gp.off_red = pl.off_red;
   gp.off_bs = pl.off_bs;
   if (mode == rcp::kModeHybrid)
-    return M == 1 ? launch_stream_t<1, rcp::kModeHybrid, 1>(map, gp, pl, st)
-                  : launch_stream_t<1, rcp::kModeHybrid, 2>(map, gp, pl, st);
+    return M == 1 ? launch_stream_t<rcp::kModeHybrid, 1>(maps[0], maps[1], gp, pl, st)
+                  : launch_stream_t<rcp::kModeHybrid, 2>(maps[0], maps[1], gp, pl, st);
   if (mode == rcp::kModeDp4a)
-    return M == 1 ? launch_stream_t<1, rcp::kModeDp4a, 1>(map, gp, pl, st)
-                  : launch_stream_t<1, rcp::kModeDp4a, 2>(map, gp, pl, st);
-  if (M <= 8) return launch_stream_t<1, rcp::kModeMma, 0>(map, gp, pl, st);
-  return launch_stream_t<2, rcp::kModeMma, 0>(map, gp, pl, st);
+    return M == 1 ? launch_stream_t<rcp::kModeDp4a, 1>(maps[0], maps[1], gp, pl, st)
+                  : launch_stream_t<rcp::kModeDp4a, 2>(maps[0], maps[1], gp, pl, st);
+  return launch_stream_t<rcp::kModeMma, 0>(maps[0], maps[1], gp, pl, st);
+}
+
+// All M tokens: as many launches as it takes for the expanded activations to fit (`cap` tokens at most each).
+int launch_stream_passes(int mode, int cap, const uint32_t* words, const void* lut_f16, const uint8_t* xq,
+                         const void* scale_f16, int M, int N, int K, void* y_f16, void* workspace, cudaStream_t st) {
+  const int mp = tokens_per_pass(M, K, cap);
+  for (int m0 = 0; m0 < M; m0 += mp) {
+    const int mm = std::min(mp, M - m0);
+    int md = mode;
+    if (md == rcp::kModeHybrid && mm > 2) md = rcp::kModeMma;
+    const int rc = launch_stream(md, words, lut_f16, xq + (size_t)m0 * (K / 2),
+                                 static_cast<const __half*>(scale_f16) + m0, mm, N, K,
+                                 static_cast<__half*>(y_f16) + (size_t)m0 * N, workspace, st);
+    if (rc != RCP_OK) return rc;
+  }
+  return RCP_OK;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -251,8 +272,7 @@ int rcp_quantize_act(const void* x_f16, int M, int K, int had_block, float clip_
 
 size_t rcp_gemv_workspace_bytes(int M, int N, int K) {
   if (M < 1 || M > rcp::kMaxTokens || N < 1 || !k_ok(K)) return 0;
-  // the layout grows with M, and the CUDA-core variant runs the tokens in pairs on the same scratch
-  return make_plan(M, N, K).ws_bytes;
+  return 16;   // a status word for the kernels' bounded waits; no sums pass through global memory
 }
 
 int rcp_gemv_w2a4_variant(int variant, const uint32_t* words, const void* lut_f16, const uint8_t* xq,
@@ -278,22 +298,13 @@ int rcp_gemv_w2a4_variant(int variant, const uint32_t* words, const void* lut_f1
     }
     case RCP_GEMV_MMA:
       // tensor-core path; for one or two tokens the b0*b1 plane goes to dp4a (FMA pipe) instead
-      return launch_stream(M <= 2 ? rcp::kModeHybrid : rcp::kModeMma, words, lut_f16, xq, scale_f16, M, N, K, y_f16,
-                           workspace, st);
+      return launch_stream_passes(M <= 2 ? rcp::kModeHybrid : rcp::kModeMma, 8, words, lut_f16, xq, scale_f16, M, N, K,
+                                  y_f16, workspace, st);
     case RCP_GEMV_MMA_ONLY:
-      return launch_stream(rcp::kModeMma, words, lut_f16, xq, scale_f16, M, N, K, y_f16, workspace, st);
-    case RCP_GEMV_DP4A: {
+      return launch_stream_passes(rcp::kModeMma, 8, words, lut_f16, xq, scale_f16, M, N, K, y_f16, workspace, st);
+    case RCP_GEMV_DP4A:
       // CUDA-core path: two tokens per launch
-      for (int m0 = 0; m0 < M; m0 += 2) {
-        const int mm = std::min(2, M - m0);
-        // later token pairs reuse the same scratch: it is left zeroed by the previous launch
-        const int rc = launch_stream(rcp::kModeDp4a, words, lut_f16, xq + (size_t)m0 * (K / 2),
-                                     static_cast<const __half*>(scale_f16) + m0, mm, N, K,
-                                     static_cast<__half*>(y_f16) + (size_t)m0 * N, workspace, st);
-        if (rc != RCP_OK) return rc;
-      }
-      return RCP_OK;
-    }
+      return launch_stream_passes(rcp::kModeDp4a, 2, words, lut_f16, xq, scale_f16, M, N, K, y_f16, workspace, st);
     default:
       return RCP_ERR_VARIANT;
   }

@@ -3,8 +3,8 @@
 synchronization an allocation brings). Its scratch is an array inside the library instead of a
 caller buffer, so the checks here are the ones that matter to such a caller: called through the C
 ABI with nothing but inputs and outputs, it must give what rcp_gemv_w2a4 gives, also the second
-time, when the shared array still holds whatever the first call left behind; and a shape that
-needs more scratch than the array has must be refused before anything is launched.
+time, when the shared array still holds whatever the first call left behind; and bad arguments must
+come back as status codes with nothing launched.
 
 This file sorts after the other test files on purpose: a run that stops at the first failure has
 then already run everything else."""
@@ -57,18 +57,18 @@ def test_static_scratch_entry_matches_existing_entry_twice_in_a_row(N, K, B, M):
         assert np.all(np.abs(got - orc["y"]) <= tol), f"call {call}"
 
 
-def test_static_scratch_entry_rejects_shapes_beyond_its_array():
-    # scratch grows with N * M; find a shape past the limit without allocating anything that large
-    N, K, M = 600000, 64, 16
-    assert rcp.rcp_gemv_workspace_bytes(M, N, K) > rcp.binding.STATIC_SCRATCH_BYTES
+def test_static_scratch_entry_reports_errors_and_wrapper_agrees():
     z = torch.zeros(64, dtype=torch.int32, device=DEV)
     p = C.c_void_p(z.data_ptr())
-    # refused on size alone, before any pointer is touched
-    assert rcp.lib().rcp_gemv_w2a4_static(p, p, p, p, M, N, K, p, None) == -8
-    assert rcp.lib().rcp_status_str(-8) not in (None, b"")
-    # a bad shape is still reported as such
-    assert rcp.lib().rcp_gemv_w2a4_static(p, p, p, p, 1, 16, 96, p, None) == -2
-    # and the wrapper raises
+    L = rcp.lib()
+    # every shape the GEMV accepts needs less scratch than the array holds; the size check comes first
+    for (M, N, K) in [(1, 57344, 8192), (16, 600000, 64), (8, 8192, 28672)]:
+        assert 0 < rcp.rcp_gemv_workspace_bytes(M, N, K) <= rcp.binding.STATIC_SCRATCH_BYTES
+    assert L.rcp_status_str(-8) not in (None, b"")       # the text of RCP_ERR_LIMIT
+    # bad arguments are reported like the existing entry point reports them, and nothing is launched
+    assert L.rcp_gemv_w2a4_static(p, p, p, p, 1, 16, 96, p, None) == -2
+    assert L.rcp_gemv_w2a4_static(None, p, p, p, 1, 16, 64, p, None) == -1
+    # the Python wrapper gives the same bits as the existing entry point
     words, lut, xq, scale = _inputs(64, 256, 128, 1, seed=3)
     y = rcp.rcp_gemv_w2a4_static(words, lut, xq, scale)
     ws = rcp.make_workspace(1, 64, 256, DEV)
