@@ -16,14 +16,14 @@
 // producer thread streams boxes of rows x 128 bytes into a shared-memory ring with TMA
 // (cp.async.bulk.tensor, 128B swizzle, mbarrier completion); sixteen consumer warps read their MMA
 // fragments bank-conflict free and keep the partial sums in registers.
-//   Rounds. Groups of 16 rows are the unit of work. As long as 16 groups per CTA are left, every
-//   CTA takes a 256-row tile (one 32 KB box per stage, tiles dealt round-robin so that the GPU
-//   sweeps memory in order) and every warp owns one group over the whole K: nobody waits on
-//   anybody, each warp finishes its rows from its registers.
-//   Leftover. The remaining groups are shared out evenly, gmax = ceil(leftover / CTAs) per CTA,
-//   and come first. A CTA then loads boxes of 16 gmax rows, KS = 16 / gmax boxes (consecutive
-//   128-byte chunks of K) per stage, and KS warps split the K range of a group between them;
-//   their sums meet in shared memory (integer atomics) and one warp per group finishes.
+//   Groups of 16 rows are the unit of work, and the work is cut into phases. In a phase every
+//   CTA takes gpc consecutive groups (gpc = 16, 8, 4, 2 or 1) and KS = 16 / gpc warps share a
+//   group, each taking every KS-th 128-byte chunk of K; a stage of the ring is KS boxes of
+//   16 gpc rows x 128 bytes (32 KB). With gpc = 16 (as many rounds as the row count allows, tiles
+//   dealt round-robin so that the GPU sweeps memory in order) a warp owns its group over the whole
+//   K and finishes its rows from its registers. The groups left over go in phases of 8, 4, 2, 1
+//   groups per CTA, so that all sixteen warps stay busy; there the sums of the KS warps of a group
+//   meet in shared memory (integer atomics) and one of them finishes the rows.
 // Nothing is exchanged between CTAs, no scratch memory is needed, and the result does not depend
 // on timing. The int4 activations are expanded once per CTA into the B-operand byte layout in
 // shared memory.
@@ -45,6 +45,13 @@ constexpr uint32_t kSpinLimit = 1u << 22;         // bounded waits: give up, fla
 
 enum GemvMode { kModeMma = 0, kModeHybrid = 1, kModeDp4a = 2 };
 
+constexpr int kMaxPhases = 6;
+// One phase, repeated reps times: `total` groups starting at group first + rep * total are shared out
+// evenly over the CTAs b < ncta, CTA b taking groups [total b / ncta, total (b+1) / ncta) of them,
+// at most gpc. KS = 16 / gpc warps share a group; the TMA box has 16 gpc rows.
+struct GemvPhase { int gpc, first, total, ncta, reps; };
+struct GemvMaps { CUtensorMap m[kMaxPhases]; };   // box of 16 gpc rows x 128 bytes for phase i
+
 struct GemvParams {
   const uint2* lut;
   const uint8_t* xq;
@@ -53,10 +60,8 @@ struct GemvParams {
   int32_t* status;      // optional: receives a code when a bounded wait gives up
   int M, N, K;
   int nchunk;           // 128-byte chunks per row, ceil(K / 512)
-  int R;                // rounds of 256-row tiles
-  int L;                // leftover groups, starting at group R * gridDim.x * 16
-  int gmax, KS;         // leftover: groups per CTA at most, warps per group
-  int SA;               // leftover: stages, ceil(nchunk / KS)
+  int nphase;
+  GemvPhase phase[kMaxPhases];
   int stages;           // ring depth
   int off_bar, off_T0c, off_scale, off_red, off_bs;   // shared-memory byte offsets from the aligned base
 };
@@ -124,8 +129,7 @@ __device__ __forceinline__ void dp4a_u8s8(int& d, uint32_t a, uint32_t b) {
 // MTOK  tokens, fixed at compile time for the dp4a modes (1 or 2); 0 = run-time, up to 8 (kModeMma)
 template <int MODE, int MTOK>
 __global__ void __launch_bounds__(kGThreads, 1)
-gemv_stream_kernel(const __grid_constant__ CUtensorMap map_left, const __grid_constant__ CUtensorMap map_round,
-                   const GemvParams p) {
+gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;           // TMA 128B swizzle wants 1024-byte alignment
@@ -138,44 +142,39 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_left, const __grid_co
   const uint32_t full0 = base + p.off_bar, empty0 = full0 + 8 * kMaxStages;
   int* const s_T0c = reinterpret_cast<int*>(gen + p.off_T0c);           // [M][nchunk]: sum of q per chunk
   float* const s_scale = reinterpret_cast<float*>(gen + p.off_scale);   // [16]
-  int* const s_red = reinterpret_cast<int*>(gen + p.off_red);           // [8 groups][16 rows][M][3]
+  int* const s_red = reinterpret_cast<int*>(gen + p.off_red);           // [2][8 groups][16 rows][M][3]
   uint8_t* const bs = gen + p.off_bs;
-
-  // ------------------------------------------------------------------ this CTA's share
-  const int G = gridDim.x, b = blockIdx.x;
-  const int lo = (int)((long long)p.L * b / G), hi = (int)((long long)p.L * (b + 1) / G);
-  const int gpc = hi - lo;                                   // leftover groups of this CTA (<= gmax)
-  const int left_row0 = (p.R * G * kCWarps + lo) * 16;       // first row of its leftover box
-  const int SA = gpc > 0 ? p.SA : 0;
-  const int KS = p.KS;
-  const uint32_t box_left = (uint32_t)p.gmax * kGroupBytes;  // bytes of one leftover box
-  if (SA == 0 && p.R == 0) return;
 
   // ------------------------------------------------------------------ producer
   // The weights do not depend on the preceding kernel: start streaming at once.
-  int pr_n = 0, pr_slot = 0;                   // stages issued so far: SA leftover stages, then R * nchunk
+  const int G = gridDim.x, b = blockIdx.x;
+  int pr_ph = 0, pr_rep = 0, pr_s = 0, pr_slot = 0;   // next stage to request: phase, repetition, stage
   uint32_t pr_phase = 0;
-  const int pr_total = SA + p.R * p.nchunk;
-  int pr_round = 0, pr_c = 0;
+  auto pr_skip = [&]() {  // moves on to the next phase this CTA takes part in
+    while (pr_ph < p.nphase && b >= p.phase[pr_ph].ncta) pr_ph++;
+  };
   auto produce = [&]() {  // one stage; the producer thread only
+    const GemvPhase ph = p.phase[pr_ph];
+    const int KS = kCWarps / ph.gpc;
     const uint32_t bar = full0 + 8 * pr_slot, dst = base + (uint32_t)pr_slot * kStageBytes;
-    if (pr_n < SA) {
-      mbar_expect_tx(bar, (uint32_t)KS * box_left);
-      for (int j = 0; j < KS; j++)
-        tma_load_2d(dst + (uint32_t)j * box_left, &map_left, (pr_n * KS + j) * kChunkWords, left_row0, bar);
-    } else {
-      mbar_expect_tx(bar, kStageBytes);
-      tma_load_2d(dst, &map_round, pr_c * kChunkWords, (pr_round * G + b) * kTileRows, bar);
-      if (++pr_c == p.nchunk) { pr_c = 0; pr_round++; }
+    const uint32_t box = (uint32_t)ph.gpc * kGroupBytes;
+    const int row0 = (ph.first + pr_rep * ph.total + (int)((long long)ph.total * b / ph.ncta)) * 16;
+    const int nbox = min(KS, p.nchunk - pr_s * KS);
+    mbar_expect_tx(bar, (uint32_t)nbox * box);
+    for (int j = 0; j < nbox; j++)
+      tma_load_2d(dst + (uint32_t)j * box, &maps.m[pr_ph], (pr_s * KS + j) * kChunkWords, row0, bar);
+    if (++pr_s * KS >= p.nchunk) {
+      pr_s = 0;
+      if (++pr_rep == ph.reps) { pr_rep = 0; pr_ph++; pr_skip(); }
     }
-    pr_n++;
     if (++pr_slot == stages) { pr_slot = 0; pr_phase ^= 1u; }
   };
   if (tid == kCWarps * 32) {
     // the producer thread sets up the barriers itself and starts the stream before the CTA meets
     for (int s = 0; s < stages; s++) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, kCWarps); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    for (int i = 0; i < stages && pr_n < pr_total; i++) produce();
+    pr_skip();
+    for (int i = 0; i < stages && pr_ph < p.nphase; i++) produce();
   }
 
   // ------------------------------------------------------------------ activations (all threads)
@@ -218,15 +217,14 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_left, const __grid_co
       if ((lane & 15) == 0 && u < total) s_T0c[col * p.nchunk + ch] = tsum;
     }
     if (tid < M) s_scale[tid] = __half2float(p.scale[tid]);
-    if (KS > 1)
-      for (int i = tid; i < 8 * 16 * M * 3; i += kGThreads) s_red[i] = 0;
+    for (int i = tid; i < 2 * 8 * 16 * M * 3; i += kGThreads) s_red[i] = 0;
   }
   __syncthreads();
 
   // ------------------------------------------------------------------ producer main loop
   if (warp == kCWarps) {
     if (lane == 0) {
-      while (pr_n < pr_total) {
+      while (pr_ph < p.nphase) {
         // the slot was filled one ring turn ago: wait until every consumer warp has released it
         if (!mbar_wait(empty0 + 8 * pr_slot, pr_phase ^ 1u)) {
           if (p.status) atomicExch(p.status, 2);
@@ -423,72 +421,61 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_left, const __grid_co
   uint32_t phase = 0;
   int T1[NE], T2[NE], T3[NE];
 
-  // ---- leftover groups of this CTA: KS warps per group, each takes every KS-th chunk
-  if (SA > 0) {
+  int nred = 0;   // phases with a shared-memory reduction so far (its two buffers alternate)
+  for (int pi = 0; pi < p.nphase; pi++) {
+    const GemvPhase ph = p.phase[pi];
+    if (b >= ph.ncta) continue;
+    const int KS = kCWarps / ph.gpc;
     const int grp = warp / KS, ks = warp - grp * KS;
-    const bool active = grp < gpc;
-    const int row_first = left_row0 + grp * 16;
-    if (active) fetch_lut(row_first);
-    const uint32_t a_off = (uint32_t)ks * box_left + (uint32_t)grp * kGroupBytes;
-    for (int s = 0; s < SA; s++) {
-      if (!mbar_wait(full0 + 8 * slot, phase)) {
-        if (lane == 0 && p.status) atomicExch(p.status, 3);
-        return;
+    const int SA = (p.nchunk + KS - 1) / KS;
+    const int lo = (int)((long long)ph.total * b / ph.ncta), hi = (int)((long long)ph.total * (b + 1) / ph.ncta);
+    const bool active = grp < hi - lo;   // fewer groups than gpc here, or warps beyond gpc KS
+    const uint32_t a_off = (uint32_t)ks * ((uint32_t)ph.gpc * kGroupBytes) + (uint32_t)grp * kGroupBytes;
+    for (int rp = 0; rp < ph.reps; rp++) {
+      const int row_first = (ph.first + rp * ph.total + lo + grp) * 16;
+      if (active) fetch_lut(row_first);
+      uint32_t b_chunk = (uint32_t)ks * chunk_stride;
+      int ch = ks;
+      for (int s = 0; s < SA; s++, ch += KS, b_chunk += (uint32_t)KS * chunk_stride) {
+        if (!mbar_wait(full0 + 8 * slot, phase)) {
+          if (lane == 0 && p.status) atomicExch(p.status, 3);
+          return;
+        }
+        if (active && ch < p.nchunk) compute_chunk(base + (uint32_t)slot * kStageBytes + a_off, b_chunk);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty0 + 8 * slot);   // this warp is done with the slot
+        if (++slot == stages) { slot = 0; phase ^= 1u; }
       }
-      const int ch = s * KS + ks;
-      if (active && ch < p.nchunk)
-        compute_chunk(base + (uint32_t)slot * kStageBytes + a_off, (uint32_t)ch * chunk_stride);
-      __syncwarp();
-      if (lane == 0) mbar_arrive(empty0 + 8 * slot);   // this warp is done with the slot
-      if (++slot == stages) { slot = 0; phase ^= 1u; }
-    }
-    collect(T1, T2, T3);
-    if (KS == 1) {
-      if (active) emit(row_first, T1, T2, T3);
-    } else {
-      // the KS warps of a group add up in shared memory; the first of them finishes the rows
-      if (active) {
+      collect(T1, T2, T3);
+      if (KS == 1) {
+        if (active) emit(row_first, T1, T2, T3);
+      } else {
+        // the KS warps of a group add up in shared memory; the first of them finishes the rows
+        int* const red = s_red + (nred & 1) * (8 * 16 * M * 3);
+        nred++;
 #pragma unroll
         for (int e = 0; e < NE; e++) {
-          if (etok[e] < M) {
-            int* d = s_red + ((grp * 16 + g + 8 * err[e]) * M + etok[e]) * 3;
+          if (active && etok[e] < M) {
+            int* d = red + ((grp * 16 + g + 8 * err[e]) * M + etok[e]) * 3;
             atomicAdd(d + 0, T1[e]);
             atomicAdd(d + 1, T2[e]);
             atomicAdd(d + 2, T3[e]);
           }
         }
-      }
-      asm volatile("bar.sync 1, %0;" ::"n"(kCWarps * 32) : "memory");   // consumer warps only
-      if (active && ks == 0) {
+        asm volatile("bar.sync 1, %0;" ::"n"(kCWarps * 32) : "memory");   // consumer warps only
+        if (active && ks == 0) {
 #pragma unroll
-        for (int e = 0; e < NE; e++) {
-          if (etok[e] < M) {
-            const int* d = s_red + ((grp * 16 + g + 8 * err[e]) * M + etok[e]) * 3;
-            T1[e] = d[0]; T2[e] = d[1]; T3[e] = d[2];
+          for (int e = 0; e < NE; e++) {
+            if (etok[e] < M) {
+              int* d = red + ((grp * 16 + g + 8 * err[e]) * M + etok[e]) * 3;
+              T1[e] = d[0]; T2[e] = d[1]; T3[e] = d[2];
+              d[0] = 0; d[1] = 0; d[2] = 0;   // ready for the reduction after next
+            }
           }
+          emit(row_first, T1, T2, T3);
         }
-        emit(row_first, T1, T2, T3);
       }
     }
-  }
-
-  // ---- rounds: a 256-row tile per CTA, a group per warp over the whole K
-  for (int r = 0; r < p.R; r++) {
-    const int row_first = (r * G + b) * kTileRows + warp * 16;
-    fetch_lut(row_first);
-    uint32_t b_chunk = 0;
-    for (int c = 0; c < p.nchunk; c++, b_chunk += chunk_stride) {
-      if (!mbar_wait(full0 + 8 * slot, phase)) {
-        if (lane == 0 && p.status) atomicExch(p.status, 3);
-        return;
-      }
-      compute_chunk(base + (uint32_t)slot * kStageBytes + (uint32_t)warp * kGroupBytes, b_chunk);
-      __syncwarp();
-      if (lane == 0) mbar_arrive(empty0 + 8 * slot);
-      if (++slot == stages) { slot = 0; phase ^= 1u; }
-    }
-    collect(T1, T2, T3);
-    emit(row_first, T1, T2, T3);
   }
 }
 

@@ -35,7 +35,8 @@ __device__ int g_pack_bad;  // set by pack_weights_kernel when it meets a code a
 // ---------------------------------------------------------------------------------------------
 // Streaming GEMV: launch plan.
 struct StreamPlan {
-  int nchunk, R, L, gmax, KS, SA, stages, grid;
+  int nchunk, nphase, stages, grid;
+  rcp::GemvPhase phase[rcp::kMaxPhases];
   int off_bar, off_T0c, off_scale, off_red, off_bs;
   size_t smem;
 };
@@ -50,21 +51,66 @@ int tokens_per_pass(int M, int K, int cap) {
   return m;
 }
 
+// Cost model of a phase in clocks: stages x (warps sharing a scheduler) x clocks per warp and
+// chunk on one of the four schedulers, plus a fixed cost per phase (LUT fetch, reduction, barrier).
+long long phase_cost(int gpc, int nchunk) {
+  const int KS = rcp::kCWarps / gpc;
+  const int stages = (nchunk + KS - 1) / KS;
+  const int per_sched = (gpc * KS + 3) / 4;
+  return (long long)stages * per_sched * 504 + 2500;
+}
+
+// Splits `rem` leftover groups (fewer than 16 per CTA) into phases: shares of 8, 4, 2 or 1 groups
+// per CTA keep all warps busy but cost a phase each; one last phase takes whatever is left,
+// ceil(left / CTAs) groups per CTA. Picks the cheapest combination. Returns the number of phases.
+int plan_leftover(int rem, int sms, int nchunk, rcp::GemvPhase* out) {
+  int best_mask = 0;
+  long long best = -1;
+  for (int mask = 0; mask < 16; mask++) {   // bit i: a phase of 8 >> i groups per CTA
+    int left = rem;
+    long long cost = 0;
+    bool ok = true;
+    for (int i = 0; i < 4; i++) {
+      if (!(mask >> i & 1)) continue;
+      const int gpc = 8 >> i;
+      if (left < gpc * sms) { ok = false; break; }
+      left -= gpc * sms;
+      cost += phase_cost(gpc, nchunk);
+    }
+    if (!ok) continue;
+    if (left >= 16 * sms) continue;
+    if (left > 0) cost += phase_cost((left + sms - 1) / sms, nchunk);
+    if (best < 0 || cost < best) { best = cost; best_mask = mask; }
+  }
+  int n = 0, first = 0, left = rem;
+  for (int i = 0; i < 4; i++) {
+    if (!(best_mask >> i & 1)) continue;
+    const int gpc = 8 >> i;
+    out[n++] = rcp::GemvPhase{gpc, first, gpc * sms, sms, 1};
+    first += gpc * sms;
+    left -= gpc * sms;
+  }
+  if (left > 0) {
+    const int ncta = std::min(left, sms);
+    out[n++] = rcp::GemvPhase{(left + ncta - 1) / ncta, first, left, ncta, 1};
+  }
+  return n;
+}
+
 StreamPlan make_plan(int M, int N, int K, int sms) {
   StreamPlan pl;
   pl.grid = sms;
   pl.nchunk = (K / 16 + rcp::kChunkWords - 1) / rcp::kChunkWords;
+  // Phases: first the groups left over when every CTA takes 16 per round, then the rounds.
   const int groups = (N + 15) / 16;
   const int per_round = sms * rcp::kCWarps;
-  pl.R = groups / per_round;
-  pl.L = groups - pl.R * per_round;
-  pl.gmax = (pl.L + sms - 1) / sms;
-  pl.KS = pl.gmax > 0 ? rcp::kCWarps / pl.gmax : 1;
-  pl.KS = std::min(pl.KS, pl.nchunk);
-  pl.SA = pl.gmax > 0 ? (pl.nchunk + pl.KS - 1) / pl.KS : 0;
+  const int R = groups / per_round;
+  pl.nphase = plan_leftover(groups - R * per_round, sms, pl.nchunk, pl.phase);
+  int first = groups - R * per_round;
+  if (R > 0) pl.phase[pl.nphase++] = rcp::GemvPhase{rcp::kCWarps, first, per_round, sms, R};
   const size_t bs_bytes = (size_t)pl.nchunk * rcp::kChunkWords * 16 * M;
   const size_t t0c_bytes = (((size_t)M * pl.nchunk * 4) + 15) / 16 * 16;
-  const size_t red_bytes = (size_t)8 * 16 * M * 3 * 4;
+  const size_t red_bytes = (size_t)2 * 8 * 16 * M * 3 * 4;
   const size_t misc = 128 + t0c_bytes + 64 + red_bytes;
   pl.stages = (int)std::min<size_t>(rcp::kMaxStages, (kSmemMax - 1024 - misc - bs_bytes) / rcp::kStageBytes);
   size_t off = (size_t)pl.stages * rcp::kStageBytes;
@@ -104,15 +150,14 @@ int sm_count() {
 }
 
 template <int MODE, int MTOK>
-int launch_stream_t(const CUtensorMap& map_left, const CUtensorMap& map_round, const rcp::GemvParams& gp,
-                    const StreamPlan& pl, cudaStream_t st) {
+int launch_stream_t(const rcp::GemvMaps& maps, const rcp::GemvParams& gp, const StreamPlan& pl, cudaStream_t st) {
   static bool attr_set = false;
   auto kern = rcp::gemv_stream_kernel<MODE, MTOK>;
   if (!attr_set) {
     RCP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax));
     attr_set = true;
   }
-  kern<<<pl.grid, rcp::kGThreads, pl.smem, st>>>(map_left, map_round, gp);
+  kern<<<pl.grid, rcp::kGThreads, pl.smem, st>>>(maps, gp);
   RCP_CUDA(cudaGetLastError());
   return RCP_OK;
 }
@@ -126,14 +171,14 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   if (!enc) return cuda_fail(cudaErrorNotSupported);
   const StreamPlan pl = make_plan(M, N, K, sm_count());
   if (pl.stages < 2 || pl.smem > kSmemMax) return RCP_ERR_SHAPE;
-  CUtensorMap maps[2];
+  rcp::GemvMaps maps;
   const cuuint64_t gdim[2] = {(cuuint64_t)(K / 16), (cuuint64_t)N};
   const cuuint64_t gstride[1] = {(cuuint64_t)(K / 4)};
   const cuuint32_t estr[2] = {1, 1};
-  const int box_rows[2] = {16 * std::max(1, pl.gmax), rcp::kTileRows};
-  for (int i = 0; i < 2; i++) {
-    const cuuint32_t box[2] = {(cuuint32_t)rcp::kChunkWords, (cuuint32_t)box_rows[i]};
-    const CUresult r = enc(&maps[i], CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t*>(words), gdim, gstride,
+  for (int i = 0; i < rcp::kMaxPhases; i++) {
+    const int gpc = i < pl.nphase ? pl.phase[i].gpc : 1;
+    const cuuint32_t box[2] = {(cuuint32_t)rcp::kChunkWords, (cuuint32_t)(16 * gpc)};
+    const CUresult r = enc(&maps.m[i], CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t*>(words), gdim, gstride,
                            box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue);
@@ -145,17 +190,19 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   gp.y = static_cast<__half*>(y_f16);
   gp.status = static_cast<int32_t*>(workspace);
   gp.M = M; gp.N = N; gp.K = K;
-  gp.nchunk = pl.nchunk; gp.R = pl.R; gp.L = pl.L; gp.gmax = pl.gmax; gp.KS = pl.KS; gp.SA = pl.SA;
+  gp.nchunk = pl.nchunk;
+  gp.nphase = pl.nphase;
+  for (int i = 0; i < rcp::kMaxPhases; i++) gp.phase[i] = i < pl.nphase ? pl.phase[i] : rcp::GemvPhase{1, 0, 0, 1, 0};
   gp.stages = pl.stages;
   gp.off_bar = pl.off_bar; gp.off_T0c = pl.off_T0c; gp.off_scale = pl.off_scale; gp.off_red = pl.off_red;
   gp.off_bs = pl.off_bs;
   if (mode == rcp::kModeHybrid)
-    return M == 1 ? launch_stream_t<rcp::kModeHybrid, 1>(maps[0], maps[1], gp, pl, st)
-                  : launch_stream_t<rcp::kModeHybrid, 2>(maps[0], maps[1], gp, pl, st);
+    return M == 1 ? launch_stream_t<rcp::kModeHybrid, 1>(maps, gp, pl, st)
+                  : launch_stream_t<rcp::kModeHybrid, 2>(maps, gp, pl, st);
   if (mode == rcp::kModeDp4a)
-    return M == 1 ? launch_stream_t<rcp::kModeDp4a, 1>(maps[0], maps[1], gp, pl, st)
-                  : launch_stream_t<rcp::kModeDp4a, 2>(maps[0], maps[1], gp, pl, st);
-  return launch_stream_t<rcp::kModeMma, 0>(maps[0], maps[1], gp, pl, st);
+    return M == 1 ? launch_stream_t<rcp::kModeDp4a, 1>(maps, gp, pl, st)
+                  : launch_stream_t<rcp::kModeDp4a, 2>(maps, gp, pl, st);
+  return launch_stream_t<rcp::kModeMma, 0>(maps, gp, pl, st);
 }
 
 // All M tokens: as many launches as it takes for the expanded activations to fit (`cap` tokens at most each).
