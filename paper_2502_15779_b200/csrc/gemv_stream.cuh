@@ -145,36 +145,48 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   int* const s_red = reinterpret_cast<int*>(gen + p.off_red);           // [2][8 groups][16 rows][M][3]
   uint8_t* const bs = gen + p.off_bs;
 
-  // ------------------------------------------------------------------ producer
-  // The weights do not depend on the preceding kernel: start streaming at once.
-  const int G = gridDim.x, b = blockIdx.x;
-  int pr_ph = 0, pr_rep = 0, pr_s = 0, pr_slot = 0;   // next stage to request: phase, repetition, stage
-  uint32_t pr_phase = 0;
-  auto pr_skip = [&]() {  // moves on to the next phase this CTA takes part in
-    while (pr_ph < p.nphase && b >= p.phase[pr_ph].ncta) pr_ph++;
-  };
-  auto produce = [&]() {  // one stage; the producer thread only
-    const GemvPhase ph = p.phase[pr_ph];
-    const int KS = kCWarps / ph.gpc;
-    const uint32_t bar = full0 + 8 * pr_slot, dst = base + (uint32_t)pr_slot * kStageBytes;
-    const uint32_t box = (uint32_t)ph.gpc * kGroupBytes;
-    const int row0 = (ph.first + pr_rep * ph.total + (int)((long long)ph.total * b / ph.ncta)) * 16;
-    const int nbox = min(KS, p.nchunk - pr_s * KS);
-    mbar_expect_tx(bar, (uint32_t)nbox * box);
-    for (int j = 0; j < nbox; j++)
-      tma_load_2d(dst + (uint32_t)j * box, &maps.m[pr_ph], (pr_s * KS + j) * kChunkWords, row0, bar);
-    if (++pr_s * KS >= p.nchunk) {
-      pr_s = 0;
-      if (++pr_rep == ph.reps) { pr_rep = 0; pr_ph++; pr_skip(); }
-    }
-    if (++pr_slot == stages) { pr_slot = 0; pr_phase ^= 1u; }
-  };
-  if (tid == kCWarps * 32) {
-    // the producer thread sets up the barriers itself and starts the stream before the CTA meets
+  const int b = blockIdx.x;
+  if (tid == 0) {
     for (int s = 0; s < stages; s++) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, kCWarps); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    pr_skip();
-    for (int i = 0; i < stages && pr_ph < p.nphase; i++) produce();
+  }
+  __syncthreads();
+
+  // ------------------------------------------------------------------ producer
+  // One thread requests every stage of this CTA in order. The weights do not depend on the
+  // preceding kernel, so it starts at once, and it never meets the other warps again.
+  if (warp == kCWarps) {
+    if (lane != 0) return;
+    int slot = 0;
+    uint32_t phase = 0;
+    int issued = 0;
+    for (int pi = 0; pi < p.nphase; pi++) {
+      const GemvPhase ph = p.phase[pi];
+      if (b >= ph.ncta) continue;
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.m[pi]) : "memory");
+      const int KS = kCWarps / ph.gpc;
+      const uint32_t box = (uint32_t)ph.gpc * kGroupBytes;
+      const int lo = (int)((long long)ph.total * b / ph.ncta);
+      const int SA = (p.nchunk + KS - 1) / KS;
+      for (int rp = 0; rp < ph.reps; rp++) {
+        const int row0 = (ph.first + rp * ph.total + lo) * 16;
+        for (int s = 0; s < SA; s++) {
+          // a slot filled one ring turn ago must have been released by every consumer warp
+          if (issued >= stages && !mbar_wait(empty0 + 8 * slot, phase ^ 1u)) {
+            if (p.status) atomicExch(p.status, 2);
+            return;
+          }
+          const uint32_t bar = full0 + 8 * slot, dst = base + (uint32_t)slot * kStageBytes;
+          const int nbox = min(KS, p.nchunk - s * KS);
+          mbar_expect_tx(bar, (uint32_t)nbox * box);
+          for (int j = 0; j < nbox; j++)
+            tma_load_2d(dst + (uint32_t)j * box, &maps.m[pi], (s * KS + j) * kChunkWords, row0, bar);
+          issued++;
+          if (++slot == stages) { slot = 0; phase ^= 1u; }
+        }
+      }
+    }
+    return;
   }
 
   // ------------------------------------------------------------------ activations (all threads)
@@ -183,7 +195,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   {
     const int W = p.K / 16;
     const int total = ncol * p.nchunk * 16;
-    for (int u0 = warp * 32; u0 < total; u0 += kGThreads) {
+    for (int u0 = warp * 32; u0 < total; u0 += kCWarps * 32) {
       const int u = u0 + lane;
       int tsum = 0;
       const int pair = u >> 4;
@@ -217,24 +229,9 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
       if ((lane & 15) == 0 && u < total) s_T0c[col * p.nchunk + ch] = tsum;
     }
     if (tid < M) s_scale[tid] = __half2float(p.scale[tid]);
-    for (int i = tid; i < 2 * 8 * 16 * M * 3; i += kGThreads) s_red[i] = 0;
+    for (int i = tid; i < 2 * 8 * 16 * M * 3; i += kCWarps * 32) s_red[i] = 0;
   }
-  __syncthreads();
-
-  // ------------------------------------------------------------------ producer main loop
-  if (warp == kCWarps) {
-    if (lane == 0) {
-      while (pr_ph < p.nphase) {
-        // the slot was filled one ring turn ago: wait until every consumer warp has released it
-        if (!mbar_wait(empty0 + 8 * pr_slot, pr_phase ^ 1u)) {
-          if (p.status) atomicExch(p.status, 2);
-          break;
-        }
-        produce();
-      }
-    }
-    return;
-  }
+  asm volatile("bar.sync 1, %0;" ::"n"(kCWarps * 32) : "memory");   // consumer warps only
 
   // ------------------------------------------------------------------ consumers
   constexpr int NF_M = (MODE == kModeDp4a) ? 0 : (MODE == kModeHybrid ? 2 : 3);  // planes on the MMA
@@ -462,7 +459,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
             atomicAdd(d + 2, T3[e]);
           }
         }
-        asm volatile("bar.sync 1, %0;" ::"n"(kCWarps * 32) : "memory");   // consumer warps only
+        asm volatile("bar.sync 2, %0;" ::"n"(kCWarps * 32) : "memory");   // consumer warps only
         if (active && ks == 0) {
 #pragma unroll
           for (int e = 0; e < NE; e++) {
