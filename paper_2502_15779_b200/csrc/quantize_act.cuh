@@ -12,7 +12,7 @@
 namespace rcp {
 
 template <int G>
-__global__ void __launch_bounds__(1024) quantize_act_kernel(const __half* __restrict__ x, int K, int B,
+__global__ void __launch_bounds__(1024) quantize_act_kernel(const __half* __restrict__ x, int K, int B, int lgB,
                                                             float inv_sqrt_b, float clip_ratio,
                                                             uint8_t* __restrict__ xq,
                                                             __half* __restrict__ scale) {
@@ -73,7 +73,10 @@ __global__ void __launch_bounds__(1024) quantize_act_kernel(const __half* __rest
         }
       }
     }
-    // strides 256 and above: radix-8 passes through shared memory
+    // strides 256 and above: passes of up to three strides (radix 8) through shared memory.
+    // A pass over strides s, 2s, .. (r = 2, 4 or 8 of them combined) works on tuples of r elements
+    // s apart; B is a multiple of r s, so the tuple index maps to an element index with shifts only:
+    // element = ((tuple >> log2 s) << log2(r s)) | (tuple & (s - 1)), plus j s for the j-th member.
     if (B > 256) {
 #pragma unroll
       for (int g = 0; g < G; g++) {
@@ -81,25 +84,21 @@ __global__ void __launch_bounds__(1024) quantize_act_kernel(const __half* __rest
 #pragma unroll
         for (int e = 0; e < 8; e++) sbuf[tid * 8 + e] = v[g][e];
         __syncthreads();
-        for (int s = 256; s < B;) {
-          int stages = 0;
-          while (stages < 3 && (s << stages) < B) stages++;
-          const int r = 1 << stages;
+        for (int ls = 8; ls < lgB;) {
+          const int lr = min(3, lgB - ls);   // log2 of the radix of this pass
           float w[8];
           int idx[8];
 #pragma unroll
           for (int e = 0; e < 8; e++) {
-            const int tau = tid * (8 / r) + e / r;  // tuple index over the whole buffer
-            const int j = e % r;
-            const int per_block = B / r;
-            const int blk = tau / per_block, tb = tau % per_block;
-            idx[e] = blk * B + (tb / s) * (r * s) + j * s + (tb % s);
+            const int tau = (tid << (3 - lr)) + (e >> lr);   // tuple index over the whole buffer
+            const int j = e & ((1 << lr) - 1);
+            idx[e] = ((tau >> ls) << (ls + lr)) + (tau & ((1 << ls) - 1)) + (j << ls);
             w[e] = sbuf[idx[e]];
           }
 #pragma unroll
           for (int t = 0; t < 3; t++) {
-            const int hh = 1 << t;  // tuple-local stride; hh < r whenever t < stages
-            if (t < stages) {
+            const int hh = 1 << t;  // tuple-local stride
+            if (t < lr) {
 #pragma unroll
               for (int e = 0; e < 8; e++) {
                 if ((e & hh) == 0) {
@@ -113,7 +112,7 @@ __global__ void __launch_bounds__(1024) quantize_act_kernel(const __half* __rest
 #pragma unroll
           for (int e = 0; e < 8; e++) sbuf[idx[e]] = w[e];
           __syncthreads();
-          s <<= stages;
+          ls += lr;
         }
 #pragma unroll
         for (int e = 0; e < 8; e++) v[g][e] = sbuf[tid * 8 + e];

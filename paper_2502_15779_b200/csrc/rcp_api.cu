@@ -303,10 +303,12 @@ int rcp_quantize_act(const void* x_f16, int M, int K, int had_block, float clip_
   const int G = (K / 8 + T - 1) / T;
   const size_t smem = B > 256 ? (size_t)T * 8 * sizeof(float) : 0;
   const float inv_sqrt_b = (float)(1.0 / std::sqrt((double)B));
+  int lgB = 0;
+  while ((1 << lgB) < B) lgB++;
   const __half* x = static_cast<const __half*>(x_f16);
   __half* sc = static_cast<__half*>(scale_f16);
 #define RCP_LAUNCH_Q(GG) \
-  rcp::quantize_act_kernel<GG><<<M, T, smem, st>>>(x, K, B, inv_sqrt_b, clip_ratio, xq, sc)
+  rcp::quantize_act_kernel<GG><<<M, T, smem, st>>>(x, K, B, lgB, inv_sqrt_b, clip_ratio, xq, sc)
   if (G <= 1) RCP_LAUNCH_Q(1);
   else if (G <= 2) RCP_LAUNCH_Q(2);
   else if (G <= 4) RCP_LAUNCH_Q(4);
