@@ -98,6 +98,9 @@ size_t rcp_gemv_workspace_bytes(int M, int N, int K);
  *   y[m][n]   = fp16( scale[m] * sum_c lut[n][c] * S_c[m][n] )   (fp32 arithmetic)
  * Constraints: 1 <= M <= 16, N >= 1, K % 64 == 0, 64 <= K <= 65536.
  *   workspace  rcp_gemv_workspace_bytes(M,N,K) bytes, see above; may be NULL if that is 0.
+ *   words, lut_f16 are the constants of the layer: the kernel may start fetching them while earlier
+ *              work on the stream is still running (programmatic dependent launch), so that work
+ *              must not be writing them. xq, scale, y and workspace obey stream order as usual.
  *   S_dbg      NULL in production. Otherwise int32 [M][N][4] receives S_c (runs the SIMPLE variant).
  * Never synchronizes.
  */

@@ -146,6 +146,8 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   uint8_t* const bs = gen + p.off_bs;
 
   const int b = blockIdx.x;
+  // Launched with programmatic stream serialization: the next kernel may start as CTAs retire.
+  asm volatile("griddepcontrol.launch_dependents;");
   if (tid == 0) {
     for (int s = 0; s < stages; s++) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, kCWarps); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -154,7 +156,8 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
 
   // ------------------------------------------------------------------ producer
   // One thread requests every stage of this CTA in order. The weights do not depend on the
-  // preceding kernel, so it starts at once, and it never meets the other warps again.
+  // preceding kernel, so it starts at once (before griddepcontrol.wait), and it never meets the
+  // other warps again.
   if (warp == kCWarps) {
     if (lane != 0) return;
     int slot = 0;
@@ -189,7 +192,11 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     return;
   }
 
-  // ------------------------------------------------------------------ activations (all threads)
+  // The packed weights and the LUT are constants of the layer; everything else (xq, scale, y) may
+  // belong to the kernel before this one: wait for it.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
+  // ------------------------------------------------------------------ activations (consumer warps)
   // One unit = (column, chunk, i, pr, t) = two words. The 16 units of a (column, chunk) are 16
   // consecutive lanes: their sum of q goes to s_T0c.
   {

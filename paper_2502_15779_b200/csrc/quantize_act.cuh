@@ -23,6 +23,10 @@ __global__ void __launch_bounds__(1024) quantize_act_kernel(const __half* __rest
   const int tid = threadIdx.x;
   const int lane = tid & 31;
   const __half* xm = x + (size_t)m * K;
+  // Launched with programmatic stream serialization: let the next kernel get started, then wait
+  // for the kernel before this one, whose output x may be and whose input xq and scale may be.
+  asm volatile("griddepcontrol.launch_dependents;");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   float v[G][8];
 #pragma unroll

@@ -4,6 +4,7 @@
 #include <algorithm>
 #include <cmath>
 #include <mutex>
+#include <utility>
 
 #include "common.cuh"
 #include "gemv_simple.cuh"
@@ -25,6 +26,25 @@ int cuda_fail(cudaError_t e) {
     cudaError_t e__ = (call);                     \
     if (e__ != cudaSuccess) return cuda_fail(e__); \
   } while (0)
+
+// Launches with programmatic stream serialization: the kernel may start while the preceding
+// kernel on the stream is still running and must execute griddepcontrol.wait before it touches
+// anything that kernel may read or write.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_overlapped(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -157,8 +177,7 @@ int launch_stream_t(const rcp::GemvMaps& maps, const rcp::GemvParams& gp, const 
     RCP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax));
     attr_set = true;
   }
-  kern<<<pl.grid, rcp::kGThreads, pl.smem, st>>>(maps, gp);
-  RCP_CUDA(cudaGetLastError());
+  RCP_CUDA(launch_overlapped(kern, dim3(pl.grid), dim3(rcp::kGThreads), pl.smem, st, maps, gp));
   return RCP_OK;
 }
 
@@ -307,15 +326,15 @@ int rcp_quantize_act(const void* x_f16, int M, int K, int had_block, float clip_
   while ((1 << lgB) < B) lgB++;
   const __half* x = static_cast<const __half*>(x_f16);
   __half* sc = static_cast<__half*>(scale_f16);
-#define RCP_LAUNCH_Q(GG) \
-  rcp::quantize_act_kernel<GG><<<M, T, smem, st>>>(x, K, B, lgB, inv_sqrt_b, clip_ratio, xq, sc)
+#define RCP_LAUNCH_Q(GG)                                                                                      \
+  RCP_CUDA(launch_overlapped(rcp::quantize_act_kernel<GG>, dim3(M), dim3(T), smem, st, x, K, B, lgB, inv_sqrt_b, \
+                             clip_ratio, xq, sc))
   if (G <= 1) RCP_LAUNCH_Q(1);
   else if (G <= 2) RCP_LAUNCH_Q(2);
   else if (G <= 4) RCP_LAUNCH_Q(4);
   else if (G <= 8) RCP_LAUNCH_Q(8);
   else return RCP_ERR_SHAPE;
 #undef RCP_LAUNCH_Q
-  RCP_CUDA(cudaGetLastError());
   return RCP_OK;
 }
 
