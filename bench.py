@@ -300,6 +300,8 @@ def main():
     ap.add_argument("--variant", default="auto", choices=["auto", "simple", "dp4a", "mma", "mma_only"])
     ap.add_argument("--no-table", action="store_true", help="skip the per-shape table of the other configs")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle leg")
+    ap.add_argument("--profile", action="store_true",
+                    help="warm-up and timed steps only, then exit (the command line the ncu summaries in profiles/ use)")
     args = ap.parse_args()
     cfg = cfgs.BY_KEY[args.workload]
     M = args.tokens
@@ -349,6 +351,13 @@ def main():
         sampler.start()
     order = [i % copies for i in range(args.steps)]
     ms = time_graph_replays(graphs, order, stream)
+    if args.profile:
+        if rank == 0:
+            print(json.dumps({"profile_run": True, "workload": cfg.key, "M": M, "steps": args.steps,
+                              "ms_per_step": ms / args.steps}), flush=True)
+        if dist is not None:
+            dist.destroy_process_group()
+        return
     # keep the GPU under the same load a little longer so that the clock sampler sees it
     t_end = time.time() + 0.6
     while time.time() < t_end:

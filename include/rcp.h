@@ -75,20 +75,25 @@ int rcp_quantize_act(const void* x_f16, int M, int K, int had_block, float clip_
 
 /*
  * Kernel variants of the LUT GEMV (all compute the same result).
- *   RCP_GEMV_AUTO    library picks.
+ *   RCP_GEMV_AUTO    library picks: DP4A for one token, MMA otherwise.
  *   RCP_GEMV_SIMPLE  one warp per output row, scalar decode; also the variant behind S_dbg.
- *   RCP_GEMV_DP4A    CUDA-core path: masked code planes times int8 activations with dp4a.
- *   RCP_GEMV_MMA     masked code planes as the A operand of int8 mma.sync, weights streamed
- *                    through a TMA/mbarrier shared-memory ring, work split evenly over the SMs;
- *                    for M <= 2 the b0*b1 plane is computed with dp4a beside the tensor cores.
+ *   RCP_GEMV_DP4A    streaming kernel, CUDA cores only: masked code planes times int8 activations
+ *                    with dp4a, two tokens per launch.
+ *   RCP_GEMV_MMA     streaming kernel with the masked code planes as the A operand of int8 mma.sync,
+ *                    up to eight tokens per launch (fewer when K is so long that their expanded
+ *                    activations would not fit in shared memory); for one or two tokens the b0*b1
+ *                    plane is computed with dp4a beside the tensor cores.
  *   RCP_GEMV_MMA_ONLY  as RCP_GEMV_MMA with all three planes on the tensor cores for every M.
+ * The streaming kernel: persistent CTAs, weights through a TMA/mbarrier shared-memory ring, 16-row
+ * groups owned by warps, no exchange between CTAs.
  */
 enum { RCP_GEMV_AUTO = 0, RCP_GEMV_SIMPLE = 1, RCP_GEMV_DP4A = 2, RCP_GEMV_MMA = 3, RCP_GEMV_MMA_ONLY = 4 };
 
 /*
- * Bytes of caller-provided scratch rcp_gemv_w2a4 needs for this shape (0 if none). The scratch
- * must be zero-filled once after allocation; every call leaves it zero-filled again, so one
- * buffer can serve any sequence of calls that do not overlap in time. Returns 0 on bad shapes.
+ * Bytes of caller-provided scratch rcp_gemv_w2a4 needs for this shape (0 on bad shapes). The scratch
+ * holds a status word that a kernel sets if one of its bounded waits ever gives up (0 = fine). It
+ * must be zero-filled once after allocation; every successful call leaves it zero-filled, so one
+ * buffer can serve any sequence of calls.
  */
 size_t rcp_gemv_workspace_bytes(int M, int N, int K);
 
@@ -97,7 +102,7 @@ size_t rcp_gemv_workspace_bytes(int M, int N, int K);
  *   S_c[m][n] = sum over k with code[n][k] == c of q[m][k]       (exact integers)
  *   y[m][n]   = fp16( scale[m] * sum_c lut[n][c] * S_c[m][n] )   (fp32 arithmetic)
  * Constraints: 1 <= M <= 16, N >= 1, K % 64 == 0, 64 <= K <= 65536.
- *   workspace  rcp_gemv_workspace_bytes(M,N,K) bytes, see above; may be NULL if that is 0.
+ *   workspace  rcp_gemv_workspace_bytes(M,N,K) bytes, see above; NULL is accepted (no status word).
  *   words, lut_f16 are the constants of the layer: the kernel may start fetching them while earlier
  *              work on the stream is still running (programmatic dependent launch), so that work
  *              must not be writing them. xq, scale, y and workspace obey stream order as usual.
@@ -154,7 +159,7 @@ int rcp_linear_w2a4_host(const void* x_host_f16, int M, int K, int had_block, fl
  *     overlapping work to rcp_gemv_w2a4 with scratch buffers of its own.
  * Never synchronizes.
  */
-#define RCP_STATIC_SCRATCH_BYTES (4u << 20)
+#define RCP_STATIC_SCRATCH_BYTES 4096u
 int rcp_gemv_w2a4_static(const uint32_t* words, const void* lut_f16, const uint8_t* xq,
                          const void* scale_f16, int M, int N, int K, void* y_f16, void* stream);
 

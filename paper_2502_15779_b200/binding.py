@@ -133,7 +133,7 @@ def rcp_gemv_w2a4(words, lut, xq, scale, y=None, workspace=None, S_dbg=None, var
     return y
 
 
-STATIC_SCRATCH_BYTES = 4 << 20
+STATIC_SCRATCH_BYTES = 4096
 
 
 def rcp_gemv_w2a4_static(words, lut, xq, scale, y=None):

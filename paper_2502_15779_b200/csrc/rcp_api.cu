@@ -352,9 +352,11 @@ int rcp_gemv_w2a4_variant(int variant, const uint32_t* words, const void* lut_f1
       (reinterpret_cast<uintptr_t>(lut_f16) & 7u) || (reinterpret_cast<uintptr_t>(y_f16) & 1u) ||
       (reinterpret_cast<uintptr_t>(scale_f16) & 1u))
     return RCP_ERR_ALIGN;
+  if (reinterpret_cast<uintptr_t>(workspace) & 3u) return RCP_ERR_ALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (S_dbg) variant = RCP_GEMV_SIMPLE;
-  if (variant == RCP_GEMV_AUTO) variant = RCP_GEMV_MMA;
+  // measured on B200: one token runs fastest on the CUDA cores alone, more tokens on the tensor cores
+  if (variant == RCP_GEMV_AUTO) variant = (M == 1) ? RCP_GEMV_DP4A : RCP_GEMV_MMA;
   switch (variant) {
     case RCP_GEMV_SIMPLE: {
       const int block = 256;
