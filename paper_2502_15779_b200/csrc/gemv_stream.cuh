@@ -63,6 +63,7 @@ struct GemvParams {
   int nphase;
   GemvPhase phase[kMaxPhases];
   int stages;           // ring depth
+  int ramp_clk;         // clocks between the first `stages` requests of a CTA
   int off_bar, off_T0c, off_scale, off_red, off_bs;   // shared-memory byte offsets from the aligned base
 };
 
@@ -163,6 +164,10 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     int slot = 0;
     uint32_t phase = 0;
     int issued = 0;
+    // The first ring-full of requests is spaced out by the time HBM needs to serve one stage for the
+    // whole grid: issued all at once, the stages of all CTAs share the bandwidth and even the first
+    // one lands only when nearly all of them have.
+    const long long t_start = clock64();
     for (int pi = 0; pi < p.nphase; pi++) {
       const GemvPhase ph = p.phase[pi];
       if (b >= ph.ncta) continue;
@@ -175,9 +180,14 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
         const int row0 = (ph.first + rp * ph.total + lo) * 16;
         for (int s = 0; s < SA; s++) {
           // a slot filled one ring turn ago must have been released by every consumer warp
-          if (issued >= stages && !mbar_wait(empty0 + 8 * slot, phase ^ 1u)) {
-            if (p.status) atomicExch(p.status, 2);
-            return;
+          if (issued >= stages) {
+            if (!mbar_wait(empty0 + 8 * slot, phase ^ 1u)) {
+              if (p.status) atomicExch(p.status, 2);
+              return;
+            }
+          } else {
+            const long long due = t_start + (long long)issued * p.ramp_clk;
+            while (clock64() < due) { }
           }
           const uint32_t bar = full0 + 8 * slot, dst = base + (uint32_t)slot * kStageBytes;
           const int nbox = min(KS, p.nchunk - s * KS);

@@ -213,6 +213,8 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   gp.nphase = pl.nphase;
   for (int i = 0; i < rcp::kMaxPhases; i++) gp.phase[i] = i < pl.nphase ? pl.phase[i] : rcp::GemvPhase{1, 0, 0, 1, 0};
   gp.stages = pl.stages;
+  // one 32 KB stage per CTA at about 6 TB/s for the whole grid, in SM clocks (about 2 GHz)
+  gp.ramp_clk = (int)((double)rcp::kStageBytes * pl.grid / 6.0e12 * 1.9e9);
   gp.off_bar = pl.off_bar; gp.off_T0c = pl.off_T0c; gp.off_scale = pl.off_scale; gp.off_red = pl.off_red;
   gp.off_bs = pl.off_bs;
   if (mode == rcp::kModeHybrid)
