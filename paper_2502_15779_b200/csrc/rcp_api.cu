@@ -316,27 +316,62 @@ int rcp_quantize_act(const void* x_f16, int M, int K, int had_block, float clip_
   if (!aligned16(x_f16) || !aligned16(xq) || (reinterpret_cast<uintptr_t>(scale_f16) & 1u)) return RCP_ERR_ALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
 
-  // Threads: 8 elements each. The thread count is a multiple of one warp (blocks up to 256 stay
-  // inside a warp) and of B/8 (larger blocks exchange through shared memory inside the CTA).
-  const int unit = B > 256 ? B / 8 : 32;
-  int T = ((K / 8 + unit - 1) / unit) * unit;
-  if (T > 1024) T = (1024 / unit) * unit;
-  const int G = (K / 8 + T - 1) / T;
+  // A cluster of C CTAs per token, 8 elements per thread, about 2048 elements per CTA (8192 at most).
+  rcp::QuantParams qp;
+  qp.x = static_cast<const __half*>(x_f16);
+  qp.xq = xq;
+  qp.scale = static_cast<__half*>(scale_f16);
+  qp.K = K; qp.B = B;
+  qp.lgB = 0;
+  while ((1 << qp.lgB) < B) qp.lgB++;
+  qp.inv_sqrt_b = (float)(1.0 / std::sqrt((double)B));
+  qp.clip_ratio = clip_ratio;
+  int C = 1;
+  while (C < 8 && K / (2 * C) >= 2048) C *= 2;
+  int T;
+  if (B == K && B > 256) {
+    // one rotation block: split it over the cluster, the top strides go through distributed shared memory
+    qp.cross = C;
+    qp.slice = K / C;
+    qp.unit = K; qp.nunits = 1;
+    qp.lg_local = qp.lgB;
+    while ((1 << qp.lg_local) > qp.slice) qp.lg_local--;
+    T = qp.slice / 8;
+  } else {
+    // whole rotation blocks per CTA
+    qp.cross = 1;
+    qp.slice = 0;
+    qp.unit = std::max(B, 64);
+    qp.nunits = K / qp.unit;
+    qp.lg_local = qp.lgB;
+    C = std::min(C, qp.nunits);
+    while (C > 1 && (C & (C - 1))) C--;   // power of two
+    int per = (qp.nunits + C - 1) / C;
+    while ((long long)per * qp.unit > 8192 && C < 8) { C *= 2; per = (qp.nunits + C - 1) / C; }
+    if ((long long)per * qp.unit > 8192) return RCP_ERR_SHAPE;
+    T = (per * qp.unit / 8 + 31) / 32 * 32;
+  }
   const size_t smem = B > 256 ? (size_t)T * 8 * sizeof(float) : 0;
-  const float inv_sqrt_b = (float)(1.0 / std::sqrt((double)B));
-  int lgB = 0;
-  while ((1 << lgB) < B) lgB++;
-  const __half* x = static_cast<const __half*>(x_f16);
-  __half* sc = static_cast<__half*>(scale_f16);
-#define RCP_LAUNCH_Q(GG)                                                                                      \
-  RCP_CUDA(launch_overlapped(rcp::quantize_act_kernel<GG>, dim3(M), dim3(T), smem, st, x, K, B, lgB, inv_sqrt_b, \
-                             clip_ratio, xq, sc))
-  if (G <= 1) RCP_LAUNCH_Q(1);
-  else if (G <= 2) RCP_LAUNCH_Q(2);
-  else if (G <= 4) RCP_LAUNCH_Q(4);
-  else if (G <= 8) RCP_LAUNCH_Q(8);
-  else return RCP_ERR_SHAPE;
-#undef RCP_LAUNCH_Q
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)M * C);
+  cfg.blockDim = dim3(T);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = C;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = C > 1 ? 2 : 1;
+  switch (C) {
+    case 1: RCP_CUDA(cudaLaunchKernelEx(&cfg, rcp::quantize_act_kernel<1>, qp)); break;
+    case 2: RCP_CUDA(cudaLaunchKernelEx(&cfg, rcp::quantize_act_kernel<2>, qp)); break;
+    case 4: RCP_CUDA(cudaLaunchKernelEx(&cfg, rcp::quantize_act_kernel<4>, qp)); break;
+    default: RCP_CUDA(cudaLaunchKernelEx(&cfg, rcp::quantize_act_kernel<8>, qp)); break;
+  }
   return RCP_OK;
 }
 
