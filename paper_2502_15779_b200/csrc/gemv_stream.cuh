@@ -82,10 +82,10 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(20000u)   // the thread may sleep up to 20 us inside one try
       : "memory");
   return ok != 0;
 }
@@ -115,6 +115,9 @@ __device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, 
 }
 __device__ __forceinline__ void dp4a_u8s8(int& d, uint32_t a, uint32_t b) {
   asm("dp4a.u32.s32 %0, %1, %2, %0;" : "+r"(d) : "r"(a), "r"(b));
+}
+__device__ __forceinline__ void dp4a_s8s8(int& d, uint32_t a, uint32_t b) {
+  asm("dp4a.s32.s32 %0, %1, %2, %0;" : "+r"(d) : "r"(a), "r"(b));
 }
 
 // Expanded activations. A chunk is 32 words of a row; consumer lane t reads 16-byte chunk 2t+i of
@@ -256,6 +259,11 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   constexpr int NTD = (NF_D == 0) ? 1 : MTOK;
   int accM[NF_M == 0 ? 1 : NF_M][2][4];
   int accD[NTD][2][NF_D == 0 ? 1 : NF_D][2];
+  // kModeDp4a: position 3 sits in bits 6 and 7 of a byte. One mask keeps both; read as unsigned
+  // bytes they weigh 64 b0 + 128 b1, read as signed bytes 64 b0 - 128 b1, so two dp4a on the same
+  // operand separate the b0 and b1 planes and a mask is saved.
+  constexpr bool kSign3 = (MODE == kModeDp4a);
+  int accP[NTD][2][2];   // [token][row][unsigned, signed]
   auto zero_acc = [&]() {
 #pragma unroll
     for (int f = 0; f < (NF_M == 0 ? 1 : NF_M); f++)
@@ -271,6 +279,10 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
         for (int f = 0; f < (NF_D == 0 ? 1 : NF_D); f++)
 #pragma unroll
           for (int h = 0; h < 2; h++) accD[a][r][f][h] = 0;
+#pragma unroll
+    for (int a = 0; a < NTD; a++)
+#pragma unroll
+      for (int r = 0; r < 2; r++) { accP[a][r][0] = 0; accP[a][r][1] = 0; }
   };
   zero_acc();
 
@@ -301,7 +313,6 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   uint32_t a_chunk[2];
 #pragma unroll
   for (int i = 0; i < 2; i++) a_chunk[i] = (uint32_t)(g * 128 + (((2 * t + i) ^ g) << 4));
-  const uint32_t bs_u32 = smem_u32(bs);
   const uint32_t half_stride = (uint32_t)ncol * 64;
   const uint32_t chunk_stride = 8 * half_stride;   // 2 (i) x 2 (pr) x 2 (half) per chunk
   uint32_t bM_lane, bD_lane[NTD];
@@ -309,30 +320,32 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     int col = g;
     if constexpr (MTOK > 0) col = g % MTOK;
     else if (col >= M) col = M - 1;
-    bM_lane = bs_u32 + (uint32_t)(col * 64 + t * 16);
+    bM_lane = (uint32_t)(col * 64 + t * 16);
   }
 #pragma unroll
-  for (int tok = 0; tok < NTD; tok++) bD_lane[tok] = bs_u32 + (uint32_t)(tok * 64 + t * 16);
+  for (int tok = 0; tok < NTD; tok++) bD_lane[tok] = (uint32_t)(tok * 64 + t * 16);
 
   // 16 rows x 128 bytes of weights at shared address a_grp against the activations of one chunk
   auto compute_chunk = [&](uint32_t a_grp, uint32_t b_chunk) {
+    const uint8_t* const a_ptr = gen + (a_grp - base);
+    const uint8_t* const b_ptr = bs + b_chunk;
 #pragma unroll
     for (int i = 0; i < 2; i++) {
-      const uint4 U = lds128(a_grp + a_chunk[i]);
-      const uint4 V = lds128(a_grp + 8 * 128 + a_chunk[i]);
+      const uint4 U = *reinterpret_cast<const uint4*>(a_ptr + a_chunk[i]);
+      const uint4 V = *reinterpret_cast<const uint4*>(a_ptr + 8 * 128 + a_chunk[i]);
       const uint32_t uw[4] = {U.x, U.y, U.z, U.w};
       const uint32_t vw[4] = {V.x, V.y, V.z, V.w};
 #pragma unroll
       for (int pr = 0; pr < 2; pr++) {
-        const uint32_t b_off = b_chunk + (uint32_t)((i * 2 + pr) * 2) * half_stride;
+        const uint32_t b_off = (uint32_t)((i * 2 + pr) * 2) * half_stride;
         // activation operands of the word pair: [position p][word]
         uint32_t bM[4][2];
         uint32_t bD[NTD][4][2];
         if constexpr (NF_D > 0) {
 #pragma unroll
           for (int tok = 0; tok < NTD; tok++) {
-            const uint4 x = lds128(bD_lane[tok] + b_off);
-            const uint4 y = lds128(bD_lane[tok] + b_off + half_stride);
+            const uint4 x = *reinterpret_cast<const uint4*>(b_ptr + bD_lane[tok] + b_off);
+            const uint4 y = *reinterpret_cast<const uint4*>(b_ptr + bD_lane[tok] + b_off + half_stride);
             bD[tok][0][0] = x.x; bD[tok][0][1] = x.y; bD[tok][1][0] = x.z; bD[tok][1][1] = x.w;
             bD[tok][2][0] = y.x; bD[tok][2][1] = y.y; bD[tok][3][0] = y.z; bD[tok][3][1] = y.w;
           }
@@ -342,8 +355,8 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
 #pragma unroll
             for (int pp = 0; pp < 4; pp++) { bM[pp][0] = bD[0][pp][0]; bM[pp][1] = bD[0][pp][1]; }
           } else {
-            const uint4 x = lds128(bM_lane + b_off);
-            const uint4 y = lds128(bM_lane + b_off + half_stride);
+            const uint4 x = *reinterpret_cast<const uint4*>(b_ptr + bM_lane + b_off);
+            const uint4 y = *reinterpret_cast<const uint4*>(b_ptr + bM_lane + b_off + half_stride);
             bM[0][0] = x.x; bM[0][1] = x.y; bM[1][0] = x.z; bM[1][1] = x.w;
             bM[2][0] = y.x; bM[2][1] = y.y; bM[3][0] = y.z; bM[3][1] = y.w;
           }
@@ -361,9 +374,24 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
 #pragma unroll
           for (int f = 0; f < NF_M; f++)
             mma_u8s8(accM[f][pp >> 1], au0[f], av0[f], au1[f], av1[f], bM[pp][0], bM[pp][1]);
+          if (kSign3 && pp == 3) {
+            const uint32_t k3 = 0xC0C0C0C0u;
+#pragma unroll
+            for (int tok = 0; tok < NTD; tok++) {
+              dp4a_u8s8(accP[tok][0][0], u0 & k3, bD[tok][3][0]);
+              dp4a_s8s8(accP[tok][0][1], u0 & k3, bD[tok][3][0]);
+              dp4a_u8s8(accP[tok][1][0], v0 & k3, bD[tok][3][0]);
+              dp4a_s8s8(accP[tok][1][1], v0 & k3, bD[tok][3][0]);
+              dp4a_u8s8(accP[tok][0][0], u1 & k3, bD[tok][3][1]);
+              dp4a_s8s8(accP[tok][0][1], u1 & k3, bD[tok][3][1]);
+              dp4a_u8s8(accP[tok][1][0], v1 & k3, bD[tok][3][1]);
+              dp4a_s8s8(accP[tok][1][1], v1 & k3, bD[tok][3][1]);
+            }
+          }
 #pragma unroll
           for (int f = 0; f < NF_D; f++) {
             const int fa = 3 - NF_D + f;  // hybrid: plane 2 only; dp4a: planes 0..2
+            if (kSign3 && pp == 3 && fa < 2) continue;
 #pragma unroll
             for (int tok = 0; tok < NTD; tok++) {
               dp4a_u8s8(accD[tok][0][f][pp >> 1], au0[fa], bD[tok][pp][0]);
@@ -399,8 +427,8 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
             a2 = (accM[1][0][r] >> 3) + (accM[1][1][r] >> 7);
             a3 = (accD[tok][rr][0][0] >> 3) + (accD[tok][rr][0][1] >> 7);
           } else {
-            a1 = (accD[tok][rr][0][0] >> 2) + (accD[tok][rr][0][1] >> 6);
-            a2 = (accD[tok][rr][1][0] >> 3) + (accD[tok][rr][1][1] >> 7);
+            a1 = (accD[tok][rr][0][0] >> 2) + (accD[tok][rr][0][1] >> 6) + ((accP[tok][rr][0] + accP[tok][rr][1]) >> 7);
+            a2 = (accD[tok][rr][1][0] >> 3) + (accD[tok][rr][1][1] >> 7) + ((accP[tok][rr][0] - accP[tok][rr][1]) >> 8);
             a3 = (accD[tok][rr][2][0] >> 3) + (accD[tok][rr][2][1] >> 7);
             a1 += __shfl_xor_sync(0xffffffffu, a1, 1); a1 += __shfl_xor_sync(0xffffffffu, a1, 2);
             a2 += __shfl_xor_sync(0xffffffffu, a2, 1); a2 += __shfl_xor_sync(0xffffffffu, a2, 2);
