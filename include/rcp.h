@@ -98,6 +98,17 @@ enum { RCP_GEMV_AUTO = 0, RCP_GEMV_SIMPLE = 1, RCP_GEMV_DP4A = 2, RCP_GEMV_MMA =
 size_t rcp_gemv_workspace_bytes(int M, int N, int K);
 
 /*
+ * Launch plan of the streaming GEMV for a shape, for inspection and tests (host only, touches no
+ * GPU). `sms` is the number of CTAs (one per SM; <= 0: 148). Writes up to `cap` ints to `out`:
+ *   out[0] tokens per launch, out[1] launches, out[2] ring stages, out[3] shared-memory bytes,
+ *   out[4] 128-byte chunks per row, out[5] number of phases, then per phase five ints:
+ *   groups per CTA at most, first group, groups in the phase, CTAs taking part, repetitions.
+ * (A group is 16 consecutive output rows; see the kernel's description.) Returns the number of
+ * ints the full description has, or a negative status.
+ */
+int rcp_gemv_plan(int M, int N, int K, int sms, int* out, int cap);
+
+/*
  * LUT GEMV / skinny GEMM (Section 4.4, Eq. "deqgrid"):
  *   S_c[m][n] = sum over k with code[n][k] == c of q[m][k]       (exact integers)
  *   y[m][n]   = fp16( scale[m] * sum_c lut[n][c] * S_c[m][n] )   (fp32 arithmetic)

@@ -375,6 +375,28 @@ int rcp_quantize_act(const void* x_f16, int M, int K, int had_block, float clip_
   return RCP_OK;
 }
 
+int rcp_gemv_plan(int M, int N, int K, int sms, int* out, int cap) {
+  if (!out && cap > 0) return RCP_ERR_NULL;
+  if (M < 1 || M > rcp::kMaxTokens || N < 1 || !k_ok(K)) return RCP_ERR_SHAPE;
+  if (sms <= 0) sms = 148;
+  const int mp = tokens_per_pass(M, K, 8);
+  const StreamPlan pl = make_plan(mp, N, K, sms);
+  int v[6 + 5 * rcp::kMaxPhases];
+  int n = 0;
+  v[n++] = mp;
+  v[n++] = (M + mp - 1) / mp;
+  v[n++] = pl.stages;
+  v[n++] = (int)pl.smem;
+  v[n++] = pl.nchunk;
+  v[n++] = pl.nphase;
+  for (int i = 0; i < pl.nphase; i++) {
+    v[n++] = pl.phase[i].gpc; v[n++] = pl.phase[i].first; v[n++] = pl.phase[i].total;
+    v[n++] = pl.phase[i].ncta; v[n++] = pl.phase[i].reps;
+  }
+  for (int i = 0; i < n && i < cap; i++) out[i] = v[i];
+  return n;
+}
+
 size_t rcp_gemv_workspace_bytes(int M, int N, int K) {
   if (M < 1 || M > rcp::kMaxTokens || N < 1 || !k_ok(K)) return 0;
   return 16;   // a status word for the kernels' bounded waits; no sums pass through global memory

@@ -1,0 +1,86 @@
+"""Host logic of the streaming GEMV: the launch plan (phases of 16-row groups over the CTAs, ring
+depth, shared-memory budget, tokens per launch). No GPU needed: rcp_gemv_plan only computes."""
+import ctypes as C
+
+import pytest
+
+from paper_2502_15779_b200 import build
+from paper_2502_15779_b200.configs import CONFIGS
+
+
+@pytest.fixture(scope="module")
+def L():
+    lib = C.CDLL(build.build())
+    lib.rcp_gemv_plan.restype = C.c_int
+    lib.rcp_gemv_plan.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int), C.c_int]
+    return lib
+
+
+def plan(L, M, N, K, sms=148):
+    buf = (C.c_int * 64)()
+    n = L.rcp_gemv_plan(M, N, K, sms, buf, 64)
+    assert n >= 6, n
+    v = list(buf[:n])
+    phases = [tuple(v[6 + 5 * i: 11 + 5 * i]) for i in range(v[5])]
+    return dict(tokens=v[0], launches=v[1], stages=v[2], smem=v[3], nchunk=v[4], phases=phases)
+
+
+def check(L, M, N, K, sms=148):
+    p = plan(L, M, N, K, sms)
+    groups = (N + 15) // 16
+    # every group is taken exactly once, in order
+    nxt = 0
+    for gpc, first, total, ncta, reps in p["phases"]:
+        assert 1 <= gpc <= 16 and 1 <= ncta <= sms and reps >= 1 and total >= 1
+        assert first == nxt
+        per_cta_max = -(-total // ncta)
+        assert per_cta_max <= gpc, (gpc, total, ncta)
+        assert (16 // gpc) * gpc <= 16
+        if 16 // gpc > 1:
+            assert gpc <= 8          # the shared-memory reduction holds eight groups
+        # shares of the CTAs tile [0, total) without gaps
+        assert sum((total * (b + 1)) // ncta - (total * b) // ncta for b in range(ncta)) == total
+        nxt += total * reps
+    assert nxt == groups, (nxt, groups)
+    assert len(p["phases"]) <= 6
+    assert p["nchunk"] == -(-K // 512)
+    assert p["stages"] >= 2 and p["smem"] <= 232448
+    assert 1 <= p["tokens"] <= 8 and p["tokens"] * p["launches"] >= M
+    assert p["tokens"] == 1 or p["tokens"] * K <= 128 * 1024   # expanded activations fit
+    return p
+
+
+def test_plans_of_all_benchmark_shapes(L):
+    for cfg in CONFIGS:
+        for layer in cfg.layers:
+            for M in cfg.Ms:
+                check(L, M, layer.N, layer.K)
+
+
+@pytest.mark.parametrize("N", [1, 15, 16, 17, 255, 256, 257, 2367, 2368, 2369, 4096, 37887, 37888, 37889, 100000])
+@pytest.mark.parametrize("K", [64, 512, 4096, 11008, 65536])
+def test_plans_cover_every_group_once(L, N, K):
+    for M in (1, 2, 8, 16):
+        check(L, M, N, K)
+    check(L, 1, N, K, sms=1)
+    check(L, 1, N, K, sms=132)
+
+
+def test_plan_examples(L):
+    # 57344 rows = 3584 groups = one round of 148 x 16 plus 1216 left over: 8 per CTA, then 32 single groups
+    p = check(L, 1, 57344, 8192)
+    assert p["phases"][-1] == (16, 1216, 2368, 148, 1)
+    assert p["phases"][0][0] == 8 and p["phases"][0][2] == 8 * 148
+    assert sum(t * r for _, _, t, _, r in p["phases"][:-1]) == 1216
+    # sixteen tokens go in two launches of eight; long K cuts the tokens per launch further
+    assert (check(L, 16, 4096, 4096)["tokens"], check(L, 16, 4096, 4096)["launches"]) == (8, 2)
+    assert check(L, 8, 8192, 28672)["tokens"] == 4
+    assert check(L, 16, 64, 65536)["tokens"] == 2
+
+
+def test_plan_rejects_bad_shapes(L):
+    buf = (C.c_int * 8)()
+    assert L.rcp_gemv_plan(0, 16, 64, 148, buf, 8) == -2
+    assert L.rcp_gemv_plan(1, 16, 100, 148, buf, 8) == -2
+    assert L.rcp_gemv_plan(17, 16, 64, 148, buf, 8) == -2
+    assert L.rcp_gemv_plan(1, 16, 64, 148, None, 8) == -1
