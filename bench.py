@@ -142,6 +142,21 @@ class LayerSet:
         return sum(L.N * L.K // 4 for L in self.layers)
 
 
+def replica_metrics(ms_local, step_bytes, steps, dist=None, device="cpu"):
+    """Whole-job throughput of independent replicas (one per rank, no data-path collective): the
+    timed region ends when the slowest rank does, so the time is the MAX over ranks and the value
+    is the bytes ALL ranks processed over that time. Returns (ms_per_step, GB/s, world)."""
+    world = 1
+    ms = float(ms_local)
+    if dist is not None:
+        world = dist.get_world_size()
+        t = torch.tensor([ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / steps
+    return ms_per_step, world * step_bytes / (ms_per_step * 1e-3) / 1e9, world
+
+
 def l2_bytes(device):
     return torch.cuda.get_device_properties(device).L2_cache_size
 
@@ -231,49 +246,60 @@ def per_shape_table(cfg, M, device, rcp, stream, variant, reps=3):
 
 
 # ------------------------------------------------------------------------------- CPU oracle leg
-def cpu_oracle_sample(cfg, M, target_seconds=12.0):
-    """Times the oracle (as it stands, one thread) on a bounded sample of the workload: the full
-    activation quantization of every linear of the layer plus the GEMV on the first `rows` output
-    rows of each. Returns (value in the benchmark's unit, description, seconds)."""
-    import oracle
-    layers = list(cfg.layers)
-    # calibration on a tiny slice
-    L0 = layers[0]
-    codes, lut = synth.make_layer(16, L0.K, L0.had_block, cfg.codes, 1)
-    x = synth.make_activations(M, L0.K, 1)
-    t = time.perf_counter()
-    qa = oracle.quantize_act(f16_bits(x), L0.had_block, 1.0)
-    oracle.gemv_w2a4(oracle.pack_weights(codes.numpy()), f16_bits(lut), qa["xq"], qa["scale"])
-    per_code = (time.perf_counter() - t) / (16 * L0.K * M)
-    total_codes = sum(L.N * L.K for L in layers) * M
-    frac = min(1.0, target_seconds / max(1e-9, per_code * total_codes))
-    nbytes, secs, desc = 0, 0.0, []
-    for li, L in enumerate(layers):
-        rows = max(16, int(L.N * frac))
-        rows = min(rows, L.N)
-        seed = cfgs.BASE_SEED + 101 * li
-        codes, lut = synth.make_layer(rows, L.K, L.had_block, cfg.codes, seed)
-        x = synth.make_activations(M, L.K, cfgs.BASE_SEED + 13 * li)
-        xb, cb, lb = f16_bits(x), codes.numpy(), f16_bits(lut)
-        words = oracle.pack_weights(cb)  # offline step, not timed
+def workload_name(cfg, M):
+    return (f"{cfg.key} ({cfg.title}), M={M}: " + ", ".join(f"{L.name} {L.N}x{L.K}" for L in cfg.layers))
+
+
+class OracleSample:
+    """A bounded sample of one step for the CPU oracle (as it stands, one thread): the full activation
+    quantization of every linear of the layer plus the GEMV on the first `rows` output rows of each,
+    `rows` chosen so that one pass takes about `target_seconds`. Inputs are generated once."""
+
+    def __init__(self, cfg, M, target_seconds):
+        import oracle
+        self.oracle = oracle
+        layers = list(cfg.layers)
+        # calibration on a tiny slice
+        L0 = layers[0]
+        codes, lut = synth.make_layer(16, L0.K, L0.had_block, cfg.codes, 1)
+        x = synth.make_activations(M, L0.K, 1)
         t = time.perf_counter()
-        qa = oracle.quantize_act(xb, L.had_block, 1.0)
-        oracle.gemv_w2a4(words, lb, qa["xq"], qa["scale"])
-        secs += time.perf_counter() - t
-        nbytes += cfgs.gemv_bytes(M, rows, L.K) + cfgs.quant_bytes(M, L.K)
-        desc.append(f"{L.name}:{rows}/{L.N} rows")
-    return nbytes / secs / 1e9, "quantize_act + gemv on " + ", ".join(desc), secs
+        qa = oracle.quantize_act(f16_bits(x), L0.had_block, 1.0)
+        oracle.gemv_w2a4(oracle.pack_weights(codes.numpy()), f16_bits(lut), qa["xq"], qa["scale"])
+        per_code = (time.perf_counter() - t) / (16 * L0.K * M)
+        total_codes = sum(L.N * L.K for L in layers) * M
+        frac = min(1.0, target_seconds / max(1e-9, per_code * total_codes))
+        self.items, self.nbytes, desc = [], 0, []
+        for li, L in enumerate(layers):
+            rows = min(L.N, max(16, int(L.N * frac)))
+            seed = cfgs.BASE_SEED + 101 * li
+            codes, lut = synth.make_layer(rows, L.K, L.had_block, cfg.codes, seed)
+            x = synth.make_activations(M, L.K, cfgs.BASE_SEED + 13 * li)
+            words = oracle.pack_weights(codes.numpy())  # offline step, not timed
+            self.items.append((f16_bits(x), L.had_block, words, f16_bits(lut)))
+            self.nbytes += cfgs.gemv_bytes(M, rows, L.K) + cfgs.quant_bytes(M, L.K)
+            desc.append(f"{L.name}:{rows}/{L.N} rows")
+        self.desc = "quantize_act + gemv on " + ", ".join(desc)
+
+    def run(self):
+        """One pass; returns (value in the benchmark's unit, seconds)."""
+        t = time.perf_counter()
+        for xb, had_block, words, lb in self.items:
+            qa = self.oracle.quantize_act(xb, had_block, 1.0)
+            self.oracle.gemv_w2a4(words, lb, qa["xq"], qa["scale"])
+        secs = time.perf_counter() - t
+        return self.nbytes / secs / 1e9, secs
 
 
 def run_reference(args, cfg, M):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    budget = 60.0 / max(1, args.steps + args.warmup)
+    budget = min(args.sample_seconds, 60.0 / max(1, args.steps + args.warmup))
+    sample = OracleSample(cfg, M, budget)
     vals, secs = [], []
-    desc = ""
     for i in range(args.warmup + args.steps):
-        v, desc, s = cpu_oracle_sample(cfg, M, target_seconds=min(12.0, budget))
+        v, s = sample.run()
         if i >= args.warmup:
             vals.append(v)
             secs.append(s)
@@ -281,8 +307,8 @@ def run_reference(args, cfg, M):
     out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
            "warmup": args.warmup, "ms_per_step": 1e3 * statistics.mean(secs), "higher_is_better": True,
            "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
-           "config": {"workload": f"{cfg.key} M={M}", "note": "CPU oracle on a bounded sample of each step"},
-           "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+           "config": {"workload": workload_name(cfg, M), "note": "CPU oracle on a bounded sample of each step"},
+           "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample.desc},
            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0}
     print(json.dumps(out), flush=True)
@@ -300,6 +326,8 @@ def main():
     ap.add_argument("--variant", default="auto", choices=["auto", "simple", "dp4a", "mma", "mma_only"])
     ap.add_argument("--no-table", action="store_true", help="skip the per-shape table of the other configs")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle leg")
+    ap.add_argument("--sample-seconds", type=float, default=12.0,
+                    help="CPU seconds the oracle sample of one step aims for (reference arm and cpu_baseline)")
     ap.add_argument("--profile", action="store_true",
                     help="warm-up and timed steps only, then exit (the command line the ncu summaries in profiles/ use)")
     args = ap.parse_args()
@@ -364,13 +392,8 @@ def main():
         time_graph_replays(graphs, order[:max(1, len(order) // 4)], stream)
     barrier()
     clocks = sampler.stop() if sampler else None
-    if dist is not None:
-        tmax = torch.tensor([ms], device=device)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms = float(tmax.item())
     step_bytes = layer.gemv_bytes() + layer.quant_bytes()
-    ms_per_step = ms / args.steps
-    value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+    ms_per_step, value, _ = replica_metrics(ms, step_bytes, args.steps, dist, device)
     launches = args.steps * 2 * len(layer.layers)
 
     # ---- dominant kernel alone: the GEMV launches of the layer, back to back, cold L2
@@ -419,12 +442,9 @@ def main():
         e1.record(stream)
     e1.synchronize()
     e2e_ms = e0.elapsed_time(e1)
-    if dist is not None:
-        tmax = torch.tensor([e2e_ms], device=device)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tmax.item())
-    e2e = {"value": round(world * step_bytes / (e2e_ms / e2e_steps * 1e-3) / 1e9, 2), "unit": UNIT,
-           "ms_per_step": round(e2e_ms / e2e_steps, 4),
+    e2e_ms_per_step, e2e_value, _ = replica_metrics(e2e_ms, step_bytes, e2e_steps, dist, device)
+    e2e = {"value": round(e2e_value, 2), "unit": UNIT,
+           "ms_per_step": round(e2e_ms_per_step, 4),
            "h2d_bytes_per_step": sum(2 * M * L.K for L in layer.layers),
            "d2h_bytes_per_step": sum(2 * M * L.N for L in layer.layers)}
 
@@ -458,14 +478,15 @@ def main():
 
     cpu = None
     if not args.no_cpu:
-        v, desc, secs = cpu_oracle_sample(cfg, M)
-        cpu = {"value": round(v, 4), "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc, "seconds": round(secs, 2)}
+        sample = OracleSample(cfg, M, args.sample_seconds)
+        v, secs = sample.run()
+        cpu = {"value": round(v, 4), "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample.desc,
+               "seconds": round(secs, 2)}
 
     out = {"metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
            "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True, "scaling": "weak",
            "vs_baseline": None, "dtype": "int32", "data": "synthetic",
-           "config": {"workload": f"{cfg.key} ({cfg.title}), M={M}: " +
-                      ", ".join(f"{L.name} {L.N}x{L.K}" for L in cfg.layers),
+           "config": {"workload": workload_name(cfg, M),
                       "step": "per linear: rcp_quantize_act + rcp_gemv_w2a4, replayed from a CUDA graph",
                       "cold_l2": f"{copies} distinct weight copies in rotation ({copies * wbytes / 1e6:.0f} MB > 2x L2 "
                                  f"of {L2 / 1e6:.0f} MB)",
