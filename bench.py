@@ -181,9 +181,9 @@ def capture(fn, stream):
     return g
 
 
-def per_shape_table(cfg, M, device, rcp, stream, variant, reps=3):
-    """us/call and GB/s for every GEMV shape of a config: graphs of back-to-back launches cycling
-    through distinct weight copies (cold L2), timed with CUDA events."""
+def per_shape_table(cfg, Ms, device, rcp, stream, variant, reps=3):
+    """us/call and GB/s for every GEMV shape of a config and every token count in Ms: graphs of
+    back-to-back launches cycling through distinct weight copies (cold L2), timed with CUDA events."""
     rows = []
     L2 = l2_bytes(device)
     seen = set()
@@ -201,45 +201,48 @@ def per_shape_table(cfg, M, device, rcp, stream, variant, reps=3):
         # distinct copies: rows rotated so contents differ but the value distribution is the same
         words = [torch.roll(base, shifts=c, dims=0).contiguous() if c else base for c in range(copies)]
         luts = [torch.roll(lut, shifts=c, dims=0).contiguous() if c else lut for c in range(copies)]
-        x = synth.make_activations(M, L.K, cfgs.BASE_SEED + 13 * li, device)
-        xq, scale = rcp.rcp_quantize_act(x, L.had_block, 1.0)
-        y = torch.empty(M, L.N, dtype=torch.float16, device=device)
-        ws = rcp.make_workspace(M, L.N, L.K, device)
         launches = copies * max(1, 64 // copies)
+        for M in Ms:
+            x = synth.make_activations(M, L.K, cfgs.BASE_SEED + 13 * li, device)
+            xq, scale = rcp.rcp_quantize_act(x, L.had_block, 1.0)
+            y = torch.empty(M, L.N, dtype=torch.float16, device=device)
+            ws = rcp.make_workspace(M, L.N, L.K, device)
 
-        def body():
-            for i in range(launches):
-                c = i % copies
-                rcp.rcp_gemv_w2a4(words[c], luts[c], xq, scale, y=y, workspace=ws, variant=variant)
+            def body():
+                for i in range(launches):
+                    c = i % copies
+                    rcp.rcp_gemv_w2a4(words[c], luts[c], xq, scale, y=y, workspace=ws, variant=variant)
 
-        with torch.cuda.stream(stream):
-            body()
-        stream.synchronize()
-        g = capture(body, stream)
-        for _ in range(3):
-            g.replay()
-        stream.synchronize()
-        best = min(time_graph_replays([g], [0], stream) for _ in range(reps))
-        us = best * 1e3 / launches
-        nbytes = cfgs.gemv_bytes(M, L.N, L.K)
-        # isolated single launch (includes launch latency)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        iso = []
-        for c in range(min(copies, 5)):
             with torch.cuda.stream(stream):
-                e0.record(stream)
-                rcp.rcp_gemv_w2a4(words[c], luts[c], xq, scale, y=y, workspace=ws, variant=variant)
-                e1.record(stream)
-            e1.synchronize()
-            iso.append(e0.elapsed_time(e1) * 1e3)
-        # the quantizer alone
-        gq = capture(lambda: [rcp.rcp_quantize_act(x, L.had_block, 1.0, xq=xq, scale=scale) for _ in range(32)], stream)
-        gq.replay()
-        stream.synchronize()
-        q_us = min(time_graph_replays([gq], [0], stream) for _ in range(reps)) * 1e3 / 32
-        rows.append({"layer": L.name, "N": L.N, "K": L.K, "M": M, "bytes": nbytes, "us_per_call": round(us, 3),
-                     "gbs": round(nbytes / us / 1e3, 1), "frac_of_8TBs": round(nbytes / us / 1e3 / NOMINAL_HBM_GBS, 4),
-                     "isolated_us": round(min(iso), 2), "quantize_us": round(q_us, 2), "copies": copies})
+                body()
+            stream.synchronize()
+            g = capture(body, stream)
+            for _ in range(3):
+                g.replay()
+            stream.synchronize()
+            best = min(time_graph_replays([g], [0], stream) for _ in range(reps))
+            us = best * 1e3 / launches
+            nbytes = cfgs.gemv_bytes(M, L.N, L.K)
+            # isolated single launch (includes launch latency)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            iso = []
+            for c in range(min(copies, 5)):
+                with torch.cuda.stream(stream):
+                    e0.record(stream)
+                    rcp.rcp_gemv_w2a4(words[c], luts[c], xq, scale, y=y, workspace=ws, variant=variant)
+                    e1.record(stream)
+                e1.synchronize()
+                iso.append(e0.elapsed_time(e1) * 1e3)
+            # the quantizer alone
+            gq = capture(lambda: [rcp.rcp_quantize_act(x, L.had_block, 1.0, xq=xq, scale=scale) for _ in range(32)],
+                         stream)
+            gq.replay()
+            stream.synchronize()
+            q_us = min(time_graph_replays([gq], [0], stream) for _ in range(reps)) * 1e3 / 32
+            rows.append({"layer": L.name, "N": L.N, "K": L.K, "M": M, "bytes": nbytes, "us_per_call": round(us, 3),
+                         "gbs": round(nbytes / us / 1e3, 1),
+                         "frac_of_8TBs": round(nbytes / us / 1e3 / NOMINAL_HBM_GBS, 4),
+                         "isolated_us": round(min(iso), 2), "quantize_us": round(q_us, 2), "copies": copies})
         del words, luts, base
         torch.cuda.empty_cache()
     return rows
@@ -456,11 +459,9 @@ def main():
     shapes = []
     if not args.no_table:
         del graphs, ggraphs
-        wl_rows = per_shape_table(cfg, M, device, rcp, stream, args.variant)
-        shapes.append({"config": cfg.key, "rows": wl_rows})
-        for other in cfgs.CONFIGS:
-            if other.key != cfg.key:
-                shapes.append({"config": other.key, "rows": per_shape_table(other, 1, device, rcp, stream, args.variant)})
+        for c in cfgs.CONFIGS:
+            Ms = tuple(sorted(set(c.Ms) | ({M} if c.key == cfg.key else set())))
+            shapes.append({"config": c.key, "rows": per_shape_table(c, Ms, device, rcp, stream, args.variant)})
 
     # offline step: weight packing throughput (not part of the decode step)
     Lp = cfg.layers[0]
