@@ -75,7 +75,7 @@ int rcp_quantize_act(const void* x_f16, int M, int K, int had_block, float clip_
 
 /*
  * Kernel variants of the LUT GEMV (all compute the same result).
- *   RCP_GEMV_AUTO    library picks: DP4A for one token, MMA otherwise.
+ *   RCP_GEMV_AUTO    library picks (as measured on B200): DP4A for one token, MMA_ONLY otherwise.
  *   RCP_GEMV_SIMPLE  one warp per output row, scalar decode; also the variant behind S_dbg.
  *   RCP_GEMV_DP4A    streaming kernel, CUDA cores only: masked code planes times int8 activations
  *                    with dp4a, two tokens per launch.

@@ -109,7 +109,7 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
 }
 __device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                          uint32_t b1) {
-  asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
@@ -364,7 +364,9 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
         const uint32_t u0 = uw[2 * pr], u1 = uw[2 * pr + 1], v0 = vw[2 * pr], v1 = vw[2 * pr + 1];
         const uint32_t u0s = u0 + u0, u1s = u1 + u1, v0s = v0 + v0, v1s = v1 + v1;  // b0 moved onto b1's bit
 #pragma unroll
-        for (int pp = 0; pp < 4; pp++) {
+        for (int po = 0; po < 4; po++) {
+          // positions in the order 0, 2, 1, 3: consecutive iterations feed different accumulators
+          const int pp = ((po & 1) << 1) | (po >> 1);
           const uint32_t m0 = 0x01010101u << (2 * pp), m1 = m0 << 1;
           // the three planes of the four words: b0, b1, b0*b1 (the last two scaled by 2)
           const uint32_t au0[3] = {u0 & m0, u0 & m1, u0 & u0s & m1};

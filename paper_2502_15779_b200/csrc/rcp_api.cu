@@ -415,7 +415,7 @@ int rcp_gemv_w2a4_variant(int variant, const uint32_t* words, const void* lut_f1
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (S_dbg) variant = RCP_GEMV_SIMPLE;
   // measured on B200: one token runs fastest on the CUDA cores alone, more tokens on the tensor cores
-  if (variant == RCP_GEMV_AUTO) variant = (M == 1) ? RCP_GEMV_DP4A : RCP_GEMV_MMA;
+  if (variant == RCP_GEMV_AUTO) variant = (M == 1) ? RCP_GEMV_DP4A : RCP_GEMV_MMA_ONLY;
   switch (variant) {
     case RCP_GEMV_SIMPLE: {
       const int block = 256;
