@@ -93,6 +93,7 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
   for (uint32_t i = 0; i < kSpinLimit; i++) {
     if (mbar_try(bar, parity)) return true;
+    __nanosleep(64);   // leave the issue slots to the warps that have work
   }
   return false;
 }
