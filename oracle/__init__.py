@@ -181,3 +181,52 @@ def dequant_weights(words, lut_bits):
     Wd = np.empty((N, W * 16), dtype=np.float64)
     lib().orc_dequant_weights(_p(words), _p(lut), C.c_int(N), C.c_int(W * 16), _p(Wd))
     return Wd
+
+
+def gemv_w2a4_grouped(words, lut_bits, xq, scale_bits, G):
+    """Group-wise grid: lut uint16 [N][K/G][4]. Returns dict(S int32 [M][N][K/G][4], y, tol float64 [M][N])."""
+    words = _c(words, np.uint32)
+    lut = _c(lut_bits, np.uint16)
+    xq = _c(xq, np.uint8)
+    scale = _c(scale_bits, np.uint16)
+    N, W = words.shape
+    K = W * 16
+    M = xq.shape[0]
+    assert K % G == 0 and lut.shape == (N, K // G, 4) and xq.shape == (M, K // 2) and scale.shape == (M,)
+    S = np.empty((M, N, K // G, 4), dtype=np.int32)
+    y = np.empty((M, N), dtype=np.float64)
+    tol = np.empty((M, N), dtype=np.float64)
+    rc = lib().orc_gemv_w2a4_grouped(_p(words), _p(lut), _p(xq), _p(scale), C.c_int(M), C.c_int(N), C.c_int(K),
+                                     C.c_int(G), _p(S), _p(y), _p(tol))
+    if rc:
+        raise ValueError(f"orc_gemv_w2a4_grouped failed: {rc}")
+    return dict(S=S, y=y, tol=tol)
+
+
+def gemv_direct_grouped(words, lut_bits, xq, scale_bits, G):
+    """Direct sum over k with a grid per group. Returns dict(y float64 [M][N], acc_int int64 [M][N])."""
+    words = _c(words, np.uint32)
+    lut = _c(lut_bits, np.uint16)
+    xq = _c(xq, np.uint8)
+    scale = _c(scale_bits, np.uint16)
+    N, W = words.shape
+    K = W * 16
+    M = xq.shape[0]
+    assert K % G == 0 and lut.shape == (N, K // G, 4)
+    y = np.empty((M, N), dtype=np.float64)
+    ai = np.empty((M, N), dtype=np.int64)
+    rc = lib().orc_gemv_direct_grouped(_p(words), _p(lut), _p(xq), _p(scale), C.c_int(M), C.c_int(N), C.c_int(K),
+                                       C.c_int(G), _p(y), _p(ai))
+    if rc:
+        raise ValueError(f"orc_gemv_direct_grouped failed: {rc}")
+    return dict(y=y, acc_int=ai)
+
+
+def percode_int_grouped(lut_bits, S):
+    lut = _c(lut_bits, np.uint16)
+    S = _c(S, np.int32)
+    M, N, NG, _ = S.shape
+    assert lut.shape == (N, NG, 4)
+    ai = np.empty((M, N), dtype=np.int64)
+    lib().orc_percode_int_grouped(_p(lut), _p(S), C.c_int(M), C.c_int(N), C.c_int(NG), _p(ai))
+    return ai

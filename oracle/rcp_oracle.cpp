@@ -21,7 +21,9 @@
 // product; library fp16 conversion; hand-computed rounding cases; brute-force 8x8 and
 // 16x32 GEMV; exact integer equality of the per-code-sum form and the direct form;
 // LUT lookup of unpacked codes == dequantized weight matrix; affine/constant LUT special
-// cases reducing to a plain integer GEMV.
+// cases reducing to a plain integer GEMV. Group-wise LUT form: one group == the per-row form;
+// equal grids in every group == the per-row form; brute force; exact integer equality with
+// its direct form; dense matrix product with the group-wise dequantized weights.
 // fp16 output y: the paper prints no worked numeric GEMV example, so y is pinned only by the
 // mathematical identities above, not by a printed value.
 #include <cstdint>
@@ -368,6 +370,93 @@ void orc_dequant_weights(const uint32_t* words, const uint16_t* lut_f16, int N, 
       W[(size_t)n * K + k] = (double)orc_f16_to_f32(lut_f16[(size_t)n * 4 + codes[k]]);
   }
   std::free(codes);
+}
+
+// ---------------------------------------------------------------------------------------
+// Group-wise LUT GEMV. Section 4.4 gives the dequantization grid the shape H x (N*4) with N
+// groups per input channel row, and Appendix A.1 sets C = N*G with group size G (128 in the
+// table of quantization configurations): weight k of row n takes its four levels from group
+// k / G. For token m, row n, group j:
+//   S_c[m][n][j] = sum over k in [jG, (j+1)G) with code[n][k] == c of q[m][k]   (exact integers)
+//   y_ref        = s_m * sum_j sum_c LUT[n][j][c] * S_c[m][n][j]                 (double)
+//   tol          = 2e-3 * ( s_m * sum_j sum_c |LUT[n][j][c]| * |S_c[m][n][j]| ) + 1e-5
+// lut_f16 is [N][K/G][4]. Outputs: S int32 [M][N][K/G][4] (may be NULL), y_ref [M][N], tol
+// [M][N] (may be NULL). Returns 0; -1 bad shape (G must divide K).
+// ---------------------------------------------------------------------------------------
+int orc_gemv_w2a4_grouped(const uint32_t* words, const uint16_t* lut_f16, const uint8_t* xq,
+                          const uint16_t* scale_f16, int M, int N, int K, int G,
+                          int32_t* S, double* y_ref, double* tol) {
+  if (M < 1 || N < 1 || K < 16 || K % 16 || G < 1 || K % G) return -1;
+  const int NG = K / G;
+  uint8_t* codes = (uint8_t*)std::malloc((size_t)K);
+  int8_t* q = (int8_t*)std::malloc((size_t)M * K);
+  orc_unpack_act(xq, (size_t)M * (K / 2), q);
+  for (int n = 0; n < N; n++) {
+    orc_unpack_weights(words + (size_t)n * (K / 16), 1, K, codes);
+    for (int m = 0; m < M; m++) {
+      double s = (double)orc_f16_to_f32(scale_f16[m]);
+      double acc = 0.0, mag = 0.0;
+      for (int j = 0; j < NG; j++) {
+        long long Sc[4] = {0, 0, 0, 0};
+        for (int k = j * G; k < (j + 1) * G; k++) Sc[codes[k]] += (long long)q[(size_t)m * K + k];
+        for (int c = 0; c < 4; c++) {
+          double L = (double)orc_f16_to_f32(lut_f16[((size_t)n * NG + j) * 4 + c]);
+          if (S) S[(((size_t)m * N + n) * NG + j) * 4 + c] = (int32_t)Sc[c];
+          acc += L * (double)Sc[c];
+          mag += std::fabs(L) * std::fabs((double)Sc[c]);
+        }
+      }
+      y_ref[(size_t)m * N + n] = s * acc;
+      if (tol) tol[(size_t)m * N + n] = 2e-3 * (s * mag) + 1e-5;
+    }
+  }
+  std::free(codes);
+  std::free(q);
+  return 0;
+}
+
+// Direct form with a grid per group: y = s_m * sum_k LUT[n][k / G][code[n][k]] * q[m][k], in
+// double, and the same sum as an exact integer with every level scaled by 2^24.
+int orc_gemv_direct_grouped(const uint32_t* words, const uint16_t* lut_f16, const uint8_t* xq,
+                            const uint16_t* scale_f16, int M, int N, int K, int G,
+                            double* y_direct, long long* acc_int) {
+  if (M < 1 || N < 1 || K < 16 || K % 16 || G < 1 || K % G) return -1;
+  const int NG = K / G;
+  uint8_t* codes = (uint8_t*)std::malloc((size_t)K);
+  int8_t* q = (int8_t*)std::malloc((size_t)M * K);
+  orc_unpack_act(xq, (size_t)M * (K / 2), q);
+  for (int n = 0; n < N; n++) {
+    orc_unpack_weights(words + (size_t)n * (K / 16), 1, K, codes);
+    for (int m = 0; m < M; m++) {
+      double acc = 0.0;
+      long long ai = 0;
+      for (int k = 0; k < K; k++) {
+        double L = (double)orc_f16_to_f32(lut_f16[((size_t)n * NG + k / G) * 4 + codes[k]]);
+        int qq = q[(size_t)m * K + k];
+        acc += L * (double)qq;
+        ai += (long long)std::ldexp(L, 24) * (long long)qq;
+      }
+      y_direct[(size_t)m * N + n] = (double)orc_f16_to_f32(scale_f16[m]) * acc;
+      if (acc_int) acc_int[(size_t)m * N + n] = ai;
+    }
+  }
+  std::free(codes);
+  std::free(q);
+  return 0;
+}
+
+// The same exact integer from the per-group per-code sums: sum_j sum_c Lint[n][j][c] * S_c[m][n][j].
+void orc_percode_int_grouped(const uint16_t* lut_f16, const int32_t* S, int M, int N, int NG, long long* acc_int) {
+  for (int m = 0; m < M; m++)
+    for (int n = 0; n < N; n++) {
+      long long ai = 0;
+      for (int j = 0; j < NG; j++)
+        for (int c = 0; c < 4; c++) {
+          long long Li = (long long)std::ldexp((double)orc_f16_to_f32(lut_f16[((size_t)n * NG + j) * 4 + c]), 24);
+          ai += Li * (long long)S[(((size_t)m * N + n) * NG + j) * 4 + c];
+        }
+      acc_int[(size_t)m * N + n] = ai;
+    }
 }
 
 }  // extern "C"

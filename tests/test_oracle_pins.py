@@ -362,3 +362,110 @@ def test_planted_mistakes_are_caught_by_the_brute_force_pin():
     rev = oracle.pack_weights(np.ascontiguousarray(codes.reshape(16, 2, 16)[:, :, ::-1].reshape(16, 32)))
     r_rev = oracle.gemv_w2a4(rev, f16_bits(lut), qa["xq"], qa["scale"])
     assert not np.array_equal(r["S"], r_rev["S"])
+
+
+# ----------------------------------------------------------------------------- GEMV, group-wise grid
+def _problem_grouped(N, K, M, G, seed, kind="uniform", B=1):
+    codes, lut = synth.make_layer_grouped(N, K, G, B, kind, seed)
+    x = synth.make_activations(M, K, seed)
+    qa = oracle.quantize_act(f16_bits(x), B, 1.0)
+    words = oracle.pack_weights(codes.numpy())
+    return codes.numpy(), lut, words, qa
+
+
+def _brute_grouped(codes, lut, q, scale_bits, G):
+    """Pure-Python loops straight from the definition: weight k of row n uses grid k // G of that row."""
+    M, K = q.shape
+    N = codes.shape[0]
+    S = np.zeros((M, N, K // G, 4), dtype=np.int64)
+    y = np.zeros((M, N))
+    lutf = lut.numpy().astype(np.float64)
+    for m in range(M):
+        s = float(scale_bits[m:m + 1].view(np.float16)[0])
+        for n in range(N):
+            acc = 0.0
+            for k in range(K):
+                S[m, n, k // G, int(codes[n, k])] += int(q[m, k])
+                acc += lutf[n, k // G, int(codes[n, k])] * float(q[m, k])
+            y[m, n] = s * acc
+    return S, y
+
+
+@pytest.mark.parametrize("N,K,M,G", [(8, 32, 1, 16), (12, 64, 2, 16), (6, 256, 1, 128), (5, 384, 3, 128)])
+def test_grouped_gemv_brute_force_small(N, K, M, G):
+    codes, lut, words, qa = _problem_grouped(N, K, M, G, seed=N + K)
+    r = oracle.gemv_w2a4_grouped(words, f16_bits(lut), qa["xq"], qa["scale"], G)
+    S, y = _brute_grouped(codes, lut, qa["q"], qa["scale"], G)
+    assert np.array_equal(r["S"], S)
+    assert np.allclose(r["y"], y, rtol=1e-12, atol=1e-300)
+
+
+def test_grouped_gemv_with_one_group_is_the_per_row_gemv():
+    N, K, M = 24, 512, 2
+    codes, lut, words, qa = _problem(N, K, M, seed=31, kind="rotated_laplace", B=128)
+    lb = f16_bits(lut)
+    r = oracle.gemv_w2a4(words, lb, qa["xq"], qa["scale"])
+    rg = oracle.gemv_w2a4_grouped(words, lb.reshape(N, 1, 4), qa["xq"], qa["scale"], K)
+    assert np.array_equal(rg["S"][:, :, 0, :], r["S"])
+    assert np.array_equal(rg["y"], r["y"]) and np.array_equal(rg["tol"], r["tol"])
+
+
+def test_grouped_gemv_with_equal_grids_sums_to_the_per_row_gemv():
+    N, K, M, G = 20, 1024, 2, 128
+    codes, lut, words, qa = _problem(N, K, M, seed=33, kind="uniform", B=64)
+    lb = f16_bits(lut)
+    lbg = np.ascontiguousarray(np.repeat(lb[:, None, :], K // G, axis=1))
+    r = oracle.gemv_w2a4(words, lb, qa["xq"], qa["scale"])
+    rg = oracle.gemv_w2a4_grouped(words, lbg, qa["xq"], qa["scale"], G)
+    assert np.array_equal(rg["S"].sum(axis=2), r["S"])
+    assert np.allclose(rg["y"], r["y"], rtol=1e-12, atol=1e-300)
+    # every group's sums add up to the group's sum of activations
+    tot = qa["q"].astype(np.int64).reshape(M, K // G, G).sum(axis=2)
+    assert np.array_equal(rg["S"].sum(axis=3), np.repeat(tot[:, None, :], N, axis=1))
+    assert np.all(rg["tol"] >= r["tol"] - 1e-18)   # |.| taken per group can only grow the bound
+
+
+@pytest.mark.parametrize("N,K,M,G,B,kind", [(40, 512, 1, 128, 128, "rotated_laplace"), (17, 2048, 2, 128, 2048, "rotated_laplace"),
+                                            (33, 384, 3, 64, 64, "uniform")])
+def test_grouped_direct_form_equals_percode_form_as_exact_integers(N, K, M, G, B, kind):
+    codes, lut, words, qa = _problem_grouped(N, K, M, G, seed=17, kind=kind, B=B)
+    lb = f16_bits(lut)
+    r = oracle.gemv_w2a4_grouped(words, lb, qa["xq"], qa["scale"], G)
+    d = oracle.gemv_direct_grouped(words, lb, qa["xq"], qa["scale"], G)
+    assert np.array_equal(d["acc_int"], oracle.percode_int_grouped(lb, r["S"]))
+    # numpy restatement: dequantize with the grid of each weight's group, then one integer matrix product
+    Li = np.round(np.ldexp(lut.numpy().astype(np.float64), 24)).astype(np.int64)          # [N][K/G][4]
+    Wi = np.take_along_axis(np.repeat(Li, G, axis=1), codes.astype(np.int64)[:, :, None], axis=2)[:, :, 0]
+    assert np.array_equal(d["acc_int"], qa["q"].astype(np.int64) @ Wi.T)
+    assert np.allclose(d["y"], r["y"], rtol=1e-12, atol=1e-300)
+
+
+def test_grouped_gemv_equals_dense_matmul_with_groupwise_dequantized_weights():
+    N, K, M, G = 48, 1024, 3, 128
+    codes, lut, words, qa = _problem_grouped(N, K, M, G, seed=23, kind="rotated_laplace", B=128)
+    r = oracle.gemv_w2a4_grouped(words, f16_bits(lut), qa["xq"], qa["scale"], G)
+    lutf = lut.numpy().astype(np.float64)
+    Wd = np.take_along_axis(np.repeat(lutf, G, axis=1), codes.astype(np.int64)[:, :, None], axis=2)[:, :, 0]
+    # the generator put every weight on one of its own group's levels
+    assert set(np.unique(Wd[3, G:2 * G])) <= set(lutf[3, 1])
+    s = qa["scale"].view(np.float16).astype(np.float64)
+    ref = (qa["q"].astype(np.float64) * s[:, None]) @ Wd.T
+    assert np.allclose(r["y"], ref, rtol=1e-11, atol=1e-15)
+    mag = s[:, None] * (np.abs(lutf)[None] * np.abs(r["S"])).sum(axis=(2, 3))
+    assert np.allclose(r["tol"], 2e-3 * mag + 1e-5, rtol=1e-12)
+
+
+def test_grouped_planted_mistakes_are_caught():
+    # a grid looked up by k % G instead of k // G, or the groups taken in reverse, changes the result
+    N, K, M, G = 8, 64, 1, 16
+    codes, lut, words, qa = _problem_grouped(N, K, M, G, seed=5)
+    r = oracle.gemv_w2a4_grouped(words, f16_bits(lut), qa["xq"], qa["scale"], G)
+    lut_rev = torch.flip(lut, dims=[1]).contiguous()
+    r_rev = oracle.gemv_w2a4_grouped(words, f16_bits(lut_rev), qa["xq"], qa["scale"], G)
+    assert not np.allclose(r["y"], r_rev["y"], rtol=1e-6)
+    perm = np.arange(K).reshape(K // G, G).T.reshape(-1)   # k -> position under the k % G reading
+    r_mod = oracle.gemv_w2a4_grouped(oracle.pack_weights(np.ascontiguousarray(codes[:, perm])), f16_bits(lut),
+                                     np.ascontiguousarray(qa["xq"]), qa["scale"], G)
+    assert not np.array_equal(r["S"], r_mod["S"])
+    with pytest.raises((ValueError, AssertionError)):   # a group size that does not divide K
+        oracle.gemv_w2a4_grouped(words, f16_bits(lut)[:, :3].copy(), qa["xq"], qa["scale"], 24)
