@@ -130,6 +130,30 @@ int rcp_gemv_w2a4_variant(int variant, const uint32_t* words, const void* lut_f1
                           void* y_f16, void* workspace, int32_t* S_dbg, void* stream);
 
 /*
+ * LUT GEMV with one grid per group of weights (Section 4.4: the dequantization grid has shape
+ * H x N*4 for N groups per row; Appendix A.1: C = N*G; the table of quantization configurations
+ * sets the weight group size G = 128). Weight k of row n takes its levels from lut[n][k / group]:
+ *   S_c[m][n][j] = sum over k in [j*group, (j+1)*group) with code[n][k] == c of q[m][k]   (exact)
+ *   y[m][n]      = fp16( scale[m] * sum_j sum_c lut[n][j][c] * S_c[m][n][j] )   (fp32 arithmetic;
+ *                  the order of the fp32 sum over groups is fixed for a shape, so results repeat)
+ *   lut_f16    DEVICE fp16 [N][K/group][4], 8-byte aligned. A constant of the layer like `words`.
+ *   group      a multiple of 16 that divides K. group == 128 runs the streaming kernels; any
+ *              other size runs the plain kernel (correct, not tuned).
+ *   S_dbg      NULL in production. Otherwise int32 [M][N][K/group][4] receives S_c (plain kernel).
+ * Everything else as for rcp_gemv_w2a4 (same workspace, same constraints on M, N, K). Returns
+ * RCP_ERR_SHAPE for a bad group size. Never synchronizes.
+ */
+int rcp_gemv_w2a4_grouped(const uint32_t* words, const void* lut_f16, int group, const uint8_t* xq,
+                          const void* scale_f16, int M, int N, int K, void* y_f16, void* workspace,
+                          int32_t* S_dbg, void* stream);
+
+/* Same, with the kernel variant chosen by the caller: RCP_GEMV_AUTO, RCP_GEMV_SIMPLE,
+ * RCP_GEMV_DP4A or RCP_GEMV_MMA_ONLY (the last two want group == 128, else RCP_ERR_VARIANT). */
+int rcp_gemv_w2a4_grouped_variant(int variant, const uint32_t* words, const void* lut_f16, int group,
+                                  const uint8_t* xq, const void* scale_f16, int M, int N, int K,
+                                  void* y_f16, void* workspace, int32_t* S_dbg, void* stream);
+
+/*
  * One decode linear layer end to end with HOST activations (Section 4.4 data path: rotate and
  * quantize the token, then the LUT GEMV): copies x from host memory, runs rcp_quantize_act and
  * rcp_gemv_w2a4, copies y back. All on `stream`, no synchronization: y_host is valid after the

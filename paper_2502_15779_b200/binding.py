@@ -47,6 +47,10 @@ def lib():
         L.rcp_gemv_w2a4.argtypes = [vp, vp, vp, vp, i, i, i, vp, vp, vp, vp]
         L.rcp_gemv_w2a4_variant.restype = i
         L.rcp_gemv_w2a4_variant.argtypes = [i, vp, vp, vp, vp, i, i, i, vp, vp, vp, vp]
+        L.rcp_gemv_w2a4_grouped.restype = i
+        L.rcp_gemv_w2a4_grouped.argtypes = [vp, vp, i, vp, vp, i, i, i, vp, vp, vp, vp]
+        L.rcp_gemv_w2a4_grouped_variant.restype = i
+        L.rcp_gemv_w2a4_grouped_variant.argtypes = [i, vp, vp, i, vp, vp, i, i, i, vp, vp, vp, vp]
         L.rcp_linear_w2a4_host.restype = i
         L.rcp_linear_w2a4_host.argtypes = [vp, i, i, i, C.c_float, vp, vp, i, vp, vp, vp, vp, vp, vp, vp]
         L.rcp_gemv_w2a4_static.restype = i
@@ -130,6 +134,31 @@ def rcp_gemv_w2a4(words, lut, xq, scale, y=None, workspace=None, S_dbg=None, var
         _check("rcp_gemv_w2a4",
                lib().rcp_gemv_w2a4_variant(v, _ptr(words), _ptr(lut), _ptr(xq), _ptr(scale), M, N, K, _ptr(y),
                                            _ptr(workspace), _ptr(S_dbg), _stream(words)))
+    return y
+
+
+def rcp_gemv_w2a4_grouped(words, lut, xq, scale, group=128, y=None, workspace=None, S_dbg=None, variant="auto"):
+    """Group-wise grid: words int32 [N][K/16], lut fp16 [N][K/group][4], xq uint8 [M][K/2], scale fp16 [M]
+    -> y fp16 [M][N]. S_dbg: int32 [M][N][K/group][4]."""
+    _dev(words, torch.int32, "words")
+    _dev(lut, torch.float16, "lut")
+    _dev(xq, torch.uint8, "xq")
+    _dev(scale, torch.float16, "scale")
+    N, W = words.shape
+    K = W * 16
+    M = xq.shape[0]
+    group = int(group)
+    if group < 1 or K % group or xq.shape != (M, K // 2) or lut.shape != (N, K // group, 4) or scale.shape != (M,):
+        raise ValueError("shape mismatch between words, lut, group, xq and scale")
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.float16, device=words.device)
+    if workspace is None and rcp_gemv_workspace_bytes(M, N, K) > 0:
+        workspace = make_workspace(M, N, K, words.device)
+    v = VARIANTS[variant] if isinstance(variant, str) else int(variant)
+    with torch.cuda.device(words.device):
+        _check("rcp_gemv_w2a4_grouped",
+               lib().rcp_gemv_w2a4_grouped_variant(v, _ptr(words), _ptr(lut), group, _ptr(xq), _ptr(scale), M, N, K,
+                                                   _ptr(y), _ptr(workspace), _ptr(S_dbg), _stream(words)))
     return y
 
 

@@ -22,4 +22,15 @@ __device__ __forceinline__ __half lut_finish(float s, uint2 lut4, int S0, int S1
   return __float2half_rn(s * acc);
 }
 
+// One group's term of the group-wise form: L0*S0 + L1*S1 + L2*S2 + L3*S3 in fp32.
+__device__ __forceinline__ float lut_dot(uint2 lut4, int S0, int S1, int S2, int S3) {
+  const float2 l01 = __half22float2(*reinterpret_cast<const __half2*>(&lut4.x));
+  const float2 l23 = __half22float2(*reinterpret_cast<const __half2*>(&lut4.y));
+  float acc = l01.x * (float)S0;
+  acc = fmaf(l01.y, (float)S1, acc);
+  acc = fmaf(l23.x, (float)S2, acc);
+  acc = fmaf(l23.y, (float)S3, acc);
+  return acc;
+}
+
 }  // namespace rcp

@@ -24,6 +24,13 @@
 //   K and finishes its rows from its registers. The groups left over go in phases of 8, 4, 2, 1
 //   groups per CTA, so that all sixteen warps stay busy; there the sums of the KS warps of a group
 //   meet in shared memory (integer atomics) and one of them finishes the rows.
+// Group-wise grid (GRP; the grid of Section 4.4 has one four-entry row per group of 128 weights):
+//   the integer sums live for one group only. A 128-byte chunk of a row is four groups. On the
+//   CUDA-core path lane t of a quad already holds exactly group t of the chunk, so after every
+//   chunk each lane turns its own sums into one fp32 term with its group's grid. On the tensor
+//   cores an MMA adds up the k of all four lanes of a quad, so there the quad reads one group at a
+//   time (8 bytes per lane instead of 16, rows dealt to the lanes so that the reads stay free of
+//   bank conflicts) and finishes it after twelve MMAs. The fp32 terms add up in a fixed order.
 // Nothing is exchanged between CTAs, no scratch memory is needed, and the result does not depend
 // on timing. The int4 activations are expanded once per CTA into the B-operand byte layout in
 // shared memory.
@@ -59,6 +66,7 @@ struct GemvParams {
   __half* y;
   int32_t* status;      // optional: receives a code when a bounded wait gives up
   int M, N, K;
+  int ngrp;             // group-wise grid: groups of 128 weights per row (K / 128), lut is [N][ngrp]; else 0
   int nchunk;           // 128-byte chunks per row, ceil(K / 512)
   int nphase;
   GemvPhase phase[kMaxPhases];
@@ -132,7 +140,8 @@ __device__ __forceinline__ void dp4a_s8s8(int& d, uint32_t a, uint32_t b) {
 // MODE  kModeMma: all three planes on the tensor cores; kModeHybrid: b0 and b1 planes on the tensor
 //       cores, the b0*b1 plane on dp4a; kModeDp4a: everything on dp4a (CUDA cores only)
 // MTOK  tokens, fixed at compile time for the dp4a modes (1 or 2); 0 = run-time, up to 8 (kModeMma)
-template <int MODE, int MTOK>
+// GRP   one grid per group of 128 weights instead of one per row (kModeHybrid has no such form)
+template <int MODE, int MTOK, bool GRP>
 __global__ void __launch_bounds__(kGThreads, 1)
 gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -145,9 +154,13 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   const int ncol = M;
   const int stages = p.stages;
   const uint32_t full0 = base + p.off_bar, empty0 = full0 + 8 * kMaxStages;
-  int* const s_T0c = reinterpret_cast<int*>(gen + p.off_T0c);           // [M][nchunk]: sum of q per chunk
+  static_assert(!(GRP && MODE == kModeHybrid), "no group-wise hybrid mode");
+  constexpr bool kRelabel = GRP && MODE == kModeMma;   // a quad shares a group: lane t takes words 8j+2t, 8j+2t+1
+  int* const s_T0c = reinterpret_cast<int*>(gen + p.off_T0c);           // [M][nchunk]: sum of q per chunk; GRP: [M][4 nchunk] per group
   float* const s_scale = reinterpret_cast<float*>(gen + p.off_scale);   // [16]
   int* const s_red = reinterpret_cast<int*>(gen + p.off_red);           // [2][8 groups][16 rows][M][3]
+  float* const s_redf = reinterpret_cast<float*>(gen + p.off_red);      // GRP: [2][16 warps][16 rows][M]
+  const int ng4 = 4 * p.nchunk;
   uint8_t* const bs = gen + p.off_bs;
 
   const int b = blockIdx.x;
@@ -222,8 +235,8 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
       const int pair = u >> 4;
       const int col = pair / p.nchunk, ch = pair - col * p.nchunk;
       if (u < total) {
-        const int tt = u & 3, pr = (u >> 2) & 1, i = (u >> 3) & 1;
-        const int wx = ch * kChunkWords + 8 * tt + 4 * i + 2 * pr;   // word index in the row
+        const int lo = u & 3, hi = (u >> 2) & 3;   // lo: 16-byte slot t of the column block; hi: 2 i + pr, or the group
+        const int wx = ch * kChunkWords + (kRelabel ? 8 * hi + 2 * lo : 8 * lo + 2 * hi);   // word index in the row
         uint4 x = make_uint4(0, 0, 0, 0);
         if (wx < W) x = __ldg(reinterpret_cast<const uint4*>(p.xq + (size_t)col * (p.K / 2)) + (wx >> 1));
         uint32_t q[4][2];
@@ -241,16 +254,27 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
             q[pp][w] = v;
           }
         }
-        uint8_t* dst = bs + ((size_t)((((ch * 2 + i) * 2 + pr) * 2) * ncol + col)) * 64 + tt * 16;
+        uint8_t* dst = bs + ((size_t)(((ch * 4 + hi) * 2) * ncol + col)) * 64 + lo * 16;
         *reinterpret_cast<uint4*>(dst) = make_uint4(q[0][0], q[0][1], q[1][0], q[1][1]);
         *reinterpret_cast<uint4*>(dst + (size_t)ncol * 64) = make_uint4(q[2][0], q[2][1], q[3][0], q[3][1]);
       }
+      if constexpr (!GRP) {
 #pragma unroll
-      for (int d = 8; d > 0; d >>= 1) tsum += __shfl_xor_sync(0xffffffffu, tsum, d);
-      if ((lane & 15) == 0 && u < total) s_T0c[col * p.nchunk + ch] = tsum;
+        for (int d = 8; d > 0; d >>= 1) tsum += __shfl_xor_sync(0xffffffffu, tsum, d);
+        if ((lane & 15) == 0 && u < total) s_T0c[col * p.nchunk + ch] = tsum;
+      } else if constexpr (kRelabel) {   // the group is bits 2,3 of the unit: add up over bits 0,1
+        tsum += __shfl_xor_sync(0xffffffffu, tsum, 1);
+        tsum += __shfl_xor_sync(0xffffffffu, tsum, 2);
+        if ((u & 3) == 0 && u < total) s_T0c[col * ng4 + ch * 4 + ((u >> 2) & 3)] = tsum;
+      } else {                           // the group is bits 0,1 of the unit: add up over bits 2,3
+        tsum += __shfl_xor_sync(0xffffffffu, tsum, 4);
+        tsum += __shfl_xor_sync(0xffffffffu, tsum, 8);
+        if ((u & 12) == 0 && u < total) s_T0c[col * ng4 + ch * 4 + (u & 3)] = tsum;
+      }
     }
     if (tid < M) s_scale[tid] = __half2float(p.scale[tid]);
-    for (int i = tid; i < 2 * 8 * 16 * M * 3; i += kCWarps * 32) s_red[i] = 0;
+    if constexpr (!GRP)
+      for (int i = tid; i < 2 * 8 * 16 * M * 3; i += kCWarps * 32) s_red[i] = 0;
   }
   asm volatile("bar.sync 1, %0;" ::"n"(kCWarps * 32) : "memory");   // consumer warps only
 
@@ -300,7 +324,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     T0v[e] = 0;
   }
   // T0 of every token: sum over the chunks, by the whole warp; a lane keeps the tokens it emits
-  for (int m = 0; m < M; m++) {
+  for (int m = 0; m < (GRP ? 0 : M); m++) {
     int a = 0;
     for (int c = lane; c < p.nchunk; c += 32) a += s_T0c[m * p.nchunk + c];
 #pragma unroll
@@ -408,6 +432,131 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     }
   };
 
+  // ---- group-wise grid
+  // Tensor-core mode: MMA row g of the fragment is row grow of the 16 (rows 0,2,4,6 in the first
+  // half-warp, 1,3,5,7 in the second: the 8-byte reads of a half-warp then hit all 32 banks once).
+  const int grow = kRelabel ? (2 * (g & 3) + (g >> 2)) : g;
+  float yacc[NE];
+#pragma unroll
+  for (int e = 0; e < NE; e++) yacc[e] = 0.f;
+  int tokc[2];   // tensor-core mode: this lane's two token columns, clamped to the tokens that exist
+  tokc[0] = min(2 * t, M - 1);
+  tokc[1] = min(2 * t + 1, M - 1);
+  // grids of the groups of chunk ch for this lane's rows: [group of the chunk][row]; the CUDA-core
+  // path needs group t only
+  constexpr int NLG = kRelabel ? 4 : 1;
+  auto fetch_lut_grp = [&](int row_first, int ch, uint2 (&dst)[NLG][2]) {
+#pragma unroll
+    for (int j = 0; j < NLG; j++) {
+      const int gi = ch * 4 + (kRelabel ? j : t);
+#pragma unroll
+      for (int rr = 0; rr < 2; rr++) {
+        const int row = row_first + grow + 8 * rr;
+        dst[j][rr] = (row < p.N && gi < p.ngrp) ? __ldg(p.lut + (size_t)row * p.ngrp + gi) : make_uint2(0, 0);
+      }
+    }
+  };
+  // CUDA-core mode, after a chunk: this lane's sums are those of group t of the chunk
+  auto flush_grp_dp4a = [&](int ch, const uint2 (&lg)[NLG][2]) {
+    if constexpr (GRP && MODE == kModeDp4a) {
+      const int gi = ch * 4 + t;
+#pragma unroll
+      for (int tok = 0; tok < NTD; tok++)
+#pragma unroll
+        for (int rr = 0; rr < 2; rr++) {
+          const int a1 = (accD[tok][rr][0][0] >> 2) + (accD[tok][rr][0][1] >> 6) + ((accP[tok][rr][0] + accP[tok][rr][1]) >> 7);
+          const int a2 = (accD[tok][rr][1][0] >> 3) + (accD[tok][rr][1][1] >> 7) + ((accP[tok][rr][0] - accP[tok][rr][1]) >> 8);
+          const int a3 = (accD[tok][rr][2][0] >> 3) + (accD[tok][rr][2][1] >> 7);
+          const int T0 = s_T0c[tok * ng4 + gi];
+          const int S1 = a1 - a3, S2 = a2 - a3;
+          yacc[tok * 2 + rr] += lut_dot(lg[0][rr], T0 - S1 - S2 - a3, S1, S2, a3);
+        }
+      zero_acc();
+    }
+  };
+  // Tensor-core mode: one chunk = four groups, each read by the whole quad, finished after its
+  // twelve MMAs.
+  auto compute_chunk_grp_mma = [&](uint32_t a_grp, uint32_t b_chunk, int ch, const uint2 (&lg)[NLG][2]) {
+    if constexpr (kRelabel) {
+      const uint8_t* const a_row = gen + (a_grp - base) + grow * 128 + ((t & 1) << 3);
+#pragma unroll
+      for (int j = 0; j < 4; j++) {
+        const uint32_t a_sw = (uint32_t)(((2 * j + (t >> 1)) ^ (grow & 7)) << 4);
+        const uint2 U = *reinterpret_cast<const uint2*>(a_row + a_sw);
+        const uint2 V = *reinterpret_cast<const uint2*>(a_row + 8 * 128 + a_sw);
+        const uint8_t* const b_ptr = bs + b_chunk + (uint32_t)(j * 2) * half_stride + bM_lane;
+        const uint4 x = *reinterpret_cast<const uint4*>(b_ptr);
+        const uint4 y = *reinterpret_cast<const uint4*>(b_ptr + half_stride);
+        const uint32_t bM[4][2] = {{x.x, x.y}, {x.z, x.w}, {y.x, y.y}, {y.z, y.w}};
+        const uint32_t u0 = U.x, u1 = U.y, v0 = V.x, v1 = V.y;
+        const uint32_t u0s = u0 + u0, u1s = u1 + u1, v0s = v0 + v0, v1s = v1 + v1;
+#pragma unroll
+        for (int po = 0; po < 4; po++) {
+          const int pp = ((po & 1) << 1) | (po >> 1);
+          const uint32_t m0 = 0x01010101u << (2 * pp), m1 = m0 << 1;
+          const uint32_t au0[3] = {u0 & m0, u0 & m1, u0 & u0s & m1};
+          const uint32_t au1[3] = {u1 & m0, u1 & m1, u1 & u1s & m1};
+          const uint32_t av0[3] = {v0 & m0, v0 & m1, v0 & v0s & m1};
+          const uint32_t av1[3] = {v1 & m0, v1 & m1, v1 & v1s & m1};
+#pragma unroll
+          for (int f = 0; f < 3; f++)
+            mma_u8s8(accM[f][pp >> 1], au0[f], av0[f], au1[f], av1[f], bM[pp][0], bM[pp][1]);
+        }
+        const int gi = ch * 4 + j;
+#pragma unroll
+        for (int r = 0; r < 4; r++) {
+          const int a1 = (accM[0][0][r] >> 2) + (accM[0][1][r] >> 6);
+          const int a2 = (accM[1][0][r] >> 3) + (accM[1][1][r] >> 7);
+          const int a3 = (accM[2][0][r] >> 3) + (accM[2][1][r] >> 7);
+          const int T0 = s_T0c[tokc[r & 1] * ng4 + gi];
+          const int S1 = a1 - a3, S2 = a2 - a3;
+          yacc[r] += lut_dot(lg[j][r >> 1], T0 - S1 - S2 - a3, S1, S2, a3);
+        }
+        zero_acc();
+      }
+    }
+  };
+  // end of a row group: the fp32 sums of this warp's chunks, for the entries this lane emits
+  auto emit_grp = [&](int row_first, bool active, int KS, int grp, int ks, int& nred) {
+    if constexpr (GRP) {
+      if constexpr (MODE == kModeDp4a) {   // the four lanes of a quad hold four groups each: add them up
+#pragma unroll
+        for (int e = 0; e < NE; e++) {
+          yacc[e] += __shfl_xor_sync(0xffffffffu, yacc[e], 1);
+          yacc[e] += __shfl_xor_sync(0xffffffffu, yacc[e], 2);
+        }
+      }
+      if (KS > 1) {
+        // every warp of the group leaves its sums in its own slot; the first adds them up in order
+        float* const red = s_redf + (nred & 1) * (kCWarps * 16 * M);
+        nred++;
+#pragma unroll
+        for (int e = 0; e < NE; e++)
+          if (active && etok[e] < M) red[(warp * 16 + g + 8 * err[e]) * M + etok[e]] = yacc[e];
+        asm volatile("bar.sync 2, %0;" ::"n"(kCWarps * 32) : "memory");   // consumer warps only
+        if (active && ks == 0) {
+#pragma unroll
+          for (int e = 0; e < NE; e++) {
+            if (etok[e] < M) {
+              float a = 0.f;
+              for (int k = 0; k < KS; k++) a += red[((grp * KS + k) * 16 + g + 8 * err[e]) * M + etok[e]];
+              yacc[e] = a;
+            }
+          }
+        }
+      }
+      if (active && ks == 0) {
+#pragma unroll
+        for (int e = 0; e < NE; e++) {
+          const int row = row_first + grow + 8 * err[e];
+          if (etok[e] < M && row < p.N) p.y[(size_t)etok[e] * p.N + row] = __float2half_rn(s_scale[etok[e]] * yacc[e]);
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < NE; e++) yacc[e] = 0.f;
+    }
+  };
+
   // this lane's entries as T1, T2, T3 from the accumulators (and clears them)
   auto collect = [&](int (&T1)[NE], int (&T2)[NE], int (&T3)[NE]) {
     if constexpr (MODE == kModeMma) {
@@ -478,9 +627,37 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     const uint32_t a_off = (uint32_t)ks * ((uint32_t)ph.gpc * kGroupBytes) + (uint32_t)grp * kGroupBytes;
     for (int rp = 0; rp < ph.reps; rp++) {
       const int row_first = (ph.first + rp * ph.total + lo + grp) * 16;
-      if (active) fetch_lut(row_first);
       uint32_t b_chunk = (uint32_t)ks * chunk_stride;
       int ch = ks;
+      if constexpr (GRP) {
+        // the grids of a chunk are fetched one chunk ahead
+        uint2 lg_cur[NLG][2], lg_nxt[NLG][2];
+        fetch_lut_grp(active ? row_first : p.N, ch, lg_nxt);
+        for (int s = 0; s < SA; s++, ch += KS, b_chunk += (uint32_t)KS * chunk_stride) {
+#pragma unroll
+          for (int j = 0; j < NLG; j++) { lg_cur[j][0] = lg_nxt[j][0]; lg_cur[j][1] = lg_nxt[j][1]; }
+          if (s + 1 < SA) fetch_lut_grp(active ? row_first : p.N, ch + KS, lg_nxt);
+          if (!mbar_wait(full0 + 8 * slot, phase)) {
+            if (lane == 0 && p.status) atomicExch(p.status, 3);
+            return;
+          }
+          if (active && ch < p.nchunk) {
+            const uint32_t a_grp = base + (uint32_t)slot * kStageBytes + a_off;
+            if constexpr (kRelabel) {
+              compute_chunk_grp_mma(a_grp, b_chunk, ch, lg_cur);
+            } else {
+              compute_chunk(a_grp, b_chunk);
+              flush_grp_dp4a(ch, lg_cur);
+            }
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(empty0 + 8 * slot);   // this warp is done with the slot
+          if (++slot == stages) { slot = 0; phase ^= 1u; }
+        }
+        emit_grp(row_first, active, KS, grp, ks, nred);
+        continue;
+      }
+      if (active) fetch_lut(row_first);
       for (int s = 0; s < SA; s++, ch += KS, b_chunk += (uint32_t)KS * chunk_stride) {
         if (!mbar_wait(full0 + 8 * slot, phase)) {
           if (lane == 0 && p.status) atomicExch(p.status, 3);

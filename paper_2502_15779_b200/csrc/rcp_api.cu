@@ -117,7 +117,7 @@ int plan_leftover(int rem, int sms, int nchunk, rcp::GemvPhase* out) {
   return n;
 }
 
-StreamPlan make_plan(int M, int N, int K, int sms) {
+StreamPlan make_plan(int M, int N, int K, int sms, bool grouped = false) {
   StreamPlan pl;
   pl.grid = sms;
   pl.nchunk = (K / 16 + rcp::kChunkWords - 1) / rcp::kChunkWords;
@@ -129,8 +129,10 @@ StreamPlan make_plan(int M, int N, int K, int sms) {
   int first = groups - R * per_round;
   if (R > 0) pl.phase[pl.nphase++] = rcp::GemvPhase{rcp::kCWarps, first, per_round, sms, R};
   const size_t bs_bytes = (size_t)pl.nchunk * rcp::kChunkWords * 16 * M;
-  const size_t t0c_bytes = (((size_t)M * pl.nchunk * 4) + 15) / 16 * 16;
-  const size_t red_bytes = (size_t)2 * 8 * 16 * M * 3 * 4;
+  // sums of q per chunk (per group of 128: four per chunk); reduction buffers: integer sums of 8
+  // row groups x 3 planes, or (group-wise grid) one fp32 term per warp
+  const size_t t0c_bytes = (((size_t)M * pl.nchunk * 4 * (grouped ? 4 : 1)) + 15) / 16 * 16;
+  const size_t red_bytes = grouped ? (size_t)2 * rcp::kCWarps * 16 * M * 4 : (size_t)2 * 8 * 16 * M * 3 * 4;
   const size_t misc = 128 + t0c_bytes + 64 + red_bytes;
   pl.stages = (int)std::min<size_t>(rcp::kMaxStages, (kSmemMax - 1024 - misc - bs_bytes) / rcp::kStageBytes);
   size_t off = (size_t)pl.stages * rcp::kStageBytes;
@@ -169,10 +171,10 @@ int sm_count() {
   return n;
 }
 
-template <int MODE, int MTOK>
+template <int MODE, int MTOK, bool GRP = false>
 int launch_stream_t(const rcp::GemvMaps& maps, const rcp::GemvParams& gp, const StreamPlan& pl, cudaStream_t st) {
   static bool attr_set = false;
-  auto kern = rcp::gemv_stream_kernel<MODE, MTOK>;
+  auto kern = rcp::gemv_stream_kernel<MODE, MTOK, GRP>;
   if (!attr_set) {
     RCP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax));
     attr_set = true;
@@ -181,14 +183,16 @@ int launch_stream_t(const rcp::GemvMaps& maps, const rcp::GemvParams& gp, const 
   return RCP_OK;
 }
 
-// One launch: M tokens (their expanded activations fit in shared memory).
+// One launch: M tokens (their expanded activations fit in shared memory). grouped: lut_f16 is
+// [N][K/128][4], one grid per group of 128 weights.
 int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const uint8_t* xq, const void* scale_f16,
-                  int M, int N, int K, void* y_f16, void* workspace, cudaStream_t st) {
+                  int M, int N, int K, void* y_f16, void* workspace, cudaStream_t st, bool grouped = false) {
   if (mode != rcp::kModeMma && M > 2) return RCP_ERR_VARIANT;
   if (M > 8) return RCP_ERR_VARIANT;
+  if (grouped && (mode == rcp::kModeHybrid || K % 128)) return RCP_ERR_VARIANT;
   EncodeTiledFn enc = encode_tiled_fn();
   if (!enc) return cuda_fail(cudaErrorNotSupported);
-  const StreamPlan pl = make_plan(M, N, K, sm_count());
+  const StreamPlan pl = make_plan(M, N, K, sm_count(), grouped);
   if (pl.stages < 2 || pl.smem > kSmemMax) return RCP_ERR_SHAPE;
   rcp::GemvMaps maps;
   const cuuint64_t gdim[2] = {(cuuint64_t)(K / 16), (cuuint64_t)N};
@@ -209,6 +213,7 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   gp.y = static_cast<__half*>(y_f16);
   gp.status = static_cast<int32_t*>(workspace);
   gp.M = M; gp.N = N; gp.K = K;
+  gp.ngrp = grouped ? K / 128 : 0;
   gp.nchunk = pl.nchunk;
   gp.nphase = pl.nphase;
   for (int i = 0; i < rcp::kMaxPhases; i++) gp.phase[i] = i < pl.nphase ? pl.phase[i] : rcp::GemvPhase{1, 0, 0, 1, 0};
@@ -217,6 +222,12 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   gp.ramp_clk = (int)((double)rcp::kStageBytes * pl.grid / 6.0e12 * 1.9e9);
   gp.off_bar = pl.off_bar; gp.off_T0c = pl.off_T0c; gp.off_scale = pl.off_scale; gp.off_red = pl.off_red;
   gp.off_bs = pl.off_bs;
+  if (grouped) {
+    if (mode == rcp::kModeDp4a)
+      return M == 1 ? launch_stream_t<rcp::kModeDp4a, 1, true>(maps, gp, pl, st)
+                    : launch_stream_t<rcp::kModeDp4a, 2, true>(maps, gp, pl, st);
+    return launch_stream_t<rcp::kModeMma, 0, true>(maps, gp, pl, st);
+  }
   if (mode == rcp::kModeHybrid)
     return M == 1 ? launch_stream_t<rcp::kModeHybrid, 1>(maps, gp, pl, st)
                   : launch_stream_t<rcp::kModeHybrid, 2>(maps, gp, pl, st);
@@ -228,7 +239,8 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
 
 // All M tokens: as many launches as it takes for the expanded activations to fit (`cap` tokens at most each).
 int launch_stream_passes(int mode, int cap, const uint32_t* words, const void* lut_f16, const uint8_t* xq,
-                         const void* scale_f16, int M, int N, int K, void* y_f16, void* workspace, cudaStream_t st) {
+                         const void* scale_f16, int M, int N, int K, void* y_f16, void* workspace, cudaStream_t st,
+                         bool grouped = false) {
   const int mp = tokens_per_pass(M, K, cap);
   for (int m0 = 0; m0 < M; m0 += mp) {
     const int mm = std::min(mp, M - m0);
@@ -236,7 +248,7 @@ int launch_stream_passes(int mode, int cap, const uint32_t* words, const void* l
     if (md == rcp::kModeHybrid && mm > 2) md = rcp::kModeMma;
     const int rc = launch_stream(md, words, lut_f16, xq + (size_t)m0 * (K / 2),
                                  static_cast<const __half*>(scale_f16) + m0, mm, N, K,
-                                 static_cast<__half*>(y_f16) + (size_t)m0 * N, workspace, st);
+                                 static_cast<__half*>(y_f16) + (size_t)m0 * N, workspace, st, grouped);
     if (rc != RCP_OK) return rc;
   }
   return RCP_OK;
@@ -445,6 +457,50 @@ int rcp_gemv_w2a4(const uint32_t* words, const void* lut_f16, const uint8_t* xq,
                   int M, int N, int K, void* y_f16, void* workspace, int32_t* S_dbg, void* stream) {
   return rcp_gemv_w2a4_variant(RCP_GEMV_AUTO, words, lut_f16, xq, scale_f16, M, N, K, y_f16, workspace,
                                S_dbg, stream);
+}
+
+int rcp_gemv_w2a4_grouped_variant(int variant, const uint32_t* words, const void* lut_f16, int group,
+                                  const uint8_t* xq, const void* scale_f16, int M, int N, int K, void* y_f16,
+                                  void* workspace, int32_t* S_dbg, void* stream) {
+  if (!words || !lut_f16 || !xq || !scale_f16 || !y_f16) return RCP_ERR_NULL;
+  if (M < 1 || M > rcp::kMaxTokens || N < 1 || !k_ok(K)) return RCP_ERR_SHAPE;
+  if (group < 16 || group % 16 || K % group) return RCP_ERR_SHAPE;
+  if (!aligned16(words) || !aligned16(xq) || !aligned16(S_dbg) ||
+      (reinterpret_cast<uintptr_t>(lut_f16) & 7u) || (reinterpret_cast<uintptr_t>(y_f16) & 1u) ||
+      (reinterpret_cast<uintptr_t>(scale_f16) & 1u))
+    return RCP_ERR_ALIGN;
+  if (reinterpret_cast<uintptr_t>(workspace) & 3u) return RCP_ERR_ALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // the streaming kernels are built for the paper's group size; other sizes take the plain kernel
+  if (S_dbg || (variant == RCP_GEMV_AUTO && group != 128)) variant = RCP_GEMV_SIMPLE;
+  if (variant == RCP_GEMV_AUTO) variant = (M <= 2) ? RCP_GEMV_DP4A : RCP_GEMV_MMA_ONLY;
+  switch (variant) {
+    case RCP_GEMV_SIMPLE: {
+      const int block = 256;
+      const int grid = (N + (block / 32) - 1) / (block / 32);
+      rcp::gemv_simple_grouped_kernel<<<grid, block, 0, st>>>(words, static_cast<const uint2*>(lut_f16), xq,
+                                                              static_cast<const __half*>(scale_f16), M, N, K, group,
+                                                              static_cast<__half*>(y_f16), S_dbg);
+      break;
+    }
+    case RCP_GEMV_MMA_ONLY:
+      if (group != 128) return RCP_ERR_VARIANT;
+      return launch_stream_passes(rcp::kModeMma, 8, words, lut_f16, xq, scale_f16, M, N, K, y_f16, workspace, st, true);
+    case RCP_GEMV_DP4A:
+      if (group != 128) return RCP_ERR_VARIANT;
+      return launch_stream_passes(rcp::kModeDp4a, 2, words, lut_f16, xq, scale_f16, M, N, K, y_f16, workspace, st, true);
+    default:
+      return RCP_ERR_VARIANT;
+  }
+  RCP_CUDA(cudaGetLastError());
+  return RCP_OK;
+}
+
+int rcp_gemv_w2a4_grouped(const uint32_t* words, const void* lut_f16, int group, const uint8_t* xq,
+                          const void* scale_f16, int M, int N, int K, void* y_f16, void* workspace, int32_t* S_dbg,
+                          void* stream) {
+  return rcp_gemv_w2a4_grouped_variant(RCP_GEMV_AUTO, words, lut_f16, group, xq, scale_f16, M, N, K, y_f16, workspace,
+                                       S_dbg, stream);
 }
 
 int rcp_gemv_w2a4_static(const uint32_t* words, const void* lut_f16, const uint8_t* xq, const void* scale_f16,
