@@ -32,6 +32,7 @@ from paper_2502_15779_b200 import synth  # noqa: E402
 METRIC = "w2a4_decode_layer_hbm_gbs"
 UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0
+GROUP = 128   # weight group size of the group-wise grid
 
 
 def measured_peaks():
@@ -201,6 +202,10 @@ def per_shape_table(cfg, Ms, device, rcp, stream, variant, reps=3):
         # distinct copies: rows rotated so contents differ but the value distribution is the same
         words = [torch.roll(base, shifts=c, dims=0).contiguous() if c else base for c in range(copies)]
         luts = [torch.roll(lut, shifts=c, dims=0).contiguous() if c else lut for c in range(copies)]
+        # the same shape with one grid per group of 128 weights (the paper's weight group size)
+        lut_g = synth.make_lut_grouped(L.N, L.K // GROUP, seed, device) if L.K % GROUP == 0 else None
+        luts_g = [torch.roll(lut_g, shifts=c, dims=0).contiguous() if c else lut_g for c in range(copies)] \
+            if lut_g is not None else None
         launches = copies * max(1, 64 // copies)
         for M in Ms:
             x = synth.make_activations(M, L.K, cfgs.BASE_SEED + 13 * li, device)
@@ -239,11 +244,31 @@ def per_shape_table(cfg, Ms, device, rcp, stream, variant, reps=3):
             gq.replay()
             stream.synchronize()
             q_us = min(time_graph_replays([gq], [0], stream) for _ in range(reps)) * 1e3 / 32
-            rows.append({"layer": L.name, "N": L.N, "K": L.K, "M": M, "bytes": nbytes, "us_per_call": round(us, 3),
-                         "gbs": round(nbytes / us / 1e3, 1),
-                         "frac_of_8TBs": round(nbytes / us / 1e3 / NOMINAL_HBM_GBS, 4),
-                         "isolated_us": round(min(iso), 2), "quantize_us": round(q_us, 2), "copies": copies})
-        del words, luts, base
+            row = {"layer": L.name, "N": L.N, "K": L.K, "M": M, "bytes": nbytes, "us_per_call": round(us, 3),
+                   "gbs": round(nbytes / us / 1e3, 1),
+                   "frac_of_8TBs": round(nbytes / us / 1e3 / NOMINAL_HBM_GBS, 4),
+                   "isolated_us": round(min(iso), 2), "quantize_us": round(q_us, 2), "copies": copies}
+            if luts_g is not None:
+                def body_g():
+                    for i in range(launches):
+                        c = i % copies
+                        rcp.rcp_gemv_w2a4_grouped(words[c], luts_g[c], xq, scale, group=GROUP, y=y, workspace=ws,
+                                                  variant=variant if variant in ("auto", "simple", "dp4a", "mma_only")
+                                                  else "auto")
+                with torch.cuda.stream(stream):
+                    body_g()
+                stream.synchronize()
+                gg = capture(body_g, stream)
+                for _ in range(3):
+                    gg.replay()
+                stream.synchronize()
+                us_g = min(time_graph_replays([gg], [0], stream) for _ in range(reps)) * 1e3 / launches
+                nbytes_g = cfgs.gemv_grouped_bytes(M, L.N, L.K, GROUP)
+                row.update({"grouped_bytes": nbytes_g, "grouped_us_per_call": round(us_g, 3),
+                            "grouped_gbs": round(nbytes_g / us_g / 1e3, 1)})
+                del gg
+            rows.append(row)
+        del words, luts, base, luts_g, lut_g
         torch.cuda.empty_cache()
     return rows
 

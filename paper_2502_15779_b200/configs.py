@@ -59,6 +59,11 @@ def gemv_bytes(M: int, N: int, K: int) -> int:
     return N * K // 4 + 8 * N + M * K // 2 + 2 * M * N
 
 
+def gemv_grouped_bytes(M: int, N: int, K: int, G: int) -> int:
+    """The same with one four-entry fp16 grid per group of G weights instead of one per row."""
+    return N * K // 4 + 8 * N * (K // G) + M * K // 2 + 2 * M * N
+
+
 def quant_bytes(M: int, K: int) -> int:
     """Algorithmic bytes of one activation-quantization call: fp16 in, nibbles + fp16 scale out."""
     return 2 * M * K + M * K // 2 + 2 * M

@@ -122,6 +122,17 @@ __device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, 
       : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+// the same with a zero accumulator coming in
+__device__ __forceinline__ void mma_u8s8_zero(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                              uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+      : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(0));
+}
+// int -> float for |x| < 2^22 with one integer add and one float add (no conversion unit)
+__device__ __forceinline__ float small_int_to_float(int x) {
+  return __int_as_float(x + 0x4B400000) - 12582912.0f;   // 1.5 * 2^23 + x, exactly
+}
 __device__ __forceinline__ void dp4a_u8s8(int& d, uint32_t a, uint32_t b) {
   asm("dp4a.u32.s32 %0, %1, %2, %0;" : "+r"(d) : "r"(a), "r"(b));
 }
@@ -160,7 +171,10 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   float* const s_scale = reinterpret_cast<float*>(gen + p.off_scale);   // [16]
   int* const s_red = reinterpret_cast<int*>(gen + p.off_red);           // [2][8 groups][16 rows][M][3]
   float* const s_redf = reinterpret_cast<float*>(gen + p.off_red);      // GRP: [2][16 warps][16 rows][M]
+  // tensor-core GRP: the same area as floats [4 nchunk][Mp], 8 x the sum of q of a group, tokens padded to even
+  float* const s_T0f = reinterpret_cast<float*>(gen + p.off_T0c);
   const int ng4 = 4 * p.nchunk;
+  const int Mp = (M + 1) & ~1;
   uint8_t* const bs = gen + p.off_bs;
 
   const int b = blockIdx.x;
@@ -265,7 +279,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
       } else if constexpr (kRelabel) {   // the group is bits 2,3 of the unit: add up over bits 0,1
         tsum += __shfl_xor_sync(0xffffffffu, tsum, 1);
         tsum += __shfl_xor_sync(0xffffffffu, tsum, 2);
-        if ((u & 3) == 0 && u < total) s_T0c[col * ng4 + ch * 4 + ((u >> 2) & 3)] = tsum;
+        if ((u & 3) == 0 && u < total) s_T0f[(ch * 4 + ((u >> 2) & 3)) * Mp + col] = (float)(8 * tsum);
       } else {                           // the group is bits 0,1 of the unit: add up over bits 2,3
         tsum += __shfl_xor_sync(0xffffffffu, tsum, 4);
         tsum += __shfl_xor_sync(0xffffffffu, tsum, 8);
@@ -439,21 +453,16 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   float yacc[NE];
 #pragma unroll
   for (int e = 0; e < NE; e++) yacc[e] = 0.f;
-  int tokc[2];   // tensor-core mode: this lane's two token columns, clamped to the tokens that exist
-  tokc[0] = min(2 * t, M - 1);
-  tokc[1] = min(2 * t + 1, M - 1);
+  const int tok2 = min(2 * t, Mp - 2);   // tensor-core mode: this lane's pair of token columns, kept inside the table
   // grids of the groups of chunk ch for this lane's rows: [group of the chunk][row]; the CUDA-core
   // path needs group t only
-  constexpr int NLG = kRelabel ? 4 : 1;
+  constexpr int NLG = 1;
   auto fetch_lut_grp = [&](int row_first, int ch, uint2 (&dst)[NLG][2]) {
+    const int gi = ch * 4 + t;   // lane t of a quad fetches group t; the tensor-core path passes it round the quad
 #pragma unroll
-    for (int j = 0; j < NLG; j++) {
-      const int gi = ch * 4 + (kRelabel ? j : t);
-#pragma unroll
-      for (int rr = 0; rr < 2; rr++) {
-        const int row = row_first + grow + 8 * rr;
-        dst[j][rr] = (row < p.N && gi < p.ngrp) ? __ldg(p.lut + (size_t)row * p.ngrp + gi) : make_uint2(0, 0);
-      }
+    for (int rr = 0; rr < 2; rr++) {
+      const int row = row_first + grow + 8 * rr;
+      dst[0][rr] = (row < p.N && gi < p.ngrp) ? __ldg(p.lut + (size_t)row * p.ngrp + gi) : make_uint2(0, 0);
     }
   };
   // CUDA-core mode, after a chunk: this lane's sums are those of group t of the chunk
@@ -499,20 +508,33 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
           const uint32_t av0[3] = {v0 & m0, v0 & m1, v0 & v0s & m1};
           const uint32_t av1[3] = {v1 & m0, v1 & m1, v1 & v1s & m1};
 #pragma unroll
-          for (int f = 0; f < 3; f++)
-            mma_u8s8(accM[f][pp >> 1], au0[f], av0[f], au1[f], av1[f], bM[pp][0], bM[pp][1]);
+          for (int f = 0; f < 3; f++) {
+            if (po < 2) mma_u8s8_zero(accM[f][pp >> 1], au0[f], av0[f], au1[f], av1[f], bM[pp][0], bM[pp][1]);
+            else mma_u8s8(accM[f][pp >> 1], au0[f], av0[f], au1[f], av1[f], bM[pp][0], bM[pp][1]);
+          }
         }
+        // The accumulators hold 4 T1 and 64 T1 (positions {0,1} and {2,3}), 8 and 128 times T2 and T3.
+        // Everything below works on 8 x the sums, in fp32 (small integers: exact); the 1/8 goes into
+        // the final scale.
         const int gi = ch * 4 + j;
+        const float2 t0 = *reinterpret_cast<const float2*>(s_T0f + gi * Mp + tok2);
+        uint2 lgj[2];
+#pragma unroll
+        for (int rr = 0; rr < 2; rr++) {
+          lgj[rr].x = __shfl_sync(0xffffffffu, lg[0][rr].x, (lane & ~3) | j);
+          lgj[rr].y = __shfl_sync(0xffffffffu, lg[0][rr].y, (lane & ~3) | j);
+        }
 #pragma unroll
         for (int r = 0; r < 4; r++) {
-          const int a1 = (accM[0][0][r] >> 2) + (accM[0][1][r] >> 6);
-          const int a2 = (accM[1][0][r] >> 3) + (accM[1][1][r] >> 7);
-          const int a3 = (accM[2][0][r] >> 3) + (accM[2][1][r] >> 7);
-          const int T0 = s_T0c[tokc[r & 1] * ng4 + gi];
-          const int S1 = a1 - a3, S2 = a2 - a3;
-          yacc[r] += lut_dot(lg[j][r >> 1], T0 - S1 - S2 - a3, S1, S2, a3);
+          const float F1 = small_int_to_float(accM[0][0][r] + (accM[0][1][r] >> 4));   // 4 T1
+          const float F2 = small_int_to_float(accM[1][0][r] + (accM[1][1][r] >> 4));   // 8 T2
+          const float F3 = small_int_to_float(accM[2][0][r] + (accM[2][1][r] >> 4));   // 8 T3 = 8 S3
+          const float S1 = fmaf(2.f, F1, -F3), S2 = F2 - F3;
+          const float S0 = (((r & 1) ? t0.y : t0.x) - S1) - (S2 + F3);
+          const float2 l01 = __half22float2(*reinterpret_cast<const __half2*>(&lgj[r >> 1].x));
+          const float2 l23 = __half22float2(*reinterpret_cast<const __half2*>(&lgj[r >> 1].y));
+          yacc[r] = fmaf(l01.x, S0, fmaf(l01.y, S1, fmaf(l23.x, S2, fmaf(l23.y, F3, yacc[r]))));
         }
-        zero_acc();
       }
     }
   };
@@ -549,7 +571,8 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
 #pragma unroll
         for (int e = 0; e < NE; e++) {
           const int row = row_first + grow + 8 * err[e];
-          if (etok[e] < M && row < p.N) p.y[(size_t)etok[e] * p.N + row] = __float2half_rn(s_scale[etok[e]] * yacc[e]);
+          if (etok[e] < M && row < p.N)
+            p.y[(size_t)etok[e] * p.N + row] = __float2half_rn(s_scale[etok[e]] * (kRelabel ? 0.125f * yacc[e] : yacc[e]));
         }
       }
 #pragma unroll

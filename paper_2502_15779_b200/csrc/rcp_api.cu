@@ -131,7 +131,7 @@ StreamPlan make_plan(int M, int N, int K, int sms, bool grouped = false) {
   const size_t bs_bytes = (size_t)pl.nchunk * rcp::kChunkWords * 16 * M;
   // sums of q per chunk (per group of 128: four per chunk); reduction buffers: integer sums of 8
   // row groups x 3 planes, or (group-wise grid) one fp32 term per warp
-  const size_t t0c_bytes = (((size_t)M * pl.nchunk * 4 * (grouped ? 4 : 1)) + 15) / 16 * 16;
+  const size_t t0c_bytes = grouped ? (size_t)(M + 1) * pl.nchunk * 16 : (((size_t)M * pl.nchunk * 4) + 15) / 16 * 16;
   const size_t red_bytes = grouped ? (size_t)2 * rcp::kCWarps * 16 * M * 4 : (size_t)2 * 8 * 16 * M * 3 * 4;
   const size_t misc = 128 + t0c_bytes + 64 + red_bytes;
   pl.stages = (int)std::min<size_t>(rcp::kMaxStages, (kSmemMax - 1024 - misc - bs_bytes) / rcp::kStageBytes);
