@@ -154,9 +154,26 @@ int rcp_gemv_w2a4_grouped_variant(int variant, const uint32_t* words, const void
                                   void* y_f16, void* workspace, int32_t* S_dbg, void* stream);
 
 /*
+ * One decode linear layer from fp16 activations: rcp_quantize_act followed by rcp_gemv_w2a4 (group
+ * == 0) or rcp_gemv_w2a4_grouped (group > 0), same arguments, same results bit for bit in xq and
+ * scale and within the GEMV's tolerance in y (Section 4.4 data path; Appendix A.7 counts the
+ * separate activation quantizer as the overhead this removes).
+ *   For one or two tokens, a rotation block of at most 512 (or one block spanning a token of at
+ *   most 8192 elements) and group in {0, 128}, a single kernel does both: every CTA rotates and
+ *   quantizes the token itself while its first weight requests are in flight. xq and scale_f16
+ *   are then optional outputs (NULL: not written). Every other case runs the two kernels one after
+ *   the other and needs xq [M][K/2] and scale_f16 [M] as staging: RCP_ERR_NULL without them.
+ *   x_f16 obeys stream order; words and lut_f16 are layer constants (see rcp_gemv_w2a4).
+ * Never synchronizes.
+ */
+int rcp_linear_w2a4(const void* x_f16, int M, int K, int had_block, float clip_ratio,
+                    const uint32_t* words, const void* lut_f16, int group, int N, void* y_f16,
+                    uint8_t* xq, void* scale_f16, void* workspace, void* stream);
+
+/*
  * One decode linear layer end to end with HOST activations (Section 4.4 data path: rotate and
- * quantize the token, then the LUT GEMV): copies x from host memory, runs rcp_quantize_act and
- * rcp_gemv_w2a4, copies y back. All on `stream`, no synchronization: y_host is valid after the
+ * quantize the token, then the LUT GEMV): copies x from host memory, runs rcp_linear_w2a4
+ * (per-row grid), copies y back. All on `stream`, no synchronization: y_host is valid after the
  * caller synchronizes the stream. Pinned host memory makes the copies asynchronous.
  *   x_host_f16  HOST fp16 [M][K];  y_host_f16  HOST fp16 [M][N].
  *   words, lut_f16             DEVICE, the resident packed layer.

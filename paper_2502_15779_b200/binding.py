@@ -51,6 +51,8 @@ def lib():
         L.rcp_gemv_w2a4_grouped.argtypes = [vp, vp, i, vp, vp, i, i, i, vp, vp, vp, vp]
         L.rcp_gemv_w2a4_grouped_variant.restype = i
         L.rcp_gemv_w2a4_grouped_variant.argtypes = [i, vp, vp, i, vp, vp, i, i, i, vp, vp, vp, vp]
+        L.rcp_linear_w2a4.restype = i
+        L.rcp_linear_w2a4.argtypes = [vp, i, i, i, C.c_float, vp, vp, i, i, vp, vp, vp, vp, vp]
         L.rcp_linear_w2a4_host.restype = i
         L.rcp_linear_w2a4_host.argtypes = [vp, i, i, i, C.c_float, vp, vp, i, vp, vp, vp, vp, vp, vp, vp]
         L.rcp_gemv_w2a4_static.restype = i
@@ -185,6 +187,30 @@ def rcp_gemv_w2a4_static(words, lut, xq, scale, y=None):
         _check("rcp_gemv_w2a4_static",
                lib().rcp_gemv_w2a4_static(_ptr(words), _ptr(lut), _ptr(xq), _ptr(scale), M, N, K, _ptr(y),
                                           _stream(words)))
+    return y
+
+
+def rcp_linear_w2a4(x, had_block, clip_ratio, words, lut, group=0, y=None, xq=None, scale=None, workspace=None):
+    """x fp16 [M][K] -> y fp16 [M][N]: activation quantization and LUT GEMV in one call (one kernel for
+    one or two tokens). lut fp16 [N][4] with group=0, [N][K/group][4] otherwise. xq / scale: optional
+    outputs on the one-kernel path, required staging otherwise (pass them to be safe)."""
+    _dev(x, torch.float16, "x")
+    _dev(words, torch.int32, "words")
+    _dev(lut, torch.float16, "lut")
+    M, K = x.shape
+    N, W = words.shape
+    group = int(group)
+    want = (N, 4) if group == 0 else (N, K // max(group, 1), 4)
+    if W * 16 != K or tuple(lut.shape) != want:
+        raise ValueError("shape mismatch between x, words, lut and group")
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.float16, device=words.device)
+    if workspace is None:
+        workspace = make_workspace(M, N, K, words.device)
+    with torch.cuda.device(words.device):
+        _check("rcp_linear_w2a4",
+               lib().rcp_linear_w2a4(_ptr(x), M, K, int(had_block), float(clip_ratio), _ptr(words), _ptr(lut), group, N,
+                                     _ptr(y), _ptr(xq), _ptr(scale), _ptr(workspace), _stream(words)))
     return y
 
 

@@ -57,7 +57,7 @@ __device__ int g_pack_bad;  // set by pack_weights_kernel when it meets a code a
 struct StreamPlan {
   int nchunk, nphase, stages, grid;
   rcp::GemvPhase phase[rcp::kMaxPhases];
-  int off_bar, off_T0c, off_scale, off_red, off_bs;
+  int off_bar, off_T0c, off_scale, off_red, off_bs, off_qbuf;
   size_t smem;
 };
 
@@ -117,7 +117,8 @@ int plan_leftover(int rem, int sms, int nchunk, rcp::GemvPhase* out) {
   return n;
 }
 
-StreamPlan make_plan(int M, int N, int K, int sms, bool grouped = false) {
+// qbuf: bytes of staging for the fused quantizer's cross-warp rotation strides (0 if unused)
+StreamPlan make_plan(int M, int N, int K, int sms, bool grouped = false, size_t qbuf = 0) {
   StreamPlan pl;
   pl.grid = sms;
   pl.nchunk = (K / 16 + rcp::kChunkWords - 1) / rcp::kChunkWords;
@@ -133,14 +134,15 @@ StreamPlan make_plan(int M, int N, int K, int sms, bool grouped = false) {
   // row groups x 3 planes, or (group-wise grid) one fp32 term per warp
   const size_t t0c_bytes = grouped ? (size_t)(M + 1) * pl.nchunk * 16 : (((size_t)M * pl.nchunk * 4) + 15) / 16 * 16;
   const size_t red_bytes = grouped ? (size_t)2 * rcp::kCWarps * 16 * M * 4 : (size_t)2 * 8 * 16 * M * 3 * 4;
-  const size_t misc = 128 + t0c_bytes + 64 + red_bytes;
+  const size_t misc = 128 + t0c_bytes + 128 + red_bytes + qbuf;
   pl.stages = (int)std::min<size_t>(rcp::kMaxStages, (kSmemMax - 1024 - misc - bs_bytes) / rcp::kStageBytes);
   size_t off = (size_t)pl.stages * rcp::kStageBytes;
   pl.off_bar = (int)off; off += 128;
   pl.off_T0c = (int)off; off += t0c_bytes;
-  pl.off_scale = (int)off; off += 64;
+  pl.off_scale = (int)off; off += 128;   // 8 scales, then 16 per-warp maxima of the fused quantizer
   pl.off_red = (int)off; off += red_bytes;
   pl.off_bs = (int)off; off += bs_bytes;
+  pl.off_qbuf = (int)off; off += qbuf;
   pl.smem = off + 1024;
   return pl;
 }
@@ -171,10 +173,10 @@ int sm_count() {
   return n;
 }
 
-template <int MODE, int MTOK, bool GRP = false>
+template <int MODE, int MTOK, bool GRP = false, bool FQ = false>
 int launch_stream_t(const rcp::GemvMaps& maps, const rcp::GemvParams& gp, const StreamPlan& pl, cudaStream_t st) {
   static bool attr_set = false;
-  auto kern = rcp::gemv_stream_kernel<MODE, MTOK, GRP>;
+  auto kern = rcp::gemv_stream_kernel<MODE, MTOK, GRP, FQ>;
   if (!attr_set) {
     RCP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax));
     attr_set = true;
@@ -185,14 +187,33 @@ int launch_stream_t(const rcp::GemvMaps& maps, const rcp::GemvParams& gp, const 
 
 // One launch: M tokens (their expanded activations fit in shared memory). grouped: lut_f16 is
 // [N][K/128][4], one grid per group of 128 weights.
+// Activations still to be rotated and quantized, for the kernels that do it themselves.
+struct FusedAct {
+  const void* x_f16;     // [M][K]
+  int B;                 // rotation block, 1 = none
+  float clip_ratio;
+  uint8_t* xq_out;       // optional
+  void* scale_out;       // optional
+};
+
+// Shapes the in-kernel quantizer takes: one or two tokens; a rotation block of at most 512, or one
+// block spanning a token of 1024 .. 8192 elements.
+bool fused_ok(int M, int K, int B) {
+  if (M > 2 || K % 16) return false;
+  if (B <= 512) return true;
+  return B == K && K <= 8192;
+}
+
 int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const uint8_t* xq, const void* scale_f16,
-                  int M, int N, int K, void* y_f16, void* workspace, cudaStream_t st, bool grouped = false) {
+                  int M, int N, int K, void* y_f16, void* workspace, cudaStream_t st, bool grouped = false,
+                  const FusedAct* fa = nullptr) {
   if (mode != rcp::kModeMma && M > 2) return RCP_ERR_VARIANT;
   if (M > 8) return RCP_ERR_VARIANT;
   if (grouped && (mode == rcp::kModeHybrid || K % 128)) return RCP_ERR_VARIANT;
+  if (fa && (mode != rcp::kModeDp4a || !fused_ok(M, K, fa->B))) return RCP_ERR_VARIANT;
   EncodeTiledFn enc = encode_tiled_fn();
   if (!enc) return cuda_fail(cudaErrorNotSupported);
-  const StreamPlan pl = make_plan(M, N, K, sm_count(), grouped);
+  const StreamPlan pl = make_plan(M, N, K, sm_count(), grouped, (fa && fa->B > 512) ? (size_t)4 * K : 0);
   if (pl.stages < 2 || pl.smem > kSmemMax) return RCP_ERR_SHAPE;
   rcp::GemvMaps maps;
   const cuuint64_t gdim[2] = {(cuuint64_t)(K / 16), (cuuint64_t)N};
@@ -222,6 +243,22 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   gp.ramp_clk = (int)((double)rcp::kStageBytes * pl.grid / 6.0e12 * 1.9e9);
   gp.off_bar = pl.off_bar; gp.off_T0c = pl.off_T0c; gp.off_scale = pl.off_scale; gp.off_red = pl.off_red;
   gp.off_bs = pl.off_bs;
+  gp.off_qbuf = pl.off_qbuf;
+  gp.x = nullptr; gp.xq_out = nullptr; gp.scale_out = nullptr;
+  gp.B = 1; gp.inv_sqrt_b = 1.f; gp.clip_ratio = 1.f;
+  if (fa) {
+    gp.x = static_cast<const __half*>(fa->x_f16);
+    gp.xq_out = fa->xq_out;
+    gp.scale_out = static_cast<__half*>(fa->scale_out);
+    gp.B = fa->B;
+    gp.inv_sqrt_b = (float)(1.0 / std::sqrt((double)fa->B));
+    gp.clip_ratio = fa->clip_ratio;
+    if (grouped)
+      return M == 1 ? launch_stream_t<rcp::kModeDp4a, 1, true, true>(maps, gp, pl, st)
+                    : launch_stream_t<rcp::kModeDp4a, 2, true, true>(maps, gp, pl, st);
+    return M == 1 ? launch_stream_t<rcp::kModeDp4a, 1, false, true>(maps, gp, pl, st)
+                  : launch_stream_t<rcp::kModeDp4a, 2, false, true>(maps, gp, pl, st);
+  }
   if (grouped) {
     if (mode == rcp::kModeDp4a)
       return M == 1 ? launch_stream_t<rcp::kModeDp4a, 1, true>(maps, gp, pl, st)
@@ -516,6 +553,33 @@ int rcp_gemv_w2a4_static(const uint32_t* words, const void* lut_f16, const uint8
                                stream);
 }
 
+int rcp_linear_w2a4(const void* x_f16, int M, int K, int had_block, float clip_ratio, const uint32_t* words,
+                    const void* lut_f16, int group, int N, void* y_f16, uint8_t* xq, void* scale_f16, void* workspace,
+                    void* stream) {
+  if (!x_f16 || !words || !lut_f16 || !y_f16) return RCP_ERR_NULL;
+  if (M < 1 || M > rcp::kMaxTokens || N < 1 || !k_ok(K)) return RCP_ERR_SHAPE;
+  const int B = had_block <= 1 ? 1 : had_block;
+  if (B > 8192 || (B & (B - 1)) || K % B) return RCP_ERR_SHAPE;
+  if (!(clip_ratio > 0.f) || !std::isfinite(clip_ratio)) return RCP_ERR_SHAPE;
+  if (group != 0 && (group < 16 || group % 16 || K % group)) return RCP_ERR_SHAPE;
+  if (!aligned16(x_f16) || !aligned16(words) || !aligned16(xq) || (reinterpret_cast<uintptr_t>(lut_f16) & 7u) ||
+      (reinterpret_cast<uintptr_t>(y_f16) & 1u) || (reinterpret_cast<uintptr_t>(scale_f16) & 1u) ||
+      (reinterpret_cast<uintptr_t>(workspace) & 3u))
+    return RCP_ERR_ALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (fused_ok(M, K, B) && (group == 0 || group == 128)) {
+    const FusedAct fa{x_f16, B, clip_ratio, xq, scale_f16};
+    return launch_stream(rcp::kModeDp4a, words, lut_f16, nullptr, nullptr, M, N, K, y_f16, workspace, st, group == 128,
+                         &fa);
+  }
+  // otherwise the two kernels one after the other; they need the staging buffers
+  if (!xq || !scale_f16) return RCP_ERR_NULL;
+  int rc = rcp_quantize_act(x_f16, M, K, had_block, clip_ratio, xq, scale_f16, stream);
+  if (rc != RCP_OK) return rc;
+  if (group == 0) return rcp_gemv_w2a4(words, lut_f16, xq, scale_f16, M, N, K, y_f16, workspace, nullptr, stream);
+  return rcp_gemv_w2a4_grouped(words, lut_f16, group, xq, scale_f16, M, N, K, y_f16, workspace, nullptr, stream);
+}
+
 int rcp_linear_w2a4_host(const void* x_host_f16, int M, int K, int had_block, float clip_ratio,
                          const uint32_t* words, const void* lut_f16, int N, void* y_host_f16, void* x_dev,
                          uint8_t* xq_dev, void* scale_dev, void* y_dev, void* workspace, void* stream) {
@@ -523,9 +587,8 @@ int rcp_linear_w2a4_host(const void* x_host_f16, int M, int K, int had_block, fl
   if (M < 1 || M > rcp::kMaxTokens || N < 1 || !k_ok(K)) return RCP_ERR_SHAPE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   RCP_CUDA(cudaMemcpyAsync(x_dev, x_host_f16, (size_t)M * K * 2, cudaMemcpyHostToDevice, st));
-  int rc = rcp_quantize_act(x_dev, M, K, had_block, clip_ratio, xq_dev, scale_dev, stream);
-  if (rc != RCP_OK) return rc;
-  rc = rcp_gemv_w2a4(words, lut_f16, xq_dev, scale_dev, M, N, K, y_dev, workspace, nullptr, stream);
+  const int rc = rcp_linear_w2a4(x_dev, M, K, had_block, clip_ratio, words, lut_f16, 0, N, y_dev, xq_dev, scale_dev,
+                                 workspace, stream);
   if (rc != RCP_OK) return rc;
   RCP_CUDA(cudaMemcpyAsync(y_host_f16, y_dev, (size_t)M * N * 2, cudaMemcpyDeviceToHost, st));
   return RCP_OK;
