@@ -129,9 +129,31 @@ class LayerSet:
     def step(self, copy, variant="auto"):
         r = self.rcp
         for li, L in enumerate(self.layers):
-            r.rcp_quantize_act(self.x[li], L.had_block, 1.0, xq=self.xq[li], scale=self.scale[li])
-            r.rcp_gemv_w2a4(self.words[li][copy], self.luts[li][copy], self.xq[li], self.scale[li], y=self.y[li],
-                            workspace=self.ws[li], variant=variant)
+            if variant == "auto":
+                # the library's own chain: one kernel where that is faster, else quantizer + GEMV
+                r.rcp_linear_w2a4(self.x[li], L.had_block, 1.0, self.words[li][copy], self.luts[li][copy], y=self.y[li],
+                                  xq=self.xq[li], scale=self.scale[li], workspace=self.ws[li])
+            else:
+                r.rcp_quantize_act(self.x[li], L.had_block, 1.0, xq=self.xq[li], scale=self.scale[li])
+                r.rcp_gemv_w2a4(self.words[li][copy], self.luts[li][copy], self.xq[li], self.scale[li], y=self.y[li],
+                                workspace=self.ws[li], variant=variant)
+
+    def launches_per_step(self, variant="auto"):
+        r = self.rcp
+        if variant == "auto":
+            return sum(r.rcp_linear_w2a4_launches(self.M, L.K, L.had_block) for L in self.layers)
+        return sum(1 + -(-self.M // (8 if variant in ("mma", "mma_only") else 2)) for L in self.layers)
+
+    def stream_kernels_only(self, copy, variant="auto"):
+        """The launches of the streaming kernel a step makes, without the stand-alone quantizer launches."""
+        r = self.rcp
+        for li, L in enumerate(self.layers):
+            if variant == "auto" and r.rcp_linear_w2a4_launches(self.M, L.K, L.had_block) == 1:
+                r.rcp_linear_w2a4(self.x[li], L.had_block, 1.0, self.words[li][copy], self.luts[li][copy], y=self.y[li],
+                                  xq=self.xq[li], scale=self.scale[li], workspace=self.ws[li])
+            else:
+                r.rcp_gemv_w2a4(self.words[li][copy], self.luts[li][copy], self.xq[li], self.scale[li], y=self.y[li],
+                                workspace=self.ws[li], variant=variant)
 
     def gemv_bytes(self):
         return sum(cfgs.gemv_bytes(self.M, L.N, L.K) for L in self.layers)
@@ -422,25 +444,41 @@ def main():
     clocks = sampler.stop() if sampler else None
     step_bytes = layer.gemv_bytes() + layer.quant_bytes()
     ms_per_step, value, _ = replica_metrics(ms, step_bytes, args.steps, dist, device)
-    launches = args.steps * 2 * len(layer.layers)
+    launches = args.steps * layer.launches_per_step(args.variant)
 
-    # ---- dominant kernel alone: the GEMV launches of the layer, back to back, cold L2
-    def gemv_only(c):
-        for li, L in enumerate(layer.layers):
-            rcp.rcp_gemv_w2a4(layer.words[li][c], layer.luts[li][c], layer.xq[li], layer.scale[li], y=layer.y[li],
-                              workspace=layer.ws[li], variant=args.variant)
-    ggraphs = [capture(lambda c=c: gemv_only(c), stream) for c in range(copies)]
+    # ---- dominant kernel alone: the streaming-kernel launches of a step (the GEMV, with the quantizer
+    # inside where the step uses the single kernel), back to back, cold L2
+    ggraphs = [capture(lambda c=c: layer.stream_kernels_only(c, args.variant), stream) for c in range(copies)]
     time_graph_replays(ggraphs, order[:8], stream)
     gms = min(time_graph_replays(ggraphs, order, stream) for _ in range(3))
-    g_launches = args.steps * len(layer.layers)
-    g_bytes_per_launch = layer.gemv_bytes() / len(layer.layers)
+    g_launches = args.steps * (layer.launches_per_step(args.variant) -
+                               sum(1 for L in layer.layers
+                                   if args.variant != "auto" or rcp.rcp_linear_w2a4_launches(M, L.K, L.had_block) > 1))
+    g_bytes_per_launch = layer.gemv_bytes() * args.steps / g_launches
     g_us = gms * 1e3 / g_launches
     achieved = g_bytes_per_launch / g_us / 1e3
     peaks, peak_kind = measured_peaks()
-    roofline = {"bound": "hbm", "kernel": "gemv_stream_kernel", "achieved": round(achieved, 1),
+    roofline = {"bound": "hbm", "kernel": "gemv_stream_kernel (with the activation quantizer inside where the step "
+                                          "uses the single kernel)", "achieved": round(achieved, 1),
                 "peak": peaks["hbm_gbs"], "peak_kind": peak_kind, "unit": "GB/s",
                 "frac": round(achieved / peaks["hbm_gbs"], 4), "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
                 "avg_launch_us": round(g_us, 3), "bytes_per_launch": int(g_bytes_per_launch), "traffic": None}
+    # for comparison: the plain GEMV launches alone (activations already quantized), same protocol
+    def plain_gemv(c):
+        for li, L in enumerate(layer.layers):
+            rcp.rcp_gemv_w2a4(layer.words[li][c], layer.luts[li][c], layer.xq[li], layer.scale[li], y=layer.y[li],
+                              workspace=layer.ws[li], variant=args.variant)
+    pgraphs = [capture(lambda c=c: plain_gemv(c), stream) for c in range(copies)]
+    time_graph_replays(pgraphs, order[:8], stream)
+    pms = min(time_graph_replays(pgraphs, order, stream) for _ in range(3))
+    p_launches = args.steps * sum(-(-M // (8 if (M > 1 or args.variant in ("mma", "mma_only")) else 2))
+                                  for _ in layer.layers)
+    p_us = pms * 1e3 / p_launches
+    p_ach = layer.gemv_bytes() * args.steps / p_launches / p_us / 1e3
+    roofline["plain_gemv"] = {"avg_launch_us": round(p_us, 3), "achieved": round(p_ach, 1),
+                              "frac": round(p_ach / peaks["hbm_gbs"], 4),
+                              "note": "rcp_gemv_w2a4 launches alone, activations quantized beforehand"}
+    del pgraphs
     prof = os.path.join(ROOT, "profiles", "traffic.json")
     if os.path.exists(prof):
         try:
@@ -513,7 +551,9 @@ def main():
            "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True, "scaling": "weak",
            "vs_baseline": None, "dtype": "int32", "data": "synthetic",
            "config": {"workload": workload_name(cfg, M),
-                      "step": "per linear: rcp_quantize_act + rcp_gemv_w2a4, replayed from a CUDA graph",
+                      "step": "per linear: rcp_linear_w2a4 (activation quantization + LUT GEMV: one kernel for one "
+                              "token of 4096 or 8192 under one rotation block, else rcp_quantize_act then "
+                              "rcp_gemv_w2a4), replayed from a CUDA graph",
                       "cold_l2": f"{copies} distinct weight copies in rotation ({copies * wbytes / 1e6:.0f} MB > 2x L2 "
                                  f"of {L2 / 1e6:.0f} MB)",
                       "variant": args.variant, "parallelism": "replicas only" if world > 1 else "single GPU",

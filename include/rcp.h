@@ -158,17 +158,22 @@ int rcp_gemv_w2a4_grouped_variant(int variant, const uint32_t* words, const void
  * == 0) or rcp_gemv_w2a4_grouped (group > 0), same arguments, same results bit for bit in xq and
  * scale and within the GEMV's tolerance in y (Section 4.4 data path; Appendix A.7 counts the
  * separate activation quantizer as the overhead this removes).
- *   For one or two tokens, a rotation block of at most 512 (or one block spanning a token of at
- *   most 8192 elements) and group in {0, 128}, a single kernel does both: every CTA rotates and
- *   quantizes the token itself while its first weight requests are in flight. xq and scale_f16
- *   are then optional outputs (NULL: not written). Every other case runs the two kernels one after
- *   the other and needs xq [M][K/2] and scale_f16 [M] as staging: RCP_ERR_NULL without them.
+ *   For one token of 4096 or 8192 elements under one rotation block (had_block == K) and group in
+ *   {0, 128}, a single kernel does both: every CTA rotates and quantizes the token itself while its
+ *   first weight requests are in flight (measured faster than two kernels for these shapes only).
+ *   xq and scale_f16 are then optional outputs (NULL: not written). Every other case runs the two
+ *   kernels one after the other and needs xq [M][K/2] and scale_f16 [M] as staging: RCP_ERR_NULL
+ *   without them.
  *   x_f16 obeys stream order; words and lut_f16 are layer constants (see rcp_gemv_w2a4).
  * Never synchronizes.
  */
 int rcp_linear_w2a4(const void* x_f16, int M, int K, int had_block, float clip_ratio,
                     const uint32_t* words, const void* lut_f16, int group, int N, void* y_f16,
                     uint8_t* xq, void* scale_f16, void* workspace, void* stream);
+
+/* Kernel launches one rcp_linear_w2a4 call makes for a shape (1: the single kernel; otherwise the
+ * quantizer plus one GEMV launch per batch of tokens). Host only. Negative status on a bad shape. */
+int rcp_linear_w2a4_launches(int M, int K, int had_block, int group);
 
 /*
  * One decode linear layer end to end with HOST activations (Section 4.4 data path: rotate and

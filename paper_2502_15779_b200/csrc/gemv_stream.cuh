@@ -74,9 +74,8 @@ struct GemvParams {
   const __half* x;
   uint8_t* xq_out;      // optional [M][K/2]: the int4 activations, written by CTA 0
   __half* scale_out;    // optional [M]
-  int B;                // rotation block (1 = none); at most 512, or the whole K (a power of two up to 8192)
-  float inv_sqrt_b, clip_ratio;
-  int off_qbuf;         // 4 K bytes of shared memory when B > 512
+  float inv_sqrt_b, clip_ratio;   // the rotation block is the whole token, K = 4096 or 8192
+  int off_qbuf;         // 4 K bytes of shared memory
   int stages;           // ring depth
   int ramp_clk;         // clocks between the first `stages` requests of a CTA
   int off_bar, off_T0c, off_scale, off_red, off_bs;   // shared-memory byte offsets from the aligned base
@@ -159,12 +158,13 @@ __device__ __forceinline__ void dp4a_s8s8(int& d, uint32_t a, uint32_t b) {
 //       cores, the b0*b1 plane on dp4a; kModeDp4a: everything on dp4a (CUDA cores only)
 // MTOK  tokens, fixed at compile time for the dp4a modes (1 or 2); 0 = run-time, up to 8 (kModeMma)
 // GRP   one grid per group of 128 weights instead of one per row (kModeHybrid has no such form)
-// FQ    the activations arrive as fp16 and every CTA rotates and quantizes them itself (Appendix A.2,
-//       Section 4.4), in the arithmetic order of the stand-alone quantizer: bit-identical int4 values.
-//       For one or two tokens this costs less than a kernel of its own and hides behind the first
-//       weight requests. A thread takes the words (16 consecutive activations) tid, tid + 512, ...:
-//       strides 1..8 in registers, 16..256 by lane exchanges, 512 and up (one block spanning the
-//       token) through shared memory, one thread per (lane, element) column over the warps.
+// FQ    one token of 4096 or 8192 activations under one rotation block: the activations arrive as
+//       fp16 and every CTA rotates and quantizes them itself (Appendix A.2, Section 4.4), in the
+//       arithmetic order of the stand-alone quantizer: bit-identical int4 values. For these shapes
+//       (where the stand-alone kernel needs a cluster and passes through distributed shared memory)
+//       it costs less than a kernel of its own. A thread takes one word (16 consecutive activations):
+//       strides 1..8 in registers, 16..256 by lane exchanges, 512 and up through shared memory, one
+//       thread per (lane, element) column over the warps.
 template <int MODE, int MTOK, bool GRP, bool FQ = false>
 __global__ void __launch_bounds__(kGThreads, 1)
 gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
@@ -252,169 +252,144 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
 
   // ------------------------------------------------------------------ fused quantizer (consumer warps)
   if constexpr (FQ) {
-    static_assert(!FQ || (MODE == kModeDp4a && MTOK > 0), "the fused quantizer serves the one- and two-token kernels");
+    static_assert(!FQ || (MODE == kModeDp4a && MTOK == 1), "the fused quantizer serves the one-token kernels");
     constexpr int NT = kCWarps * 32;
-    const int W = p.K / 16;
-    const int nr = (W + NT - 1) / NT;
-    const int B = p.B;
-    float* const qbuf = reinterpret_cast<float*>(gen + p.off_qbuf);   // [16][W] when B > 512
+    const int W = p.K / 16;                                           // 256 or 512 words: one per thread
+    float* const qbuf = reinterpret_cast<float*>(gen + p.off_qbuf);   // [16][W]
     float* const s_amax = s_scale + 8;                                // [16 warps] behind the scales
-    // one word: 16 activations, rotated within the block as far as registers and lanes reach
-    auto load_rotate = [&](int col, int word, float (&v)[16]) {
-      if (word < W) {
-        const uint4* src = reinterpret_cast<const uint4*>(p.x + (size_t)col * p.K + (size_t)word * 16);
-        const uint4 r0 = __ldg(src), r1 = __ldg(src + 1);
-        const __half2* h0 = reinterpret_cast<const __half2*>(&r0);
-        const __half2* h1 = reinterpret_cast<const __half2*>(&r1);
+    float v[16];
+    if (tid < W) {
+      const uint4* src = reinterpret_cast<const uint4*>(p.x + (size_t)tid * 16);
+      const uint4 r0 = __ldg(src), r1 = __ldg(src + 1);
+      const __half2* h0 = reinterpret_cast<const __half2*>(&r0);
+      const __half2* h1 = reinterpret_cast<const __half2*>(&r1);
 #pragma unroll
-        for (int e = 0; e < 4; e++) {
-          const float2 f0 = __half22float2(h0[e]), f1 = __half22float2(h1[e]);
-          v[2 * e] = f0.x; v[2 * e + 1] = f0.y; v[8 + 2 * e] = f1.x; v[8 + 2 * e + 1] = f1.y;
-        }
-      } else {
-#pragma unroll
-        for (int e = 0; e < 16; e++) v[e] = 0.f;
+      for (int e = 0; e < 4; e++) {
+        const float2 f0 = __half22float2(h0[e]), f1 = __half22float2(h1[e]);
+        v[2 * e] = f0.x; v[2 * e + 1] = f0.y; v[8 + 2 * e] = f1.x; v[8 + 2 * e + 1] = f1.y;
       }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 16; e++) v[e] = 0.f;
+    }
+    // strides 1 .. 8: inside the word
+#pragma unroll
+    for (int h = 1; h < 16; h *= 2) {
+#pragma unroll
+      for (int e = 0; e < 16; e++) {
+        if ((e & h) == 0) {
+          const float u = v[e], w = v[e + h];
+          v[e] = __fadd_rn(u, w);
+          v[e + h] = __fsub_rn(u, w);
+        }
+      }
+    }
+    // strides 16 .. 256: element stride 16 d <-> lane distance d
+#pragma unroll
+    for (int d = 1; d < 32; d *= 2) {
+      const bool upper = (lane & d) != 0;
+#pragma unroll
+      for (int e = 0; e < 16; e++) {
+        const float other = __shfl_xor_sync(0xffffffffu, v[e], d);
+        v[e] = upper ? __fsub_rn(other, v[e]) : __fadd_rn(v[e], other);
+      }
+    }
+    // strides 512 .. K/2: across the R = W / 32 warps that hold data, through shared memory; thread
+    // (element tid >> 5, lane) takes the R values of its column, 32 words apart
+    {
+      if (tid < W) {
+#pragma unroll
+        for (int e = 0; e < 16; e++) qbuf[e * W + tid] = v[e];
+      }
+      asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");
+      const int R = W >> 5;   // 8 or 16
+      float* const colp = qbuf + (tid >> 5) * W + lane;
+      float tv[16];
+#pragma unroll
+      for (int w = 0; w < 16; w++) tv[w] = (w < R) ? colp[w * 32] : 0.f;
 #pragma unroll
       for (int h = 1; h < 16; h *= 2) {
-        if (h < B) {
+        if (h < R) {
 #pragma unroll
-          for (int e = 0; e < 16; e++) {
-            if ((e & h) == 0) {
-              const float u = v[e], w = v[e + h];
-              v[e] = __fadd_rn(u, w);
-              v[e + h] = __fsub_rn(u, w);
+          for (int w = 0; w < 16; w++) {
+            if ((w & h) == 0) {
+              const float u = tv[w], z = tv[w + h];
+              tv[w] = __fadd_rn(u, z);
+              tv[w + h] = __fsub_rn(u, z);
             }
           }
         }
       }
 #pragma unroll
-      for (int d = 1; d < 32; d *= 2) {   // element stride 16 d <-> lane distance d
-        if (16 * d < B) {
-          const bool upper = (lane & d) != 0;
-#pragma unroll
-          for (int e = 0; e < 16; e++) {
-            const float other = __shfl_xor_sync(0xffffffffu, v[e], d);
-            v[e] = upper ? __fsub_rn(other, v[e]) : __fadd_rn(v[e], other);
-          }
-        }
-      }
-    };
-    // strides 512 .. B/2 (B == K > 512, one word per thread): across the warps through shared memory
-    auto cross_warps = [&](float (&v)[16]) {
-      if (B > 512) {
-        if (tid < W) {
-#pragma unroll
-          for (int e = 0; e < 16; e++) qbuf[e * W + tid] = v[e];
-        }
-        asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");
-        const int R = W >> 5;   // warps that hold data: 2, 4, 8 or 16
-        float* const colp = qbuf + (tid >> 5) * W + lane;   // column (element tid >> 5, lane): R values 32 apart
-        float tv[16];
-#pragma unroll
-        for (int w = 0; w < 16; w++) tv[w] = (w < R) ? colp[w * 32] : 0.f;
-#pragma unroll
-        for (int h = 1; h < 16; h *= 2) {
-          if (h < R) {
-#pragma unroll
-            for (int w = 0; w < 16; w++) {
-              if ((w & h) == 0) {
-                const float u = tv[w], z = tv[w + h];
-                tv[w] = __fadd_rn(u, z);
-                tv[w + h] = __fsub_rn(u, z);
-              }
-            }
-          }
-        }
-#pragma unroll
-        for (int w = 0; w < 16; w++) if (w < R) colp[w * 32] = tv[w];
-        asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");
-        if (tid < W) {
-#pragma unroll
-          for (int e = 0; e < 16; e++) v[e] = qbuf[e * W + tid];
-        }
-      }
-    };
-    for (int col = 0; col < M; col++) {
-      float v[16];
-      // pass 1: the token's absmax
-      float amax = 0.f;
-      for (int r = 0; r < nr; r++) {
-        load_rotate(col, tid + r * NT, v);
-        cross_warps(v);
-#pragma unroll
-        for (int e = 0; e < 16; e++) {
-          if (B > 1) v[e] = __fmul_rn(v[e], p.inv_sqrt_b);
-          amax = fmaxf(amax, fabsf(v[e]));
-        }
-      }
-#pragma unroll
-      for (int d = 16; d > 0; d >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, d));
-      if (lane == 0) s_amax[warp] = amax;
+      for (int w = 0; w < 16; w++) if (w < R) colp[w * 32] = tv[w];
       asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");
+      if (tid < W) {
 #pragma unroll
-      for (int w = 0; w < kCWarps; w++) amax = fmaxf(amax, s_amax[w]);
-      const float s32 = __fdiv_rn(__fmul_rn(amax, p.clip_ratio), 7.0f);
-      const __half s16 = __float2half_rn(s32);
-      const float sc = __half2float(s16);
-      if (tid == 0) {
-        s_scale[col] = sc;
-        if (b == 0 && p.scale_out) p.scale_out[col] = s16;
+        for (int e = 0; e < 16; e++) v[e] = qbuf[e * W + tid];
       }
-      // pass 2: quantize (with several words per thread the rotation is simply done again)
-      for (int r = 0; r < nr; r++) {
-        const int word = tid + r * NT;
-        if (nr > 1) {
-          load_rotate(col, word, v);
+    }
+    float amax = 0.f;
 #pragma unroll
-          for (int e = 0; e < 16; e++) if (B > 1) v[e] = __fmul_rn(v[e], p.inv_sqrt_b);
-        }
-        int q[16];
-        int tsum = 0;
+    for (int e = 0; e < 16; e++) {
+      v[e] = __fmul_rn(v[e], p.inv_sqrt_b);
+      amax = fmaxf(amax, fabsf(v[e]));
+    }
 #pragma unroll
-        for (int e = 0; e < 16; e++) {
-          int qq = 0;
-          if (sc != 0.f && word < W) qq = max(-8, min(7, __float2int_rn(__fdiv_rn(v[e], sc))));
-          q[e] = qq;
-          tsum += qq;
-        }
-        const int ch = word >> 5, wi = word & 31;
-        if (word < p.nchunk * kChunkWords) {
-          uint32_t Q[4];
+    for (int d = 16; d > 0; d >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, d));
+    if (lane == 0) s_amax[warp] = amax;
+    asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");
 #pragma unroll
-          for (int pp = 0; pp < 4; pp++) {
-            const int m = (pp & 1) ? 1 : 4;   // even positions carry 4 q
-            Q[pp] = (uint32_t)((q[pp] * m) & 0xFF) | ((uint32_t)((q[4 + pp] * m) & 0xFF) << 8) |
-                    ((uint32_t)((q[8 + pp] * m) & 0xFF) << 16) | ((uint32_t)((q[12 + pp] * m) & 0xFF) << 24);
-          }
-          uint8_t* dst = bs + ((size_t)(((ch * 4 + ((wi >> 1) & 3)) * 2) * ncol + col)) * 64 + (wi >> 3) * 16 + (wi & 1) * 4;
-          *reinterpret_cast<uint32_t*>(dst) = Q[0];
-          *reinterpret_cast<uint32_t*>(dst + 8) = Q[1];
-          *reinterpret_cast<uint32_t*>(dst + (size_t)ncol * 64) = Q[2];
-          *reinterpret_cast<uint32_t*>(dst + (size_t)ncol * 64 + 8) = Q[3];
-        }
-        if (b == 0 && p.xq_out && word < W) {
-          uint32_t lo32 = 0, hi32 = 0;
+    for (int w = 0; w < kCWarps; w++) amax = fmaxf(amax, s_amax[w]);
+    const float s32 = __fdiv_rn(__fmul_rn(amax, p.clip_ratio), 7.0f);
+    const __half s16 = __float2half_rn(s32);
+    const float sc = __half2float(s16);
+    if (tid == 0) {
+      s_scale[0] = sc;
+      if (b == 0 && p.scale_out) p.scale_out[0] = s16;
+    }
+    int q[16];
+    int tsum = 0;
 #pragma unroll
-          for (int e = 0; e < 8; e++) {
-            lo32 |= (uint32_t)(q[e] & 0xF) << (4 * e);
-            hi32 |= (uint32_t)(q[8 + e] & 0xF) << (4 * e);
-          }
-          *reinterpret_cast<uint2*>(p.xq_out + (size_t)col * (p.K / 2) + (size_t)word * 8) = make_uint2(lo32, hi32);
-        }
-        // sums of q: a warp holds exactly one chunk (32 consecutive words), eight lanes one group of 128
-        tsum += __shfl_xor_sync(0xffffffffu, tsum, 1);
-        tsum += __shfl_xor_sync(0xffffffffu, tsum, 2);
-        tsum += __shfl_xor_sync(0xffffffffu, tsum, 4);
-        if constexpr (GRP) {
-          if ((lane & 7) == 0 && ch < p.nchunk) s_T0c[col * ng4 + (word >> 3)] = tsum;
-        } else {
-          tsum += __shfl_xor_sync(0xffffffffu, tsum, 8);
-          tsum += __shfl_xor_sync(0xffffffffu, tsum, 16);
-          if (lane == 0 && ch < p.nchunk) s_T0c[col * p.nchunk + ch] = tsum;
-        }
+    for (int e = 0; e < 16; e++) {
+      int qq = 0;
+      if (sc != 0.f && tid < W) qq = max(-8, min(7, __float2int_rn(__fdiv_rn(v[e], sc))));
+      q[e] = qq;
+      tsum += qq;
+    }
+    const int ch = tid >> 5, wi = tid & 31;
+    if (tid < p.nchunk * kChunkWords) {
+      uint32_t Q[4];
+#pragma unroll
+      for (int pp = 0; pp < 4; pp++) {
+        const int m = (pp & 1) ? 1 : 4;   // even positions carry 4 q
+        Q[pp] = (uint32_t)((q[pp] * m) & 0xFF) | ((uint32_t)((q[4 + pp] * m) & 0xFF) << 8) |
+                ((uint32_t)((q[8 + pp] * m) & 0xFF) << 16) | ((uint32_t)((q[12 + pp] * m) & 0xFF) << 24);
       }
-      asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");   // s_amax and qbuf are free for the next token
+      uint8_t* dst = bs + (size_t)((ch * 4 + ((wi >> 1) & 3)) * 2) * 64 + (wi >> 3) * 16 + (wi & 1) * 4;
+      *reinterpret_cast<uint32_t*>(dst) = Q[0];
+      *reinterpret_cast<uint32_t*>(dst + 8) = Q[1];
+      *reinterpret_cast<uint32_t*>(dst + 64) = Q[2];
+      *reinterpret_cast<uint32_t*>(dst + 64 + 8) = Q[3];
+    }
+    if (b == 0 && p.xq_out && tid < W) {
+      uint32_t lo32 = 0, hi32 = 0;
+#pragma unroll
+      for (int e = 0; e < 8; e++) {
+        lo32 |= (uint32_t)(q[e] & 0xF) << (4 * e);
+        hi32 |= (uint32_t)(q[8 + e] & 0xF) << (4 * e);
+      }
+      *reinterpret_cast<uint2*>(p.xq_out + (size_t)tid * 8) = make_uint2(lo32, hi32);
+    }
+    // sums of q: a warp holds exactly one chunk (32 consecutive words), eight lanes one group of 128
+    tsum += __shfl_xor_sync(0xffffffffu, tsum, 1);
+    tsum += __shfl_xor_sync(0xffffffffu, tsum, 2);
+    tsum += __shfl_xor_sync(0xffffffffu, tsum, 4);
+    if constexpr (GRP) {
+      if ((lane & 7) == 0 && ch < p.nchunk) s_T0c[tid >> 3] = tsum;
+    } else {
+      tsum += __shfl_xor_sync(0xffffffffu, tsum, 8);
+      tsum += __shfl_xor_sync(0xffffffffu, tsum, 16);
+      if (lane == 0 && ch < p.nchunk) s_T0c[ch] = tsum;
     }
     if constexpr (!GRP)
       for (int i = tid; i < 2 * 8 * 16 * M * 3; i += kCWarps * 32) s_red[i] = 0;

@@ -45,9 +45,11 @@ def _check(N, K, B, M, group, clip, seed, kind="uniform", rows=None, staging=Tru
 
 
 CASES = [
-    # N, K, B, M: rotation inside a word, inside a warp, across warps (one block per token), none; ragged K
+    # N, K, B, M. One token of 4096 or 8192 under one block takes the single kernel (several row counts:
+    # rounds, leftover phases, ragged tail); everything else the two kernels
     (40, 64, 1, 1), (40, 64, 64, 2), (100, 256, 16, 1), (33, 512, 128, 2), (64, 512, 512, 1), (129, 1024, 1024, 1),
     (300, 2048, 2048, 1), (300, 2048, 2048, 2), (256, 4096, 4096, 1), (77, 8192, 8192, 2), (500, 8192, 128, 1),
+    (77, 8192, 8192, 1), (2500, 8192, 8192, 1), (4097, 4096, 4096, 1), (1, 4096, 4096, 1), (5000, 8192, 8192, 1),
     (130, 11008, 128, 1), (64, 28672, 128, 2), (40, 14336, 128, 1), (513, 1152, 128, 2), (2500, 4096, 256, 1),
     (4800, 1024, 512, 2), (64, 32768, 512, 1),
     # shapes the single kernel does not take: the two kernels run one after the other
@@ -65,7 +67,9 @@ def test_linear_matches_oracle(N, K, B, M, group):
 
 def test_linear_clip_ratio_zero_token_and_optional_outputs():
     _check(70, 2048, 2048, 2, 0, 0.9, seed=3)
-    _check(70, 1024, 128, 1, 128, 0.9, seed=4, staging=False)   # the single kernel needs no staging
+    _check(70, 4096, 4096, 1, 0, 0.9, seed=5)
+    _check(70, 8192, 8192, 1, 128, 0.9, seed=4, staging=False)   # the single kernel needs no staging
+    _check(600, 4096, 4096, 1, 0, 1.0, seed=6, staging=False)
     N, K, M = 48, 1024, 2
     codes, lut = synth.make_layer(N, K, 128, "uniform", 9, device=DEV)
     x = synth.make_activations(M, K, 9, device=DEV)
