@@ -471,8 +471,10 @@ def main():
     pgraphs = [capture(lambda c=c: plain_gemv(c), stream) for c in range(copies)]
     time_graph_replays(pgraphs, order[:8], stream)
     pms = min(time_graph_replays(pgraphs, order, stream) for _ in range(3))
-    p_launches = args.steps * sum(-(-M // (8 if (M > 1 or args.variant in ("mma", "mma_only")) else 2))
-                                  for _ in layer.layers)
+    # had_block 1 never takes the single kernel: the count is the quantizer plus the GEMV launches
+    p_launches = args.steps * sum(rcp.rcp_linear_w2a4_launches(M, L.K, 1) - 1 if args.variant == "auto"
+                                  else -(-M // (8 if args.variant in ("mma", "mma_only") else 2))
+                                  for L in layer.layers)
     p_us = pms * 1e3 / p_launches
     p_ach = layer.gemv_bytes() * args.steps / p_launches / p_us / 1e3
     roofline["plain_gemv"] = {"avg_launch_us": round(p_us, 3), "achieved": round(p_ach, 1),
