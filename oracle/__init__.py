@@ -230,3 +230,21 @@ def percode_int_grouped(lut_bits, S):
     ai = np.empty((M, N), dtype=np.int64)
     lib().orc_percode_int_grouped(_p(lut), _p(S), C.c_int(M), C.c_int(N), C.c_int(NG), _p(ai))
     return ai
+
+
+def ldp_export(w_f16_bits, sb, sg, s1, s2, G):
+    """Partitioning quantizer export. w uint16 [N][K] (fp16 bits); sb, sg, s1, s2 float32 [N][K/G] (the
+    sigmoids of beta, gamma, s_1, s_2). Returns dict(codes u8 [N][K], lut uint16 [N][K/G][4])."""
+    w = _c(w_f16_bits, np.uint16)
+    N, K = w.shape
+    assert K % G == 0
+    arrs = [_c(a, np.float32) for a in (sb, sg, s1, s2)]
+    for a in arrs:
+        assert a.shape == (N, K // G)
+    codes = np.empty((N, K), dtype=np.uint8)
+    lut = np.empty((N, K // G, 4), dtype=np.uint16)
+    rc = lib().orc_ldp_export(_p(w), _p(arrs[0]), _p(arrs[1]), _p(arrs[2]), _p(arrs[3]), C.c_int(N), C.c_int(K),
+                              C.c_int(G), _p(codes), _p(lut))
+    if rc:
+        raise ValueError(f"orc_ldp_export failed: {rc}")
+    return dict(codes=codes, lut=lut)

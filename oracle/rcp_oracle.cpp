@@ -23,7 +23,10 @@
 // LUT lookup of unpacked codes == dequantized weight matrix; affine/constant LUT special
 // cases reducing to a plain integer GEMV. Group-wise LUT form: one group == the per-row form;
 // equal grids in every group == the per-row form; brute force; exact integer equality with
-// its direct form; dense matrix product with the group-wise dequantized weights.
+// its direct form; dense matrix product with the group-wise dequantized weights. Export of the
+// partitioning quantizer: hand-computed fixture, the uniform initial point == the textbook
+// asymmetric 2-bit quantizer, the range ends and bin centres the paper states, monotone codes,
+// the sum form of the dequantizer == LUT lookup.
 // fp16 output y: the paper prints no worked numeric GEMV example, so y is pinned only by the
 // mathematical identities above, not by a printed value.
 #include <cstdint>
@@ -457,6 +460,81 @@ void orc_percode_int_grouped(const uint16_t* lut_f16, const int32_t* S, int M, i
         }
       acc_int[(size_t)m * N + n] = ai;
     }
+}
+
+// ---------------------------------------------------------------------------------------
+// Learnable direct partitioning, export of a trained layer to the kernel's inputs (Section 3.3,
+// Eqs. "partition", the grid t_i, "quant", "dequantgrid" and Section 3.4 Eq. "deqgrid"; clipping
+// range from Section 3.2). One quantization unit = G consecutive weights of a row. Per unit, in
+// fp32 with one rounding per operation (the precision the export kernel works in):
+//   lo = sb * min(W_r), hi = sg * max(W_r), h = hi - lo      (sb, sg: the sigmoids of beta, gamma)
+//   W_rc = clip(W_r, lo, hi)
+//   p1 = s1, p2 = (1 - p1) s2, p3 = (1 - p1)(1 - s2)         (s1, s2: the sigmoids of s_1, s_2)
+//   t1 = p1 / 2, t2 = t1 + (p1 + p2) / 2, t3 = t2 + (p2 + p3) / 2
+//   code = u(x - t1) + u(x - t2) + u(x - t3), x = (W_rc - lo) / h, u(z) = 1 for z >= 0 else 0
+//   w0 = 0, w1 = (t1 + t2) / 2, w2 = (t2 + t3) / 2, w3 = 1;  LUT_i = fp16(lo + h w_i)
+// Readings: the normalized weight is taken relative to the range minimum (Eq. "quant" prints W/h,
+// Eq. "dequant" offsets the levels by the minimum: only the offset form puts the thresholds
+// inside the range); the step function counts z = 0 as reached; a unit with h <= 0 gets code 0
+// everywhere and four levels equal to lo. The sigmoids are inputs (the caller evaluates them),
+// so that both sides work from identical fp32 numbers.
+// Inputs: w_f16 [N][K], sb, sg, s1, s2 float [N][K/G]. Outputs: codes u8 [N][K], lut fp16 bits
+// [N][K/G][4]. Returns 0, -1 bad shape.
+// ---------------------------------------------------------------------------------------
+int orc_ldp_export(const uint16_t* w_f16, const float* sb, const float* sg, const float* s1, const float* s2,
+                   int N, int K, int G, uint8_t* codes, uint16_t* lut_f16) {
+  if (N < 1 || K < 1 || G < 1 || K % G) return -1;
+  const int NG = K / G;
+  for (int n = 0; n < N; n++)
+    for (int j = 0; j < NG; j++) {
+      const uint16_t* w = w_f16 + (size_t)n * K + (size_t)j * G;
+      const size_t u = (size_t)n * NG + j;
+      float wmin = orc_f16_to_f32(w[0]), wmax = wmin;
+      for (int k = 1; k < G; k++) {
+        float v = orc_f16_to_f32(w[k]);
+        if (v < wmin) wmin = v;
+        if (v > wmax) wmax = v;
+      }
+      volatile float lo = sb[u] * wmin;
+      volatile float hi = sg[u] * wmax;
+      volatile float h = hi - lo;
+      volatile float p1 = s1[u];
+      volatile float rest = 1.0f - p1;
+      volatile float p2 = rest * s2[u];
+      volatile float one_m = 1.0f - s2[u];
+      volatile float p3 = rest * one_m;
+      volatile float t1 = p1 / 2.0f;
+      volatile float p12 = p1 + p2;
+      volatile float h12 = p12 / 2.0f;
+      volatile float t2 = t1 + h12;
+      volatile float p23 = p2 + p3;
+      volatile float h23 = p23 / 2.0f;
+      volatile float t3 = t2 + h23;
+      volatile float s12 = t1 + t2;
+      volatile float w1 = s12 / 2.0f;
+      volatile float s23 = t2 + t3;
+      volatile float w2 = s23 / 2.0f;
+      const float lv[4] = {0.0f, w1, w2, 1.0f};
+      const bool ok = h > 0.0f;
+      for (int c = 0; c < 4; c++) {
+        volatile float prod = h * lv[c];
+        volatile float level = lo + prod;
+        lut_f16[u * 4 + c] = orc_f32_to_f16(ok ? (float)level : (float)lo);
+      }
+      for (int k = 0; k < G; k++) {
+        int code = 0;
+        if (ok) {
+          float v = orc_f16_to_f32(w[k]);
+          if (v < lo) v = lo;
+          if (v > hi) v = hi;
+          volatile float d = v - lo;
+          volatile float x = d / h;
+          code = (x >= t1) + (x >= t2) + (x >= t3);
+        }
+        codes[(size_t)n * K + (size_t)j * G + k] = (uint8_t)code;
+      }
+    }
+  return 0;
 }
 
 }  // extern "C"

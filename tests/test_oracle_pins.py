@@ -1,5 +1,6 @@
 """Pins for the CPU oracle: every check here compares the oracle with something other than
 itself -- a library routine, a closed form, a hand-written fixture or a brute-force loop."""
+import fractions
 import itertools
 import os
 
@@ -469,3 +470,119 @@ def test_grouped_planted_mistakes_are_caught():
     assert not np.array_equal(r["S"], r_mod["S"])
     with pytest.raises((ValueError, AssertionError)):   # a group size that does not divide K
         oracle.gemv_w2a4_grouped(words, f16_bits(lut)[:, :3].copy(), qa["xq"], qa["scale"], 24)
+
+
+# ----------------------------------------------------------------------------- partitioning quantizer export
+def _ldp_inputs(N, K, G, seed, clip=True):
+    rng = np.random.default_rng(seed)
+    w = torch.from_numpy(rng.laplace(0.0, 0.02, size=(N, K)).astype(np.float32)).to(torch.float16)
+    NG = K // G
+    sig = lambda a: (1.0 / (1.0 + np.exp(-a))).astype(np.float32)
+    sb = sig(rng.normal(3.0, 1.0, size=(N, NG))) if clip else np.ones((N, NG), np.float32)
+    sg = sig(rng.normal(3.0, 1.0, size=(N, NG))) if clip else np.ones((N, NG), np.float32)
+    s1 = sig(rng.normal(-0.7, 0.5, size=(N, NG)))
+    s2 = sig(rng.normal(0.0, 0.5, size=(N, NG)))
+    return w, sb, sg, s1, s2
+
+
+def test_ldp_hand_case_from_fixture():
+    ws, codes, sig, lut = [], [], None, None
+    for ln in open(os.path.join(GOLD, "ldp_hand_case.txt")):
+        ln = ln.strip()
+        if not ln or ln.startswith("#"):
+            continue
+        if ln.startswith("sig"):
+            sig = [float(v) for v in ln.split()[1:]]
+        elif ln.startswith("lut"):
+            lut = [float(v) for v in ln.split()[1:]]
+        else:
+            a, b = ln.split("->")
+            ws.append(float(a))
+            codes.append(int(b))
+    G = 16
+    w = torch.tensor([ws + [0.5] * (G - len(ws))], dtype=torch.float16)
+    one = np.ones((1, 1), np.float32)
+    r = oracle.ldp_export(f16_bits(w), one, one, one * sig[0], one * sig[1], G)
+    assert list(r["codes"][0, :len(ws)]) == codes
+    assert list(r["lut"][0, 0].view(np.float16).astype(np.float64)) == lut
+
+
+def test_ldp_uniform_initial_point_is_the_textbook_asymmetric_quantizer():
+    # fixture: p = t = w at initialisation; then the quantizer is round((w - min) / (h / 3)) with levels min + h i / 3
+    fx = {}
+    for ln in open(os.path.join(GOLD, "ldp_uniform_init.txt")):
+        if ln.strip() and not ln.startswith("#"):
+            k, *v = ln.split()
+            fx[k] = [float(fractions.Fraction(x)) for x in v]
+    assert fx["t"] == [1 / 6, 1 / 2, 5 / 6] and fx["w"] == [0, 1 / 3, 2 / 3, 1]
+    N, K, G = 6, 512, 128
+    w, _, _, _, _ = _ldp_inputs(N, K, G, 1)
+    one = np.ones((N, K // G), np.float32)
+    r = oracle.ldp_export(f16_bits(w), one, one, (one / 3).astype(np.float32), (one / 2).astype(np.float32), G)
+    wf = w.numpy().astype(np.float64).reshape(N, K // G, G)
+    lo, hi = wf.min(axis=2, keepdims=True), wf.max(axis=2, keepdims=True)
+    xq = (wf - lo) / ((hi - lo) / 3.0)
+    ref = np.clip(np.rint(xq), 0, 3)
+    near_tie = np.abs(xq - np.floor(xq) - 0.5) < 1e-5
+    got = r["codes"].reshape(N, K // G, G)
+    assert near_tie.sum() < 5 and np.array_equal(got[~near_tie], ref[~near_tie].astype(np.uint8))
+    levels = lo + (hi - lo) * np.array(fx["w"])[None, None, :]
+    assert np.allclose(r["lut"].view(np.float16).astype(np.float64), levels, rtol=2e-3, atol=1e-7)
+
+
+def test_ldp_range_ends_bin_centres_monotone_codes_and_sum_form():
+    N, K, G = 5, 768, 128
+    w, sb, sg, s1, s2 = _ldp_inputs(N, K, G, 2)
+    r = oracle.ldp_export(f16_bits(w), sb, sg, s1, s2, G)
+    wf = w.numpy().astype(np.float64).reshape(N, K // G, G)
+    codes = r["codes"].reshape(N, K // G, G)
+    lut = r["lut"].view(np.float16).astype(np.float64)
+    lo = sb.astype(np.float64) * wf.min(axis=2)
+    hi = sg.astype(np.float64) * wf.max(axis=2)
+    h = hi - lo
+    # the lowest level is the clipped minimum, the highest the clipped maximum (lo + h = hi)
+    assert np.allclose(lut[..., 0], lo, rtol=1e-3, atol=1e-7) and np.allclose(lut[..., 3], hi, rtol=1e-3, atol=1e-7)
+    # partitions fill the range: the thresholds and the bin centres in exact arithmetic
+    p1 = s1.astype(np.float64)
+    p2 = (1 - p1) * s2
+    p3 = (1 - p1) * (1 - s2.astype(np.float64))
+    assert np.allclose(p1 + p2 + p3, 1.0)
+    t1 = p1 / 2
+    t2 = t1 + (p1 + p2) / 2
+    t3 = t2 + (p2 + p3) / 2
+    assert np.allclose(t3 + p3 / 2, 1.0)
+    assert np.allclose(lut[..., 1], lo + h * (t1 + t2) / 2, rtol=1e-3, atol=1e-7)
+    assert np.allclose(lut[..., 2], lo + h * (t2 + t3) / 2, rtol=1e-3, atol=1e-7)
+    # codes are monotone in the weight, and each weight sits in the partition its code names
+    x = (np.clip(wf, lo[..., None], hi[..., None]) - lo[..., None]) / h[..., None]
+    T = np.stack([np.zeros_like(t1) - 1, t1, t2, t3, np.ones_like(t1) * 2], axis=-1)
+    lower = np.take_along_axis(T, codes.astype(np.int64), axis=-1)
+    upper = np.take_along_axis(T, codes.astype(np.int64) + 1, axis=-1)
+    assert np.all(x >= lower - 1e-6) and np.all(x <= upper + 1e-6)
+    order = np.argsort(wf, axis=2, kind="stable")
+    assert np.all(np.diff(np.take_along_axis(codes.astype(np.int64), order, axis=2), axis=2) >= 0)
+    assert len(np.unique(codes)) == 4
+    # sum form of the dequantizer (three steps, each adding the gap to the next level) == LUT lookup
+    w0, w1, w2, w3 = 0.0, (t1 + t2) / 2, (t2 + t3) / 2, 1.0
+    u = lambda z: (z >= -1e-12).astype(np.float64)
+    dq = lo[..., None] + h[..., None] * (u(x - t1[..., None]) * (w1 - w0)[..., None] + u(x - t2[..., None]) * (w2 - w1)[..., None]
+                                         + u(x - t3[..., None]) * (w3 - w2)[..., None])
+    interior = (np.abs(x - t1[..., None]) > 1e-5) & (np.abs(x - t2[..., None]) > 1e-5) & (np.abs(x - t3[..., None]) > 1e-5)
+    look = np.take_along_axis(lut, codes.astype(np.int64), axis=-1)
+    assert np.allclose(dq[interior], look[interior], rtol=2e-3, atol=1e-6)
+
+
+def test_ldp_degenerate_unit_and_planted_mistakes():
+    G = 32
+    w = torch.full((1, 2 * G), 0.25, dtype=torch.float16)
+    w[0, G:] = torch.linspace(-1, 1, G).to(torch.float16)
+    one = np.ones((1, 2), np.float32)
+    r = oracle.ldp_export(f16_bits(w), one, one, one * 0.3, one * 0.6, G)
+    assert np.all(r["codes"][0, :G] == 0) and np.all(r["lut"][0, 0].view(np.float16) == np.float16(0.25))
+    # swapping the two partition parameters, or the two clipping parameters, changes the second unit
+    a = oracle.ldp_export(f16_bits(w), one * 0.9, one * 0.7, one * 0.3, one * 0.6, G)
+    b = oracle.ldp_export(f16_bits(w), one * 0.9, one * 0.7, one * 0.6, one * 0.3, G)
+    c = oracle.ldp_export(f16_bits(w), one * 0.7, one * 0.9, one * 0.3, one * 0.6, G)
+    assert not np.array_equal(a["codes"], b["codes"]) and not np.array_equal(a["lut"], c["lut"])
+    with pytest.raises((ValueError, AssertionError)):
+        oracle.ldp_export(f16_bits(w), one, one, one, one, 48)
