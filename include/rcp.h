@@ -130,6 +130,30 @@ int rcp_gemv_w2a4_variant(int variant, const uint32_t* words, const void* lut_f1
                           void* y_f16, void* workspace, int32_t* S_dbg, void* stream);
 
 /*
+ * Export of a layer trained with learnable direct partitioning to the GEMV's inputs: 2-bit codes,
+ * packed, and the four-entry grid of every quantization unit (Section 3.3: Eq. "partition", the
+ * equation for t_i, Eq. "quant", Eq. "dequantgrid"; Section 3.4, Eq. "deqgrid"; clipping range of
+ * Section 3.2). Offline, like rcp_pack_weights. A unit is `group` consecutive weights of a row:
+ *   lo = sig_beta * min(W), hi = sig_gamma * max(W), h = hi - lo, W clipped to [lo, hi];
+ *   p1 = sig_s1, p2 = (1 - p1) sig_s2, p3 = (1 - p1)(1 - sig_s2);
+ *   t1 = p1/2, t2 = t1 + (p1 + p2)/2, t3 = t2 + (p2 + p3)/2;
+ *   code = number of thresholds t_i that (W - lo)/h has reached (equal counts as reached);
+ *   levels lo + h * {0, (t1 + t2)/2, (t2 + t3)/2, 1}, rounded to fp16.
+ * fp32 arithmetic, one rounding per operation. A unit with h <= 0 gets code 0 and four levels lo.
+ *   w_f16      DEVICE fp16 [N][K], the rotated weights; 16-byte aligned.
+ *   sig_*      DEVICE float [N][K/group]: the sigmoids of beta, gamma, s_1, s_2, evaluated by the
+ *              caller (so that the 2-bit decision does not depend on an exponential's last bit).
+ *   group      a multiple of 16 dividing K (K for one grid per row).
+ *   words      DEVICE uint32 [N][K/16] (the format of rcp_pack_weights);
+ *   lut_f16    DEVICE fp16 [N][K/group][4] (the lut of rcp_gemv_w2a4_grouped; of rcp_gemv_w2a4 when
+ *              group == K).
+ * Never synchronizes.
+ */
+int rcp_ldp_export(const void* w_f16, const float* sig_beta, const float* sig_gamma,
+                   const float* sig_s1, const float* sig_s2, int N, int K, int group,
+                   uint32_t* words, void* lut_f16, void* stream);
+
+/*
  * LUT GEMV with one grid per group of weights (Section 4.4: the dequantization grid has shape
  * H x N*4 for N groups per row; Appendix A.1: C = N*G; the table of quantization configurations
  * sets the weight group size G = 128). Weight k of row n takes its levels from lut[n][k / group]:

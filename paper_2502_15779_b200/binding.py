@@ -51,6 +51,8 @@ def lib():
         L.rcp_gemv_w2a4_grouped.argtypes = [vp, vp, i, vp, vp, i, i, i, vp, vp, vp, vp]
         L.rcp_gemv_w2a4_grouped_variant.restype = i
         L.rcp_gemv_w2a4_grouped_variant.argtypes = [i, vp, vp, i, vp, vp, i, i, i, vp, vp, vp, vp]
+        L.rcp_ldp_export.restype = i
+        L.rcp_ldp_export.argtypes = [vp, vp, vp, vp, vp, i, i, i, vp, vp, vp]
         L.rcp_linear_w2a4.restype = i
         L.rcp_linear_w2a4.argtypes = [vp, i, i, i, C.c_float, vp, vp, i, i, vp, vp, vp, vp, vp]
         L.rcp_linear_w2a4_launches.restype = i
@@ -91,6 +93,25 @@ def rcp_pack_weights(codes: torch.Tensor, out: torch.Tensor = None) -> torch.Ten
     with torch.cuda.device(codes.device):
         _check("rcp_pack_weights", lib().rcp_pack_weights(_ptr(codes), N, K, _ptr(words), _stream(codes)))
     return words
+
+
+def rcp_ldp_export(w, sig_beta, sig_gamma, sig_s1, sig_s2, group):
+    """Rotated weights fp16 [N][K] and the sigmoids of the clipping and partition parameters (float32
+    [N][K/group]) -> (words int32 [N][K/16], lut fp16 [N][K/group][4])."""
+    _dev(w, torch.float16, "w")
+    N, K = w.shape
+    group = int(group)
+    for name, a in (("sig_beta", sig_beta), ("sig_gamma", sig_gamma), ("sig_s1", sig_s1), ("sig_s2", sig_s2)):
+        _dev(a, torch.float32, name)
+        if group < 1 or K % group or tuple(a.shape) != (N, K // group):
+            raise ValueError(f"{name}: expected shape [N][K/group]")
+    words = torch.empty((N, K // 16), dtype=torch.int32, device=w.device)
+    lut = torch.empty((N, K // group, 4), dtype=torch.float16, device=w.device)
+    with torch.cuda.device(w.device):
+        _check("rcp_ldp_export",
+               lib().rcp_ldp_export(_ptr(w), _ptr(sig_beta), _ptr(sig_gamma), _ptr(sig_s1), _ptr(sig_s2), N, K, group,
+                                    _ptr(words), _ptr(lut), _stream(w)))
+    return words, lut
 
 
 def rcp_quantize_act(x: torch.Tensor, had_block: int, clip_ratio: float = 1.0, xq=None, scale=None):

@@ -9,6 +9,7 @@
 #include "common.cuh"
 #include "gemv_simple.cuh"
 #include "gemv_stream.cuh"
+#include "ldp_export.cuh"
 #include "pack.cuh"
 #include "quantize_act.cuh"
 
@@ -346,6 +347,29 @@ int rcp_pack_weights(const uint8_t* codes, int N, int K, uint32_t* words, void* 
   RCP_CUDA(cudaMemcpyAsync(&h_bad, bad, sizeof(int), cudaMemcpyDeviceToHost, st));
   RCP_CUDA(cudaStreamSynchronize(st));
   return h_bad ? RCP_ERR_CODE : RCP_OK;
+}
+
+int rcp_ldp_export(const void* w_f16, const float* sig_beta, const float* sig_gamma, const float* sig_s1,
+                   const float* sig_s2, int N, int K, int group, uint32_t* words, void* lut_f16, void* stream) {
+  if (!w_f16 || !sig_beta || !sig_gamma || !sig_s1 || !sig_s2 || !words || !lut_f16) return RCP_ERR_NULL;
+  if (N < 1 || !k_ok(K) || group < 16 || group % 16 || K % group) return RCP_ERR_SHAPE;
+  if (!aligned16(w_f16) || !aligned16(words) || (reinterpret_cast<uintptr_t>(lut_f16) & 7u) ||
+      (reinterpret_cast<uintptr_t>(sig_beta) & 3u) || (reinterpret_cast<uintptr_t>(sig_gamma) & 3u) ||
+      (reinterpret_cast<uintptr_t>(sig_s1) & 3u) || (reinterpret_cast<uintptr_t>(sig_s2) & 3u))
+    return RCP_ERR_ALIGN;
+  rcp::LdpParams lp;
+  lp.w = static_cast<const __half*>(w_f16);
+  lp.sb = sig_beta; lp.sg = sig_gamma; lp.s1 = sig_s1; lp.s2 = sig_s2;
+  lp.words = words;
+  lp.lut = static_cast<uint2*>(lut_f16);
+  lp.N = N; lp.K = K; lp.G = group;
+  lp.units = (long long)N * (K / group);
+  const int block = 256;
+  const long long want = (lp.units + (block / 32) - 1) / (block / 32);
+  const int grid = (int)std::min<long long>(want, (long long)sm_count() * 16);
+  rcp::ldp_export_kernel<<<grid, block, 0, static_cast<cudaStream_t>(stream)>>>(lp);
+  RCP_CUDA(cudaGetLastError());
+  return RCP_OK;
 }
 
 int rcp_quantize_act(const void* x_f16, int M, int K, int had_block, float clip_ratio, uint8_t* xq,

@@ -1,0 +1,88 @@
+"""GPU parity of rcp_ldp_export (partitioning quantizer -> packed codes and grids) against the CPU oracle:
+codes and fp16 levels bit for bit; and the exported layer through the GEMV against the oracle's GEMV."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2502_15779_b200 as rcp
+from paper_2502_15779_b200 import synth
+from helpers import f16_bits
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _inputs(N, K, G, seed):
+    g = torch.Generator(device="cpu")
+    g.manual_seed(seed)
+    u = torch.rand(N, K, generator=g, dtype=torch.float64) - 0.5
+    w = (-0.02 * torch.sign(u) * torch.log1p(-2.0 * u.abs())).to(torch.float16)   # Laplace(0, 0.02)
+    NG = K // G
+    sb = torch.sigmoid(3.0 + torch.randn(N, NG, generator=g)).float()
+    sg = torch.sigmoid(3.0 + torch.randn(N, NG, generator=g)).float()
+    s1 = torch.sigmoid(-0.7 + 0.5 * torch.randn(N, NG, generator=g)).float()
+    s2 = torch.sigmoid(0.5 * torch.randn(N, NG, generator=g)).float()
+    return w, sb, sg, s1, s2
+
+
+@pytest.mark.parametrize("N,K,G", [(1, 64, 16), (5, 128, 128), (33, 1024, 128), (17, 11008, 128), (64, 4096, 4096),
+                                   (9, 2048, 64), (300, 512, 256), (3, 28672, 128), (2, 8192, 8192), (40, 384, 48)])
+def test_ldp_export_bit_exact(N, K, G):
+    w, sb, sg, s1, s2 = _inputs(N, K, G, N + K + G)
+    if N > 2:
+        w[1, :G] = 0.125            # a unit without range: code 0, four equal levels
+        w[2, :G] = w[2, :G].abs()   # a unit whose minimum is positive
+    ref = oracle.ldp_export(f16_bits(w), sb.numpy(), sg.numpy(), s1.numpy(), s2.numpy(), G)
+    words, lut = rcp.rcp_ldp_export(w.to(DEV), sb.to(DEV), sg.to(DEV), s1.to(DEV), s2.to(DEV), G)
+    assert np.array_equal(words.cpu().numpy().view(np.uint32), oracle.pack_weights(ref["codes"]))
+    assert np.array_equal(f16_bits(lut), ref["lut"])
+    assert len(np.unique(ref["codes"])) == 4
+
+
+def test_ldp_export_at_the_uniform_initial_point_and_exact_thresholds():
+    # weights on a grid of sixteenths over [0, 1], sigmoids 1/2: thresholds 1/4, 5/8, 7/8 are hit exactly
+    G = 32
+    w = (torch.arange(G, dtype=torch.float32) / 16.0).clamp(max=1.0).to(torch.float16)[None, :].repeat(2, 2).contiguous()
+    half = torch.full((2, 2), 0.5, dtype=torch.float32)
+    one = torch.ones(2, 2, dtype=torch.float32)
+    ref = oracle.ldp_export(f16_bits(w), one.numpy(), one.numpy(), half.numpy(), half.numpy(), G)
+    words, lut = rcp.rcp_ldp_export(w.to(DEV), one.to(DEV), one.to(DEV), half.to(DEV), half.to(DEV), G)
+    assert np.array_equal(words.cpu().numpy().view(np.uint32), oracle.pack_weights(ref["codes"]))
+    assert list(ref["codes"][0, :17]) == [0, 0, 0, 0, 1, 1, 1, 1, 1, 1, 2, 2, 2, 2, 3, 3, 3]
+    assert lut[0, 0].tolist() == [0.0, 0.4375, 0.75, 1.0]
+
+
+@pytest.mark.parametrize("N,K,G,M", [(200, 1024, 128, 1), (300, 4096, 128, 3), (150, 2048, 2048, 2)])
+def test_exported_layer_through_the_gemv(N, K, G, M):
+    w, sb, sg, s1, s2 = _inputs(N, K, G, 7 * N + M)
+    words, lut = rcp.rcp_ldp_export(w.to(DEV), sb.to(DEV), sg.to(DEV), s1.to(DEV), s2.to(DEV), G)
+    x = synth.make_activations(M, K, 11, device=DEV)
+    B = 128
+    xq, scale = rcp.rcp_quantize_act(x, B, 1.0)
+    ref_q = oracle.ldp_export(f16_bits(w), sb.numpy(), sg.numpy(), s1.numpy(), s2.numpy(), G)
+    qa = oracle.quantize_act(f16_bits(x), B, 1.0)
+    w_ref = oracle.pack_weights(ref_q["codes"])
+    if G == K:
+        y = rcp.rcp_gemv_w2a4(words, lut.reshape(N, 4).contiguous(), xq, scale)
+        ref = oracle.gemv_w2a4(w_ref, ref_q["lut"].reshape(N, 4), qa["xq"], qa["scale"])
+    else:
+        y = rcp.rcp_gemv_w2a4_grouped(words, lut, xq, scale, group=G)
+        ref = oracle.gemv_w2a4_grouped(w_ref, ref_q["lut"], qa["xq"], qa["scale"], G)
+    got = y.float().cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(got - ref["y"]) <= ref["tol"])
+    # sanity: the 2-bit layer (untrained partition parameters) still follows the full-precision product
+    full = (qa["q"].astype(np.float64) * qa["scale"].view(np.float16).astype(np.float64)[:, None]) @ w.numpy().astype(np.float64).T
+    assert np.corrcoef(got.ravel(), full.ravel())[0, 1] > 0.6
+
+
+def test_ldp_export_argument_errors():
+    L = rcp.lib()
+    z = torch.zeros(4096, dtype=torch.int32, device=DEV)
+    p = z.data_ptr()
+    f = L.rcp_ldp_export
+    assert f(None, p, p, p, p, 4, 128, 128, p, p, None) == -1
+    assert f(p, p, p, p, p, 0, 128, 128, p, p, None) == -2
+    assert f(p, p, p, p, p, 4, 128, 48, p, p, None) == -2      # group does not divide K
+    assert f(p, p, p, p, p, 4, 128, 8, p, p, None) == -2       # group below 16
+    assert f(p + 2, p, p, p, p, 4, 128, 128, p, p, None) == -3
