@@ -481,12 +481,13 @@ def main():
                               "frac": round(p_ach / peaks["hbm_gbs"], 4),
                               "note": "rcp_gemv_w2a4 launches alone, activations quantized beforehand"}
     del pgraphs
-    prof = os.path.join(ROOT, "profiles", "traffic.json")
+    # DRAM bytes per launch from the committed ncu summary (null when there is none for this workload)
+    prof = os.path.join(ROOT, "profiles", "dram_traffic.txt")
     if os.path.exists(prof):
-        try:
-            roofline["traffic"] = json.load(open(prof)).get(f"{cfg.key}_M{M}")
-        except Exception:
-            pass
+        for ln in open(prof):
+            parts = ln.split()
+            if len(parts) == 2 and parts[0] == f"{cfg.key}_M{M}_{args.variant}":
+                roofline["traffic"] = int(parts[1])
 
     # ---- end to end through the C ABI with host buffers
     xh = [layer.x[li].cpu().pin_memory() for li in range(len(layer.layers))]
