@@ -38,6 +38,7 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include "quantize_act.cuh"
 
 namespace rcp {
 
@@ -258,94 +259,10 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     float* const qbuf = reinterpret_cast<float*>(gen + p.off_qbuf);   // [16][W]
     float* const s_amax = s_scale + 8;                                // [16 warps] behind the scales
     float v[16];
-    if (tid < W) {
-      const uint4* src = reinterpret_cast<const uint4*>(p.x + (size_t)tid * 16);
-      const uint4 r0 = __ldg(src), r1 = __ldg(src + 1);
-      const __half2* h0 = reinterpret_cast<const __half2*>(&r0);
-      const __half2* h1 = reinterpret_cast<const __half2*>(&r1);
-#pragma unroll
-      for (int e = 0; e < 4; e++) {
-        const float2 f0 = __half22float2(h0[e]), f1 = __half22float2(h1[e]);
-        v[2 * e] = f0.x; v[2 * e + 1] = f0.y; v[8 + 2 * e] = f1.x; v[8 + 2 * e + 1] = f1.y;
-      }
-    } else {
-#pragma unroll
-      for (int e = 0; e < 16; e++) v[e] = 0.f;
-    }
-    // strides 1 .. 8: inside the word
-#pragma unroll
-    for (int h = 1; h < 16; h *= 2) {
-#pragma unroll
-      for (int e = 0; e < 16; e++) {
-        if ((e & h) == 0) {
-          const float u = v[e], w = v[e + h];
-          v[e] = __fadd_rn(u, w);
-          v[e + h] = __fsub_rn(u, w);
-        }
-      }
-    }
-    // strides 16 .. 256: element stride 16 d <-> lane distance d
-#pragma unroll
-    for (int d = 1; d < 32; d *= 2) {
-      const bool upper = (lane & d) != 0;
-#pragma unroll
-      for (int e = 0; e < 16; e++) {
-        const float other = __shfl_xor_sync(0xffffffffu, v[e], d);
-        v[e] = upper ? __fsub_rn(other, v[e]) : __fadd_rn(v[e], other);
-      }
-    }
-    // strides 512 .. K/2: across the R = W / 32 warps that hold data, through shared memory; thread
-    // (element tid >> 5, lane) takes the R values of its column, 32 words apart
-    {
-      if (tid < W) {
-#pragma unroll
-        for (int e = 0; e < 16; e++) qbuf[e * W + tid] = v[e];
-      }
-      asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");
-      const int R = W >> 5;   // 8 or 16
-      float* const colp = qbuf + (tid >> 5) * W + lane;
-      float tv[16];
-#pragma unroll
-      for (int w = 0; w < 16; w++) tv[w] = (w < R) ? colp[w * 32] : 0.f;
-#pragma unroll
-      for (int h = 1; h < 16; h *= 2) {
-        if (h < R) {
-#pragma unroll
-          for (int w = 0; w < 16; w++) {
-            if ((w & h) == 0) {
-              const float u = tv[w], z = tv[w + h];
-              tv[w] = __fadd_rn(u, z);
-              tv[w + h] = __fsub_rn(u, z);
-            }
-          }
-        }
-      }
-#pragma unroll
-      for (int w = 0; w < 16; w++) if (w < R) colp[w * 32] = tv[w];
-      asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");
-      if (tid < W) {
-#pragma unroll
-        for (int e = 0; e < 16; e++) v[e] = qbuf[e * W + tid];
-      }
-    }
-    float amax = 0.f;
-#pragma unroll
-    for (int e = 0; e < 16; e++) {
-      v[e] = __fmul_rn(v[e], p.inv_sqrt_b);
-      amax = fmaxf(amax, fabsf(v[e]));
-    }
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, d));
-    if (lane == 0) s_amax[warp] = amax;
-    asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");
-#pragma unroll
-    for (int w = 0; w < kCWarps; w++) amax = fmaxf(amax, s_amax[w]);
-    const float s32 = __fdiv_rn(__fmul_rn(amax, p.clip_ratio), 7.0f);
-    const __half s16 = __float2half_rn(s32);
-    const float sc = __half2float(s16);
+    const float sc = rotate_token_words<NT>(p.x, W, p.inv_sqrt_b, p.clip_ratio, qbuf, s_amax, v);
     if (tid == 0) {
       s_scale[0] = sc;
-      if (b == 0 && p.scale_out) p.scale_out[0] = s16;
+      if (b == 0 && p.scale_out) p.scale_out[0] = __float2half_rn(sc);
     }
     int q[16];
     int tsum = 0;

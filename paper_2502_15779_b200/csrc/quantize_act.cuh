@@ -256,4 +256,126 @@ __global__ void __launch_bounds__(1024) quantize_act_kernel(const QuantParams p)
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// One token of W = K / 16 words (256 or 512) under a single rotation block, by NT = 512 threads of one
+// CTA: thread tid holds word tid (16 consecutive activations). Strides 1..8 inside the word, 16..256
+// by lane exchanges, 512 and up through shared memory (thread (element tid >> 5, lane) takes the
+// R = W / 32 values of its column, 32 words apart), then the scale by 1/sqrt(K) and the token's
+// absmax. Same operations in the same order as quantize_act_kernel. Leaves the rotated, scaled
+// activations of the thread's word in v and returns the quantization scale (as rounded to fp16).
+// Uses named barrier 1 with NT threads; qbuf: 16 * W floats, s_amax: NT / 32 floats.
+template <int NT>
+__device__ __forceinline__ float rotate_token_words(const __half* x, int W, float inv_sqrt_b, float clip_ratio,
+                                                    float* qbuf, float* s_amax, float (&v)[16]) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid < W) {
+    const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)tid * 16);
+    const uint4 r0 = __ldg(src), r1 = __ldg(src + 1);
+    const __half2* h0 = reinterpret_cast<const __half2*>(&r0);
+    const __half2* h1 = reinterpret_cast<const __half2*>(&r1);
+#pragma unroll
+    for (int e = 0; e < 4; e++) {
+      const float2 f0 = __half22float2(h0[e]), f1 = __half22float2(h1[e]);
+      v[2 * e] = f0.x; v[2 * e + 1] = f0.y; v[8 + 2 * e] = f1.x; v[8 + 2 * e + 1] = f1.y;
+    }
+  } else {
+#pragma unroll
+    for (int e = 0; e < 16; e++) v[e] = 0.f;
+  }
+#pragma unroll
+  for (int h = 1; h < 16; h *= 2) {
+#pragma unroll
+    for (int e = 0; e < 16; e++) {
+      if ((e & h) == 0) {
+        const float u = v[e], w = v[e + h];
+        v[e] = __fadd_rn(u, w);
+        v[e + h] = __fsub_rn(u, w);
+      }
+    }
+  }
+#pragma unroll
+  for (int d = 1; d < 32; d *= 2) {   // element stride 16 d <-> lane distance d
+    const bool upper = (lane & d) != 0;
+#pragma unroll
+    for (int e = 0; e < 16; e++) {
+      const float other = __shfl_xor_sync(0xffffffffu, v[e], d);
+      v[e] = upper ? __fsub_rn(other, v[e]) : __fadd_rn(v[e], other);
+    }
+  }
+  if (tid < W) {
+#pragma unroll
+    for (int e = 0; e < 16; e++) qbuf[e * W + tid] = v[e];
+  }
+  asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");
+  {
+    const int R = W >> 5;   // 8 or 16 warps hold data
+    float* const colp = qbuf + warp * W + lane;
+    float tv[16];
+#pragma unroll
+    for (int w = 0; w < 16; w++) tv[w] = (w < R) ? colp[w * 32] : 0.f;
+#pragma unroll
+    for (int h = 1; h < 16; h *= 2) {
+      if (h < R) {
+#pragma unroll
+        for (int w = 0; w < 16; w++) {
+          if ((w & h) == 0) {
+            const float u = tv[w], z = tv[w + h];
+            tv[w] = __fadd_rn(u, z);
+            tv[w + h] = __fsub_rn(u, z);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int w = 0; w < 16; w++) if (w < R) colp[w * 32] = tv[w];
+  }
+  asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");
+  if (tid < W) {
+#pragma unroll
+    for (int e = 0; e < 16; e++) v[e] = qbuf[e * W + tid];
+  }
+  float amax = 0.f;
+#pragma unroll
+  for (int e = 0; e < 16; e++) {
+    v[e] = __fmul_rn(v[e], inv_sqrt_b);
+    amax = fmaxf(amax, fabsf(v[e]));
+  }
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, d));
+  if (lane == 0) s_amax[warp] = amax;
+  asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");
+#pragma unroll
+  for (int w = 0; w < NT / 32; w++) amax = fmaxf(amax, s_amax[w]);
+  const float s32 = __fdiv_rn(__fmul_rn(amax, clip_ratio), 7.0f);
+  return __half2float(__float2half_rn(s32));
+}
+
+// One CTA of 512 threads per token, for a token of 4096 or 8192 elements under one rotation block:
+// faster than the cluster form above for these shapes (no cluster launch, no passes through
+// distributed shared memory).
+__global__ void __launch_bounds__(512) quantize_act_wide_kernel(const QuantParams p) {
+  extern __shared__ float sbuf[];   // 16 * W floats
+  __shared__ float s_amax[16];
+  const int m = blockIdx.x, tid = threadIdx.x;
+  asm volatile("griddepcontrol.launch_dependents;");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int W = p.K / 16;
+  float v[16];
+  const float s = rotate_token_words<512>(p.x + (size_t)m * p.K, W, p.inv_sqrt_b, p.clip_ratio, sbuf, s_amax, v);
+  if (tid == 0) p.scale[m] = __float2half_rn(s);
+  if (tid < W) {
+    uint32_t lo32 = 0, hi32 = 0;
+    if (s != 0.f) {
+#pragma unroll
+      for (int e = 0; e < 8; e++) {
+        const int q0 = max(-8, min(7, __float2int_rn(__fdiv_rn(v[e], s))));
+        const int q1 = max(-8, min(7, __float2int_rn(__fdiv_rn(v[8 + e], s))));
+        lo32 |= (uint32_t)(q0 & 0xF) << (4 * e);
+        hi32 |= (uint32_t)(q1 & 0xF) << (4 * e);
+      }
+    }
+    *reinterpret_cast<uint2*>(p.xq + (size_t)m * (p.K / 2) + (size_t)tid * 8) = make_uint2(lo32, hi32);
+  }
+}
+
 }  // namespace rcp

@@ -392,6 +392,12 @@ int rcp_quantize_act(const void* x_f16, int M, int K, int had_block, float clip_
   while ((1 << qp.lgB) < B) qp.lgB++;
   qp.inv_sqrt_b = (float)(1.0 / std::sqrt((double)B));
   qp.clip_ratio = clip_ratio;
+  if (B == K && (K == 4096 || K == 8192)) {
+    // one rotation block over a long token: one CTA of 512 threads per token (measured faster than a cluster)
+    qp.cross = 1; qp.slice = 0; qp.unit = K; qp.nunits = 1; qp.lg_local = qp.lgB;
+    RCP_CUDA(launch_overlapped(rcp::quantize_act_wide_kernel, dim3((unsigned)M), dim3(512), (size_t)4 * K, st, qp));
+    return RCP_OK;
+  }
   int C = 1;
   while (C < 8 && K / (2 * C) >= 2048) C *= 2;
   int T;
