@@ -1,0 +1,69 @@
+"""Seeded random sweep of shapes through every GEMV entry point against the CPU oracle: row counts around
+the tile and phase boundaries of the streaming kernel, K any multiple of 64 (128 with the group-wise grid),
+1 to 16 tokens, every kernel variant."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2502_15779_b200 as rcp
+from paper_2502_15779_b200 import synth
+from helpers import f16_bits
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _cases(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        # rows: small, around one tile (256), around a round of 148 x 256 rows, and in between
+        N = int(rng.choice([rng.integers(1, 40), rng.integers(200, 300), rng.integers(2300, 2450),
+                            rng.integers(37800, 38000), rng.integers(1, 6000)]))
+        if N > 30000:
+            K = 64 * int(rng.integers(1, 9))
+        else:
+            K = 64 * int(rng.choice([rng.integers(1, 20), rng.integers(20, 180), 128, 172, 224, 448]))
+        M = int(rng.choice([1, 1, 2, 3, 5, 8, 9, 16]))
+        variant = str(rng.choice(["auto", "dp4a", "mma", "mma_only", "simple"]))
+        grouped = bool(rng.integers(0, 2)) and K % 128 == 0
+        if grouped and variant == "mma":
+            variant = "mma_only"
+        out.append(pytest.param(N, K, M, variant, grouped, i, id=f"{i}-N{N}-K{K}-M{M}-{variant}{'-g' if grouped else ''}"))
+    return out
+
+
+@pytest.mark.parametrize("N,K,M,variant,grouped,i", _cases(48, 20250215))
+def test_random_shape(N, K, M, variant, grouped, i):
+    B = 64 if K % 128 else int(np.random.default_rng(i).choice([1, 64, 128]))
+    seed = 5000 + i
+    if grouped:
+        codes, lut = synth.make_layer_grouped(N, K, 128, B, "uniform", seed, device=DEV)
+    else:
+        codes, lut = synth.make_layer(N, K, B, "uniform", seed, device=DEV)
+    x = synth.make_activations(M, K, seed, device=DEV)
+    words = rcp.rcp_pack_weights(codes)
+    xq, scale = rcp.rcp_quantize_act(x, B, 1.0)
+    ws = rcp.make_workspace(M, N, K, DEV)
+    if grouped:
+        y = rcp.rcp_gemv_w2a4_grouped(words, lut, xq, scale, group=128, workspace=ws, variant=variant)
+    else:
+        y = rcp.rcp_gemv_w2a4(words, lut, xq, scale, workspace=ws, variant=variant)
+    y_lin = rcp.rcp_linear_w2a4(x, B, 1.0, words, lut, group=128 if grouped else 0, xq=torch.empty_like(xq),
+                                scale=torch.empty_like(scale), workspace=ws)
+    torch.cuda.synchronize()
+    assert int(ws.abs().max()) == 0
+    rows = np.arange(N) if N * K * M <= 1 << 24 else np.unique(np.concatenate(
+        [np.arange(64), np.arange(N - 64, N), np.random.default_rng(i).integers(0, N, size=256)]))
+    qa = oracle.quantize_act(f16_bits(x), B, 1.0)
+    assert np.array_equal(xq.cpu().numpy(), qa["xq"]) and np.array_equal(f16_bits(scale), qa["scale"])
+    w_ref = oracle.pack_weights(codes.cpu().numpy()[rows])
+    assert np.array_equal(words.cpu().numpy().view(np.uint32)[rows], w_ref)
+    lb = np.ascontiguousarray(f16_bits(lut)[rows])
+    ref = (oracle.gemv_w2a4_grouped(w_ref, lb, qa["xq"], qa["scale"], 128) if grouped
+           else oracle.gemv_w2a4(w_ref, lb, qa["xq"], qa["scale"]))
+    for out in (y, y_lin):
+        got = out.float().cpu().numpy().astype(np.float64)[:, rows]
+        assert np.all(np.isfinite(got))
+        assert np.all(np.abs(got - ref["y"]) <= ref["tol"])
