@@ -341,6 +341,19 @@ class OracleSample:
         return self.nbytes / secs / 1e9, secs
 
 
+def host_cpu():
+    """Model name and logical core count of the host the oracle is timed on."""
+    model = "unknown"
+    try:
+        for ln in open("/proc/cpuinfo"):
+            if ln.lower().startswith("model name"):
+                model = ln.split(":", 1)[1].strip()
+                break
+    except OSError:
+        pass
+    return {"cpu_model": model, "nproc": os.cpu_count()}
+
+
 def run_reference(args, cfg, M):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -358,7 +371,8 @@ def run_reference(args, cfg, M):
            "warmup": args.warmup, "ms_per_step": 1e3 * statistics.mean(secs), "higher_is_better": True,
            "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
            "config": {"workload": workload_name(cfg, M), "note": "CPU oracle on a bounded sample of each step"},
-           "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample.desc},
+           "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample.desc,
+                            **host_cpu()},
            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0}
     print(json.dumps(out), flush=True)
@@ -557,7 +571,7 @@ def main():
         sample = OracleSample(cfg, M, args.sample_seconds)
         v, secs = sample.run()
         cpu = {"value": round(v, 4), "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample.desc,
-               "seconds": round(secs, 2)}
+               "seconds": round(secs, 2), **host_cpu()}
 
     out = {"metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
            "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True, "scaling": "weak",
