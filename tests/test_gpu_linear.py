@@ -114,3 +114,31 @@ def test_linear_full_size_configs_sampled_rows(ci, N, K, B):
     rows = np.unique(np.concatenate([np.arange(min(N, 32)), np.arange(max(0, N - 32), N),
                                      rng.integers(0, N, size=min(N, 128))]))
     _check(N, K, B, 1, 0, 1.0, seed=3000 + ci, rows=rows)
+
+
+@pytest.mark.parametrize("pinned", [True, False])
+@pytest.mark.parametrize("N,K,B,M", [(300, 8192, 8192, 1), (200, 4096, 128, 1), (150, 11008, 128, 2), (64, 2048, 2048, 3)])
+def test_linear_host_buffers(N, K, B, M, pinned):
+    """rcp_linear_w2a4_host: activations from and results to host memory (pinned or pageable), twice with
+    different activations in the same buffers (no stale data between calls)."""
+    codes, lut = synth.make_layer(N, K, B, "uniform", N + K, device=DEV)
+    words = rcp.rcp_pack_weights(codes)
+    xh = torch.empty(M, K, dtype=torch.float16)
+    yh = torch.empty(M, N, dtype=torch.float16)
+    if pinned:
+        xh, yh = xh.pin_memory(), yh.pin_memory()
+    x_dev = torch.empty(M, K, dtype=torch.float16, device=DEV)
+    xq = torch.empty(M, K // 2, dtype=torch.uint8, device=DEV)
+    scale = torch.empty(M, dtype=torch.float16, device=DEV)
+    y_dev = torch.empty(M, N, dtype=torch.float16, device=DEV)
+    ws = rcp.make_workspace(M, N, K, DEV)
+    w_ref = oracle.pack_weights(codes.cpu().numpy())
+    for rep in range(2):
+        xh.copy_(synth.make_activations(M, K, 100 + rep))
+        yh.fill_(float("nan"))
+        rcp.rcp_linear_w2a4_host(xh, B, 1.0, words, lut, yh, x_dev, xq, scale, y_dev, ws)
+        torch.cuda.synchronize()
+        qa = oracle.quantize_act(f16_bits(xh), B, 1.0)
+        ref = oracle.gemv_w2a4(w_ref, f16_bits(lut), qa["xq"], qa["scale"])
+        got = yh.float().numpy().astype(np.float64)
+        assert np.all(np.isfinite(got)) and np.all(np.abs(got - ref["y"]) <= ref["tol"])
