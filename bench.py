@@ -537,6 +537,8 @@ def main():
     e2e_ms_per_step, e2e_value, _ = replica_metrics(e2e_ms, step_bytes, e2e_steps, dist, device)
     e2e = {"value": round(e2e_value, 2), "unit": UNIT,
            "ms_per_step": round(e2e_ms_per_step, 4),
+           "transfer": "rcp_linear_w2a4_host on pinned buffers: the quantizer reads x from host memory and the GEMV "
+                       "stores y into it directly (no staging copy); the host waits for the stream after every step",
            "h2d_bytes_per_step": sum(2 * M * L.K for L in layer.layers),
            "d2h_bytes_per_step": sum(2 * M * L.N for L in layer.layers)}
 

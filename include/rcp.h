@@ -203,7 +203,9 @@ int rcp_linear_w2a4_launches(int M, int K, int had_block, int group);
  * One decode linear layer end to end with HOST activations (Section 4.4 data path: rotate and
  * quantize the token, then the LUT GEMV): copies x from host memory, runs rcp_linear_w2a4
  * (per-row grid), copies y back. All on `stream`, no synchronization: y_host is valid after the
- * caller synchronizes the stream. Pinned host memory makes the copies asynchronous.
+ * caller synchronizes the stream. Page-locked (pinned) host buffers are used in place: the quantizer
+ * reads x and the GEMV stores y directly in host memory, no copy is made and the staging buffers
+ * x_dev / y_dev stay untouched; pageable buffers go through cudaMemcpyAsync and the staging.
  *   x_host_f16  HOST fp16 [M][K];  y_host_f16  HOST fp16 [M][N].
  *   words, lut_f16             DEVICE, the resident packed layer.
  *   x_dev [M][K] fp16, xq_dev [M][K/2], scale_dev [M] fp16, y_dev [M][N] fp16, workspace:

@@ -4,6 +4,7 @@ Argument marshalling only: tensors are allocated by torch (device memory and str
 computation runs in the library's CUDA kernels.  There is no fallback: if the shared library
 is missing or a call fails, an exception is raised.
 """
+import contextlib
 import ctypes as C
 import os
 
@@ -75,6 +76,17 @@ def _ptr(t):
     return C.c_void_p(t.data_ptr()) if t is not None else None
 
 
+_NULL_CTX = contextlib.nullcontext()
+
+
+def _on(t):
+    """Context that makes t's device current (nothing to do when it already is: the common case, and the
+    device guard costs microseconds that a decode step notices)."""
+    if torch.cuda.current_device() == t.device.index:
+        return _NULL_CTX
+    return torch.cuda.device(t.device)
+
+
 def _stream(t):
     return C.c_void_p(torch.cuda.current_stream(t.device).cuda_stream)
 
@@ -90,7 +102,7 @@ def rcp_pack_weights(codes: torch.Tensor, out: torch.Tensor = None) -> torch.Ten
     _dev(codes, torch.uint8, "codes")
     N, K = codes.shape
     words = out if out is not None else torch.empty((N, K // 16), dtype=torch.int32, device=codes.device)
-    with torch.cuda.device(codes.device):
+    with _on(codes):
         _check("rcp_pack_weights", lib().rcp_pack_weights(_ptr(codes), N, K, _ptr(words), _stream(codes)))
     return words
 
@@ -107,7 +119,7 @@ def rcp_ldp_export(w, sig_beta, sig_gamma, sig_s1, sig_s2, group):
             raise ValueError(f"{name}: expected shape [N][K/group]")
     words = torch.empty((N, K // 16), dtype=torch.int32, device=w.device)
     lut = torch.empty((N, K // group, 4), dtype=torch.float16, device=w.device)
-    with torch.cuda.device(w.device):
+    with _on(w):
         _check("rcp_ldp_export",
                lib().rcp_ldp_export(_ptr(w), _ptr(sig_beta), _ptr(sig_gamma), _ptr(sig_s1), _ptr(sig_s2), N, K, group,
                                     _ptr(words), _ptr(lut), _stream(w)))
@@ -122,7 +134,7 @@ def rcp_quantize_act(x: torch.Tensor, had_block: int, clip_ratio: float = 1.0, x
         xq = torch.empty((M, K // 2), dtype=torch.uint8, device=x.device)
     if scale is None:
         scale = torch.empty((M,), dtype=torch.float16, device=x.device)
-    with torch.cuda.device(x.device):
+    with _on(x):
         _check("rcp_quantize_act",
                lib().rcp_quantize_act(_ptr(x), M, K, int(had_block), float(clip_ratio), _ptr(xq), _ptr(scale),
                                       _stream(x)))
@@ -155,7 +167,7 @@ def rcp_gemv_w2a4(words, lut, xq, scale, y=None, workspace=None, S_dbg=None, var
     if workspace is None and rcp_gemv_workspace_bytes(M, N, K) > 0:
         workspace = make_workspace(M, N, K, words.device)
     v = VARIANTS[variant] if isinstance(variant, str) else int(variant)
-    with torch.cuda.device(words.device):
+    with _on(words):
         _check("rcp_gemv_w2a4",
                lib().rcp_gemv_w2a4_variant(v, _ptr(words), _ptr(lut), _ptr(xq), _ptr(scale), M, N, K, _ptr(y),
                                            _ptr(workspace), _ptr(S_dbg), _stream(words)))
@@ -180,7 +192,7 @@ def rcp_gemv_w2a4_grouped(words, lut, xq, scale, group=128, y=None, workspace=No
     if workspace is None and rcp_gemv_workspace_bytes(M, N, K) > 0:
         workspace = make_workspace(M, N, K, words.device)
     v = VARIANTS[variant] if isinstance(variant, str) else int(variant)
-    with torch.cuda.device(words.device):
+    with _on(words):
         _check("rcp_gemv_w2a4_grouped",
                lib().rcp_gemv_w2a4_grouped_variant(v, _ptr(words), _ptr(lut), group, _ptr(xq), _ptr(scale), M, N, K,
                                                    _ptr(y), _ptr(workspace), _ptr(S_dbg), _stream(words)))
@@ -206,7 +218,7 @@ def rcp_gemv_w2a4_static(words, lut, xq, scale, y=None):
         raise ValueError("shape mismatch between words, lut, xq and scale")
     if y is None:
         y = torch.empty((M, N), dtype=torch.float16, device=words.device)
-    with torch.cuda.device(words.device):
+    with _on(words):
         _check("rcp_gemv_w2a4_static",
                lib().rcp_gemv_w2a4_static(_ptr(words), _ptr(lut), _ptr(xq), _ptr(scale), M, N, K, _ptr(y),
                                           _stream(words)))
@@ -230,7 +242,7 @@ def rcp_linear_w2a4(x, had_block, clip_ratio, words, lut, group=0, y=None, xq=No
         y = torch.empty((M, N), dtype=torch.float16, device=words.device)
     if workspace is None:
         workspace = make_workspace(M, N, K, words.device)
-    with torch.cuda.device(words.device):
+    with _on(words):
         _check("rcp_linear_w2a4",
                lib().rcp_linear_w2a4(_ptr(x), M, K, int(had_block), float(clip_ratio), _ptr(words), _ptr(lut), group, N,
                                      _ptr(y), _ptr(xq), _ptr(scale), _ptr(workspace), _stream(words)))
@@ -252,7 +264,7 @@ def rcp_linear_w2a4_host(x_host, had_block, clip_ratio, words, lut, y_host, x_de
     N = words.shape[0]
     if x_host.is_cuda or y_host.is_cuda or x_host.dtype != torch.float16 or y_host.dtype != torch.float16:
         raise TypeError("x_host / y_host must be fp16 host tensors")
-    with torch.cuda.device(words.device):
+    with _on(words):
         _check("rcp_linear_w2a4_host",
                lib().rcp_linear_w2a4_host(_ptr(x_host), M, K, int(had_block), float(clip_ratio), _ptr(words), _ptr(lut),
                                           N, _ptr(y_host), _ptr(x_dev), _ptr(xq_dev), _ptr(scale_dev), _ptr(y_dev),

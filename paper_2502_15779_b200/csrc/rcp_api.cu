@@ -616,14 +616,39 @@ int rcp_linear_w2a4(const void* x_f16, int M, int K, int had_block, float clip_r
 int rcp_linear_w2a4_host(const void* x_host_f16, int M, int K, int had_block, float clip_ratio,
                          const uint32_t* words, const void* lut_f16, int N, void* y_host_f16, void* x_dev,
                          uint8_t* xq_dev, void* scale_dev, void* y_dev, void* workspace, void* stream) {
-  if (!x_host_f16 || !y_host_f16 || !x_dev || !y_dev) return RCP_ERR_NULL;
+  if (!x_host_f16 || !y_host_f16 || !x_dev || !y_dev) return RCP_ERR_NULL;   // staging is needed for pageable memory
   if (M < 1 || M > rcp::kMaxTokens || N < 1 || !k_ok(K)) return RCP_ERR_SHAPE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  RCP_CUDA(cudaMemcpyAsync(x_dev, x_host_f16, (size_t)M * K * 2, cudaMemcpyHostToDevice, st));
-  const int rc = rcp_linear_w2a4(x_dev, M, K, had_block, clip_ratio, words, lut_f16, 0, N, y_dev, xq_dev, scale_dev,
-                                 workspace, stream);
+  // Page-locked host memory is visible to the GPU: the quantizer (a handful of CTAs) then reads the
+  // few kilobytes of activations straight from it, which saves a trip through the copy engine. The
+  // single-kernel form would have every CTA fetch them across the bus, so it is not used here.
+  cudaPointerAttributes attr;
+  const void* x_mapped = nullptr;
+  if (xq_dev && scale_dev && cudaPointerGetAttributes(&attr, x_host_f16) == cudaSuccess &&
+      attr.type == cudaMemoryTypeHost && attr.devicePointer && aligned16(attr.devicePointer))
+    x_mapped = attr.devicePointer;
+  else
+    (void)cudaGetLastError();   // an unregistered pointer is not an error here
+  // Likewise the GEMV can store its few kilobytes of results straight into page-locked host memory.
+  void* y_mapped = nullptr;
+  if (cudaPointerGetAttributes(&attr, y_host_f16) == cudaSuccess && attr.type == cudaMemoryTypeHost &&
+      attr.devicePointer)
+    y_mapped = attr.devicePointer;
+  else
+    (void)cudaGetLastError();
+  void* const y_out = y_mapped ? y_mapped : y_dev;
+  int rc;
+  if (x_mapped) {
+    rc = rcp_quantize_act(x_mapped, M, K, had_block, clip_ratio, xq_dev, scale_dev, stream);
+    if (rc == RCP_OK)
+      rc = rcp_gemv_w2a4(words, lut_f16, xq_dev, scale_dev, M, N, K, y_out, workspace, nullptr, stream);
+  } else {
+    RCP_CUDA(cudaMemcpyAsync(x_dev, x_host_f16, (size_t)M * K * 2, cudaMemcpyHostToDevice, st));
+    rc = rcp_linear_w2a4(x_dev, M, K, had_block, clip_ratio, words, lut_f16, 0, N, y_out, xq_dev, scale_dev, workspace,
+                         stream);
+  }
   if (rc != RCP_OK) return rc;
-  RCP_CUDA(cudaMemcpyAsync(y_host_f16, y_dev, (size_t)M * N * 2, cudaMemcpyDeviceToHost, st));
+  if (!y_mapped) RCP_CUDA(cudaMemcpyAsync(y_host_f16, y_dev, (size_t)M * N * 2, cudaMemcpyDeviceToHost, st));
   return RCP_OK;
 }
 
