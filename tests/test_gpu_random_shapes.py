@@ -67,3 +67,34 @@ def test_random_shape(N, K, M, variant, grouped, i):
         got = out.float().cpu().numpy().astype(np.float64)[:, rows]
         assert np.all(np.isfinite(got))
         assert np.all(np.abs(got - ref["y"]) <= ref["tol"])
+
+
+@pytest.mark.parametrize("N,K,M,grouped", [(70, 65536, 1, False), (40, 65536, 8, False), (33, 65536, 2, True),
+                                           (20, 65536, 5, True), (300000, 64, 1, False), (150000, 128, 3, True),
+                                           (1, 64, 16, False), (1, 128, 16, True)])
+def test_extreme_shapes(N, K, M, grouped):
+    """The longest K the library takes, very many short rows, a single row: through the default variant."""
+    B = 128 if K >= 128 else 64
+    seed = N + K + M
+    if grouped:
+        codes, lut = synth.make_layer_grouped(N, K, 128, B, "uniform", seed, device=DEV)
+    else:
+        codes, lut = synth.make_layer(N, K, B, "uniform", seed, device=DEV)
+    x = synth.make_activations(M, K, seed, device=DEV)
+    words = rcp.rcp_pack_weights(codes)
+    xq, scale = rcp.rcp_quantize_act(x, B, 1.0)
+    ws = rcp.make_workspace(M, N, K, DEV)
+    y = (rcp.rcp_gemv_w2a4_grouped(words, lut, xq, scale, group=128, workspace=ws) if grouped
+         else rcp.rcp_gemv_w2a4(words, lut, xq, scale, workspace=ws))
+    torch.cuda.synchronize()
+    assert int(ws.abs().max()) == 0
+    rows = np.arange(N) if N <= 4096 else np.unique(np.concatenate(
+        [np.arange(64), np.arange(N - 64, N), np.random.default_rng(seed).integers(0, N, size=512)]))
+    qa = oracle.quantize_act(f16_bits(x), B, 1.0)
+    assert np.array_equal(xq.cpu().numpy(), qa["xq"]) and np.array_equal(f16_bits(scale), qa["scale"])
+    w_ref = oracle.pack_weights(codes.cpu().numpy()[rows])
+    lb = np.ascontiguousarray(f16_bits(lut)[rows])
+    ref = (oracle.gemv_w2a4_grouped(w_ref, lb, qa["xq"], qa["scale"], 128) if grouped
+           else oracle.gemv_w2a4(w_ref, lb, qa["xq"], qa["scale"]))
+    got = y.float().cpu().numpy().astype(np.float64)[:, rows]
+    assert np.all(np.isfinite(got)) and np.all(np.abs(got - ref["y"]) <= ref["tol"])
