@@ -123,6 +123,11 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
   return v;
 }
+__device__ __forceinline__ uint2 lds64(uint32_t addr) {
+  uint2 v;
+  asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+  return v;
+}
 __device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                          uint32_t b1) {
   asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -440,12 +445,12 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
 
   // 16 rows x 128 bytes of weights at shared address a_grp against the activations of one chunk
   auto compute_chunk = [&](uint32_t a_grp, uint32_t b_chunk) {
-    const uint8_t* const a_ptr = gen + (a_grp - base);
-    const uint8_t* const b_ptr = bs + b_chunk;
+    const uint32_t a_ptr = a_grp;                          // 32-bit shared-memory addresses throughout
+    const uint32_t b_ptr = base + (uint32_t)p.off_bs + b_chunk;
 #pragma unroll
     for (int i = 0; i < 2; i++) {
-      const uint4 U = *reinterpret_cast<const uint4*>(a_ptr + a_chunk[i]);
-      const uint4 V = *reinterpret_cast<const uint4*>(a_ptr + 8 * 128 + a_chunk[i]);
+      const uint4 U = lds128(a_ptr + a_chunk[i]);
+      const uint4 V = lds128(a_ptr + 8 * 128 + a_chunk[i]);
       const uint32_t uw[4] = {U.x, U.y, U.z, U.w};
       const uint32_t vw[4] = {V.x, V.y, V.z, V.w};
 #pragma unroll
@@ -457,8 +462,8 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
         if constexpr (NF_D > 0) {
 #pragma unroll
           for (int tok = 0; tok < NTD; tok++) {
-            const uint4 x = *reinterpret_cast<const uint4*>(b_ptr + bD_lane[tok] + b_off);
-            const uint4 y = *reinterpret_cast<const uint4*>(b_ptr + bD_lane[tok] + b_off + half_stride);
+            const uint4 x = lds128(b_ptr + bD_lane[tok] + b_off);
+            const uint4 y = lds128(b_ptr + bD_lane[tok] + b_off + half_stride);
             bD[tok][0][0] = x.x; bD[tok][0][1] = x.y; bD[tok][1][0] = x.z; bD[tok][1][1] = x.w;
             bD[tok][2][0] = y.x; bD[tok][2][1] = y.y; bD[tok][3][0] = y.z; bD[tok][3][1] = y.w;
           }
@@ -468,8 +473,8 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
 #pragma unroll
             for (int pp = 0; pp < 4; pp++) { bM[pp][0] = bD[0][pp][0]; bM[pp][1] = bD[0][pp][1]; }
           } else {
-            const uint4 x = *reinterpret_cast<const uint4*>(b_ptr + bM_lane + b_off);
-            const uint4 y = *reinterpret_cast<const uint4*>(b_ptr + bM_lane + b_off + half_stride);
+            const uint4 x = lds128(b_ptr + bM_lane + b_off);
+            const uint4 y = lds128(b_ptr + bM_lane + b_off + half_stride);
             bM[0][0] = x.x; bM[0][1] = x.y; bM[1][0] = x.z; bM[1][1] = x.w;
             bM[2][0] = y.x; bM[2][1] = y.y; bM[3][0] = y.z; bM[3][1] = y.w;
           }
@@ -561,15 +566,16 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   // twelve MMAs.
   auto compute_chunk_grp_mma = [&](uint32_t a_grp, uint32_t b_chunk, int ch, const uint2 (&lg)[NLG][2]) {
     if constexpr (kRelabel) {
-      const uint8_t* const a_row = gen + (a_grp - base) + grow * 128 + ((t & 1) << 3);
+      const uint32_t a_row = a_grp + (uint32_t)(grow * 128 + ((t & 1) << 3));
+      const uint32_t b_grp = base + (uint32_t)p.off_bs + b_chunk + bM_lane;
 #pragma unroll
       for (int j = 0; j < 4; j++) {
         const uint32_t a_sw = (uint32_t)(((2 * j + (t >> 1)) ^ (grow & 7)) << 4);
-        const uint2 U = *reinterpret_cast<const uint2*>(a_row + a_sw);
-        const uint2 V = *reinterpret_cast<const uint2*>(a_row + 8 * 128 + a_sw);
-        const uint8_t* const b_ptr = bs + b_chunk + (uint32_t)(j * 2) * half_stride + bM_lane;
-        const uint4 x = *reinterpret_cast<const uint4*>(b_ptr);
-        const uint4 y = *reinterpret_cast<const uint4*>(b_ptr + half_stride);
+        const uint2 U = lds64(a_row + a_sw);
+        const uint2 V = lds64(a_row + 8 * 128 + a_sw);
+        const uint32_t b_ptr = b_grp + (uint32_t)(j * 2) * half_stride;
+        const uint4 x = lds128(b_ptr);
+        const uint4 y = lds128(b_ptr + half_stride);
         const uint32_t bM[4][2] = {{x.x, x.y}, {x.z, x.w}, {y.x, y.y}, {y.z, y.w}};
         const uint32_t u0 = U.x, u1 = U.y, v0 = V.x, v1 = V.y;
         const uint32_t u0s = u0 + u0, u1s = u1 + u1, v0s = v0 + v0, v1s = v1 + v1;
