@@ -145,6 +145,13 @@ __device__ __forceinline__ void mma_u8s8_zero(int (&d)[4], uint32_t a0, uint32_t
 __device__ __forceinline__ float small_int_to_float(int x) {
   return __int_as_float(x + 0x4B400000) - 12582912.0f;   // 1.5 * 2^23 + x, exactly
 }
+// a & b & c as one three-input logic operation (written out: the compiler would otherwise keep a & b as a
+// common subexpression of the four positions and spend a fifth operation per word)
+__device__ __forceinline__ uint32_t and3(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("lop3.b32 %0, %1, %2, %3, 0x80;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
 __device__ __forceinline__ void dp4a_u8s8(int& d, uint32_t a, uint32_t b) {
   asm("dp4a.u32.s32 %0, %1, %2, %0;" : "+r"(d) : "r"(a), "r"(b));
 }
@@ -487,10 +494,10 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
           const int pp = ((po & 1) << 1) | (po >> 1);
           const uint32_t m0 = 0x01010101u << (2 * pp), m1 = m0 << 1;
           // the three planes of the four words: b0, b1, b0*b1 (the last two scaled by 2)
-          const uint32_t au0[3] = {u0 & m0, u0 & m1, u0 & u0s & m1};
-          const uint32_t au1[3] = {u1 & m0, u1 & m1, u1 & u1s & m1};
-          const uint32_t av0[3] = {v0 & m0, v0 & m1, v0 & v0s & m1};
-          const uint32_t av1[3] = {v1 & m0, v1 & m1, v1 & v1s & m1};
+          const uint32_t au0[3] = {u0 & m0, u0 & m1, and3(u0, u0s, m1)};
+          const uint32_t au1[3] = {u1 & m0, u1 & m1, and3(u1, u1s, m1)};
+          const uint32_t av0[3] = {v0 & m0, v0 & m1, and3(v0, v0s, m1)};
+          const uint32_t av1[3] = {v1 & m0, v1 & m1, and3(v1, v1s, m1)};
 #pragma unroll
           for (int f = 0; f < NF_M; f++)
             mma_u8s8(accM[f][pp >> 1], au0[f], av0[f], au1[f], av1[f], bM[pp][0], bM[pp][1]);
@@ -583,10 +590,10 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
         for (int po = 0; po < 4; po++) {
           const int pp = ((po & 1) << 1) | (po >> 1);
           const uint32_t m0 = 0x01010101u << (2 * pp), m1 = m0 << 1;
-          const uint32_t au0[3] = {u0 & m0, u0 & m1, u0 & u0s & m1};
-          const uint32_t au1[3] = {u1 & m0, u1 & m1, u1 & u1s & m1};
-          const uint32_t av0[3] = {v0 & m0, v0 & m1, v0 & v0s & m1};
-          const uint32_t av1[3] = {v1 & m0, v1 & m1, v1 & v1s & m1};
+          const uint32_t au0[3] = {u0 & m0, u0 & m1, and3(u0, u0s, m1)};
+          const uint32_t au1[3] = {u1 & m0, u1 & m1, and3(u1, u1s, m1)};
+          const uint32_t av0[3] = {v0 & m0, v0 & m1, and3(v0, v0s, m1)};
+          const uint32_t av1[3] = {v1 & m0, v1 & m1, and3(v1, v1s, m1)};
 #pragma unroll
           for (int f = 0; f < 3; f++) {
             if (po < 2) mma_u8s8_zero(accM[f][pp >> 1], au0[f], av0[f], au1[f], av1[f], bM[pp][0], bM[pp][1]);
