@@ -98,3 +98,39 @@ def test_extreme_shapes(N, K, M, grouped):
            else oracle.gemv_w2a4(w_ref, lb, qa["xq"], qa["scale"]))
     got = y.float().cpu().numpy().astype(np.float64)[:, rows]
     assert np.all(np.isfinite(got)) and np.all(np.abs(got - ref["y"]) <= ref["tol"])
+
+
+@pytest.mark.parametrize("N,K,M,variant,grouped", [(4096, 4096, 1, "auto", False), (5000, 2048, 8, "auto", False),
+                                                   (3000, 11008, 2, "auto", True), (2600, 8192, 1, "linear", False)])
+def test_many_launches_repeat_bit_for_bit(N, K, M, variant, grouped):
+    """A few thousand back-to-back launches (the ring, its barriers and the phases restart every time): the
+    status word stays clear and every launch returns the same bits."""
+    B = K if (K & (K - 1)) == 0 else 128
+    if grouped:
+        codes, lut = synth.make_layer_grouped(N, K, 128, B, "uniform", 77, device=DEV)
+    else:
+        codes, lut = synth.make_layer(N, K, B, "uniform", 77, device=DEV)
+    x = synth.make_activations(M, K, 77, device=DEV)
+    words = rcp.rcp_pack_weights(codes)
+    xq, scale = rcp.rcp_quantize_act(x, B, 1.0)
+    ws = rcp.make_workspace(M, N, K, DEV)
+    ys = [torch.empty(M, N, dtype=torch.float16, device=DEV) for _ in range(2)]
+
+    def launch(y):
+        if variant == "linear":
+            rcp.rcp_linear_w2a4(x, B, 1.0, words, lut, y=y, xq=xq, scale=scale, workspace=ws)
+        elif grouped:
+            rcp.rcp_gemv_w2a4_grouped(words, lut, xq, scale, group=128, y=y, workspace=ws)
+        else:
+            rcp.rcp_gemv_w2a4(words, lut, xq, scale, y=y, workspace=ws)
+
+    launch(ys[0])
+    ref = ys[0].clone()
+    for i in range(3000):
+        launch(ys[i & 1])
+        if i % 500 == 499:
+            torch.cuda.synchronize()
+            assert torch.equal(ys[0].view(torch.int16), ref.view(torch.int16))
+            assert torch.equal(ys[1].view(torch.int16), ref.view(torch.int16))
+    torch.cuda.synchronize()
+    assert int(ws.abs().max()) == 0
