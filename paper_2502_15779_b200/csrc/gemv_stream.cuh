@@ -206,10 +206,12 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   const int b = blockIdx.x;
   // Launched with programmatic stream serialization: the next kernel may start as CTAs retire.
   asm volatile("griddepcontrol.launch_dependents;");
+  int* const s_T0tot = reinterpret_cast<int*>(s_scale + 24);   // [8]: sum of q per token, behind scales and maxima
   if (tid == 0) {
     for (int s = 0; s < stages; s++) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, kCWarps); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  if (tid < 8) s_T0tot[tid] = 0;
   __syncthreads();
 
   // ------------------------------------------------------------------ producer
@@ -318,14 +320,15 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     } else {
       tsum += __shfl_xor_sync(0xffffffffu, tsum, 8);
       tsum += __shfl_xor_sync(0xffffffffu, tsum, 16);
-      if (lane == 0 && ch < p.nchunk) s_T0c[ch] = tsum;
+      if (lane == 0 && ch < p.nchunk) atomicAdd(&s_T0tot[0], tsum);
     }
     if constexpr (!GRP)
       for (int i = tid; i < 2 * 8 * 16 * M * 3; i += kCWarps * 32) s_red[i] = 0;
   } else
   // ------------------------------------------------------------------ activations (consumer warps)
   // One unit = (column, chunk, i, pr, t) = two words. The 16 units of a (column, chunk) are 16
-  // consecutive lanes: their sum of q goes to s_T0c.
+  // consecutive lanes: their sum of q is added to the token's total s_T0tot (per-row grid) or kept per group
+  // of 128 in s_T0c (group-wise grid).
   {
     const int W = p.K / 16;
     const int total = ncol * p.nchunk * 16;
@@ -361,7 +364,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
       if constexpr (!GRP) {
 #pragma unroll
         for (int d = 8; d > 0; d >>= 1) tsum += __shfl_xor_sync(0xffffffffu, tsum, d);
-        if ((lane & 15) == 0 && u < total) s_T0c[col * p.nchunk + ch] = tsum;
+        if ((lane & 15) == 0 && u < total) atomicAdd(&s_T0tot[col], tsum);   // integer: any order gives the same sum
       } else if constexpr (kRelabel) {   // the group is bits 2,3 of the unit: add up over bits 0,1
         tsum += __shfl_xor_sync(0xffffffffu, tsum, 1);
         tsum += __shfl_xor_sync(0xffffffffu, tsum, 2);
@@ -423,14 +426,10 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     else { etok[e] = (t == 0) ? (e >> 1) : kMaxTokens; err[e] = e & 1; }
     T0v[e] = 0;
   }
-  // T0 of every token: sum over the chunks, by the whole warp; a lane keeps the tokens it emits
-  for (int m = 0; m < (GRP ? 0 : M); m++) {
-    int a = 0;
-    for (int c = lane; c < p.nchunk; c += 32) a += s_T0c[m * p.nchunk + c];
+  // T0 of the tokens this lane emits (added up while the activations were expanded)
+  if constexpr (!GRP) {
 #pragma unroll
-    for (int d = 16; d > 0; d >>= 1) a += __shfl_xor_sync(0xffffffffu, a, d);
-#pragma unroll
-    for (int e = 0; e < NE; e++) if (etok[e] == m) T0v[e] = a;
+    for (int e = 0; e < NE; e++) if (etok[e] < M) T0v[e] = s_T0tot[etok[e]];
   }
 
   // per-lane constant parts of the shared-memory addresses
