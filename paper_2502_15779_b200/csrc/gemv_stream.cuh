@@ -69,6 +69,7 @@ struct GemvParams {
   int M, N, K;
   int ngrp;             // group-wise grid: groups of 128 weights per row (K / 128), lut is [N][ngrp]; else 0
   int nchunk;           // 128-byte chunks per row, ceil(K / 512)
+  int inv_nchunk;       // ceil(2^20 / nchunk): x / nchunk == (x * inv_nchunk) >> 20 for x < 2^20 / nchunk
   int nphase;
   GemvPhase phase[kMaxPhases];
   // fused activation quantizer (FQ): x fp16 [M][K] replaces xq and scale as input
@@ -336,7 +337,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
       const int u = u0 + lane;
       int tsum = 0;
       const int pair = u >> 4;
-      const int col = pair / p.nchunk, ch = pair - col * p.nchunk;
+      const int col = (int)(((uint32_t)pair * (uint32_t)p.inv_nchunk) >> 20), ch = pair - col * p.nchunk;   // pair / nchunk
       if (u < total) {
         const int lo = u & 3, hi = (u >> 2) & 3;   // lo: 16-byte slot t of the column block; hi: 2 i + pr, or the group
         const int wx = ch * kChunkWords + (kRelabel ? 8 * hi + 2 * lo : 8 * lo + 2 * hi);   // word index in the row
@@ -344,18 +345,21 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
         if (wx < W) x = __ldg(reinterpret_cast<const uint4*>(p.xq + (size_t)col * (p.K / 2)) + (wx >> 1));
         uint32_t q[4][2];
 #pragma unroll
-        for (int pp = 0; pp < 4; pp++) {
+        for (int w = 0; w < 2; w++) {
+          const uint32_t lo32 = w ? x.z : x.x, hi32 = w ? x.w : x.y;   // codes 0..7 and 8..15 of the word
+          // even and odd codes of each half as bytes, each nibble sign-extended to a byte
+          uint32_t n4[4] = {lo32 & 0x0F0F0F0Fu, (lo32 >> 4) & 0x0F0F0F0Fu, hi32 & 0x0F0F0F0Fu, (hi32 >> 4) & 0x0F0F0F0Fu};
 #pragma unroll
-          for (int w = 0; w < 2; w++) {
-            const uint32_t lo32 = w ? x.z : x.x, hi32 = w ? x.w : x.y;   // codes 0..7 and 8..15 of the word
-            const uint32_t a = (lo32 >> (4 * pp)) & 0x000F000Fu;
-            const uint32_t c = (hi32 >> (4 * pp)) & 0x000F000Fu;
-            uint32_t v = __byte_perm(a, c, 0x6420);        // nibbles of codes p, 4+p, 8+p, 12+p
-            v |= (v & 0x08080808u) * 0x1Eu;                 // sign-extend each nibble to a byte
-            tsum = __dp4a((int)v, 0x01010101, tsum);
-            if ((pp & 1) == 0) v = (v << 2) & 0xFCFCFCFCu;  // even positions carry 4 q
-            q[pp][w] = v;
+          for (int h = 0; h < 4; h++) {
+            n4[h] |= (n4[h] & 0x08080808u) * 0x1Eu;
+            tsum = __dp4a((int)n4[h], 0x01010101, tsum);
           }
+          // position p of a byte of codes: codes p, 4+p, 8+p, 12+p; even positions carry 4 q
+          const uint32_t v0 = __byte_perm(n4[0], n4[2], 0x6420), v2 = __byte_perm(n4[0], n4[2], 0x7531);
+          q[0][w] = (v0 << 2) & 0xFCFCFCFCu;
+          q[1][w] = __byte_perm(n4[1], n4[3], 0x6420);
+          q[2][w] = (v2 << 2) & 0xFCFCFCFCu;
+          q[3][w] = __byte_perm(n4[1], n4[3], 0x7531);
         }
         uint8_t* dst = bs + ((size_t)(((ch * 4 + hi) * 2) * ncol + col)) * 64 + lo * 16;
         *reinterpret_cast<uint4*>(dst) = make_uint4(q[0][0], q[0][1], q[1][0], q[1][1]);

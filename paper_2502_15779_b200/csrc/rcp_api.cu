@@ -234,6 +234,7 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   gp.M = M; gp.N = N; gp.K = K;
   gp.ngrp = grouped ? K / 128 : 0;
   gp.nchunk = pl.nchunk;
+  gp.inv_nchunk = ((1 << 20) + pl.nchunk - 1) / pl.nchunk;
   gp.nphase = pl.nphase;
   for (int i = 0; i < rcp::kMaxPhases; i++) gp.phase[i] = i < pl.nphase ? pl.phase[i] : rcp::GemvPhase{1, 0, 0, 1, 0};
   gp.stages = pl.stages;
