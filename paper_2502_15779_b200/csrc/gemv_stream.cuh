@@ -55,9 +55,15 @@ enum GemvMode { kModeMma = 0, kModeHybrid = 1, kModeDp4a = 2 };
 
 constexpr int kMaxPhases = 6;
 // One phase, repeated reps times: `total` groups starting at group first + rep * total are shared out
-// evenly over the CTAs b < ncta, CTA b taking groups [total b / ncta, total (b+1) / ncta) of them,
-// at most gpc. KS = 16 / gpc warps share a group; the TMA box has 16 gpc rows.
-struct GemvPhase { int gpc, first, total, ncta, reps; };
+// evenly over the CTAs b < ncta: with q = total / ncta and r = total % ncta the first r CTAs take q + 1
+// consecutive groups, the others q (at most gpc). KS = 16 / gpc warps share a group; the TMA box has
+// 16 gpc rows. The host works out everything that would need a division in the kernel.
+struct GemvPhase {
+  int gpc, first, total, ncta, reps;
+  int q, r;        // total / ncta, total % ncta
+  int ks, inv_ks;  // KS, and ceil(256 / KS): warp / KS == (warp * inv_ks) >> 8 for warp < 16
+  int sa;          // stages per repetition: ceil(nchunk / KS)
+};
 struct GemvMaps { CUtensorMap m[kMaxPhases]; };   // box of 16 gpc rows x 128 bytes for phase i
 
 struct GemvParams {
@@ -232,10 +238,10 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
       const GemvPhase ph = p.phase[pi];
       if (b >= ph.ncta) continue;
       asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.m[pi]) : "memory");
-      const int KS = kCWarps / ph.gpc;
+      const int KS = ph.ks;
       const uint32_t box = (uint32_t)ph.gpc * kGroupBytes;
-      const int lo = (int)((long long)ph.total * b / ph.ncta);
-      const int SA = (p.nchunk + KS - 1) / KS;
+      const int lo = ph.q * b + min(b, ph.r);
+      const int SA = ph.sa;
       for (int rp = 0; rp < ph.reps; rp++) {
         const int row0 = (ph.first + rp * ph.total + lo) * 16;
         for (int s = 0; s < SA; s++) {
@@ -732,10 +738,10 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   for (int pi = 0; pi < p.nphase; pi++) {
     const GemvPhase ph = p.phase[pi];
     if (b >= ph.ncta) continue;
-    const int KS = kCWarps / ph.gpc;
-    const int grp = warp / KS, ks = warp - grp * KS;
-    const int SA = (p.nchunk + KS - 1) / KS;
-    const int lo = (int)((long long)ph.total * b / ph.ncta), hi = (int)((long long)ph.total * (b + 1) / ph.ncta);
+    const int KS = ph.ks;
+    const int grp = (warp * ph.inv_ks) >> 8, ks = warp - grp * KS;
+    const int SA = ph.sa;
+    const int lo = ph.q * b + min(b, ph.r), hi = lo + ph.q + (b < ph.r ? 1 : 0);
     const bool active = grp < hi - lo;   // fewer groups than gpc here, or warps beyond gpc KS
     const uint32_t a_off = (uint32_t)ks * ((uint32_t)ph.gpc * kGroupBytes) + (uint32_t)grp * kGroupBytes;
     for (int rp = 0; rp < ph.reps; rp++) {

@@ -81,6 +81,18 @@ long long phase_cost(int gpc, int nchunk) {
   return (long long)stages * per_sched * 504 + 2500;
 }
 
+// A phase with the quotients the kernel would otherwise divide for.
+rcp::GemvPhase make_phase(int gpc, int first, int total, int ncta, int reps, int nchunk) {
+  rcp::GemvPhase ph;
+  ph.gpc = gpc; ph.first = first; ph.total = total; ph.ncta = ncta; ph.reps = reps;
+  ph.q = total / ncta;
+  ph.r = total % ncta;
+  ph.ks = rcp::kCWarps / gpc;
+  ph.inv_ks = (256 + ph.ks - 1) / ph.ks;
+  ph.sa = (nchunk + ph.ks - 1) / ph.ks;
+  return ph;
+}
+
 // Splits `rem` leftover groups (fewer than 16 per CTA) into phases: shares of 8, 4, 2 or 1 groups
 // per CTA keep all warps busy but cost a phase each; one last phase takes whatever is left,
 // ceil(left / CTAs) groups per CTA. Picks the cheapest combination. Returns the number of phases.
@@ -107,13 +119,13 @@ int plan_leftover(int rem, int sms, int nchunk, rcp::GemvPhase* out) {
   for (int i = 0; i < 4; i++) {
     if (!(best_mask >> i & 1)) continue;
     const int gpc = 8 >> i;
-    out[n++] = rcp::GemvPhase{gpc, first, gpc * sms, sms, 1};
+    out[n++] = make_phase(gpc, first, gpc * sms, sms, 1, nchunk);
     first += gpc * sms;
     left -= gpc * sms;
   }
   if (left > 0) {
     const int ncta = std::min(left, sms);
-    out[n++] = rcp::GemvPhase{(left + ncta - 1) / ncta, first, left, ncta, 1};
+    out[n++] = make_phase((left + ncta - 1) / ncta, first, left, ncta, 1, nchunk);
   }
   return n;
 }
@@ -129,7 +141,7 @@ StreamPlan make_plan(int M, int N, int K, int sms, bool grouped = false, size_t 
   const int R = groups / per_round;
   pl.nphase = plan_leftover(groups - R * per_round, sms, pl.nchunk, pl.phase);
   int first = groups - R * per_round;
-  if (R > 0) pl.phase[pl.nphase++] = rcp::GemvPhase{rcp::kCWarps, first, per_round, sms, R};
+  if (R > 0) pl.phase[pl.nphase++] = make_phase(rcp::kCWarps, first, per_round, sms, R, pl.nchunk);
   const size_t bs_bytes = (size_t)pl.nchunk * rcp::kChunkWords * 16 * M;
   // sums of q per chunk (per group of 128: four per chunk); reduction buffers: integer sums of 8
   // row groups x 3 planes, or (group-wise grid) one fp32 term per warp
@@ -236,7 +248,7 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   gp.nchunk = pl.nchunk;
   gp.inv_nchunk = ((1 << 20) + pl.nchunk - 1) / pl.nchunk;
   gp.nphase = pl.nphase;
-  for (int i = 0; i < rcp::kMaxPhases; i++) gp.phase[i] = i < pl.nphase ? pl.phase[i] : rcp::GemvPhase{1, 0, 0, 1, 0};
+  for (int i = 0; i < rcp::kMaxPhases; i++) gp.phase[i] = i < pl.nphase ? pl.phase[i] : make_phase(1, 0, 0, 1, 0, pl.nchunk);
   gp.stages = pl.stages;
   // one 32 KB stage per CTA at about 6 TB/s for the whole grid, in SM clocks (about 2 GHz)
   gp.ramp_clk = (int)((double)rcp::kStageBytes * pl.grid / 6.0e12 * 1.9e9);

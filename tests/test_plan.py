@@ -38,8 +38,9 @@ def check(L, M, N, K, sms=148):
         assert (16 // gpc) * gpc <= 16
         if 16 // gpc > 1:
             assert gpc <= 8          # the shared-memory reduction holds eight groups
-        # shares of the CTAs tile [0, total) without gaps
-        assert sum((total * (b + 1)) // ncta - (total * b) // ncta for b in range(ncta)) == total
+        # shares of the CTAs tile [0, total) without gaps: the first total % ncta CTAs take one group more
+        q, r = divmod(total, ncta)
+        assert sum(q + (1 if b < r else 0) for b in range(ncta)) == total and q + (1 if r else 0) == per_cta_max
         nxt += total * reps
     assert nxt == groups, (nxt, groups)
     assert len(p["phases"]) <= 6
