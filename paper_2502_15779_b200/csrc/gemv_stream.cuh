@@ -214,18 +214,24 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   // Launched with programmatic stream serialization: the next kernel may start as CTAs retire.
   asm volatile("griddepcontrol.launch_dependents;");
   int* const s_T0tot = reinterpret_cast<int*>(s_scale + 24);   // [8]: sum of q per token, behind scales and maxima
-  if (tid == 0) {
-    for (int s = 0; s < stages; s++) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, kCWarps); }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  // The producer warp sets up the ring's barriers and only announces that (bar.arrive): its first
+  // requests go out without waiting for anybody. The consumer warps wait for the announcement.
+  if (warp != kCWarps) {
+    if (tid < 8) s_T0tot[tid] = 0;
+    asm volatile("bar.sync 3, %0;" ::"n"(kGThreads) : "memory");
   }
-  if (tid < 8) s_T0tot[tid] = 0;
-  __syncthreads();
 
   // ------------------------------------------------------------------ producer
   // One thread requests every stage of this CTA in order. The weights do not depend on the
   // preceding kernel, so it starts at once (before griddepcontrol.wait), and it never meets the
   // other warps again.
   if (warp == kCWarps) {
+    if (lane == 0) {
+      for (int s = 0; s < stages; s++) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, kCWarps); }
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    asm volatile("bar.arrive 3, %0;" ::"n"(kGThreads) : "memory");
     if (lane != 0) return;
     int slot = 0;
     uint32_t phase = 0;
