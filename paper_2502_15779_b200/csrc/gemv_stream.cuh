@@ -293,13 +293,14 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     }
     int q[16];
     int tsum = 0;
+    if (sc != 0.f) {   // the same for the whole CTA; threads beyond the token hold zeros
+      quantize_int4x16(v, sc, q);
+    } else {
 #pragma unroll
-    for (int e = 0; e < 16; e++) {
-      int qq = 0;
-      if (sc != 0.f && tid < W) qq = max(-8, min(7, __float2int_rn(__fdiv_rn(v[e], sc))));
-      q[e] = qq;
-      tsum += qq;
+      for (int e = 0; e < 16; e++) q[e] = 0;
     }
+#pragma unroll
+    for (int e = 0; e < 16; e++) tsum += q[e];
     const int ch = tid >> 5, wi = tid & 31;
     if (tid < p.nchunk * kChunkWords) {
       uint32_t Q[4];

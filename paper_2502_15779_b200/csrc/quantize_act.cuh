@@ -363,16 +363,19 @@ __global__ void __launch_bounds__(512) quantize_act_wide_kernel(const QuantParam
   float v[16];
   const float s = rotate_token_words<512>(p.x + (size_t)m * p.K, W, p.inv_sqrt_b, p.clip_ratio, sbuf, s_amax, v);
   if (tid == 0) p.scale[m] = __float2half_rn(s);
+  int q[16];
+  if (s != 0.f) {   // the same for the whole CTA; threads beyond the token hold zeros
+    quantize_int4x16(v, s, q);
+  } else {
+#pragma unroll
+    for (int e = 0; e < 16; e++) q[e] = 0;
+  }
   if (tid < W) {
     uint32_t lo32 = 0, hi32 = 0;
-    if (s != 0.f) {
 #pragma unroll
-      for (int e = 0; e < 8; e++) {
-        const int q0 = max(-8, min(7, __float2int_rn(__fdiv_rn(v[e], s))));
-        const int q1 = max(-8, min(7, __float2int_rn(__fdiv_rn(v[8 + e], s))));
-        lo32 |= (uint32_t)(q0 & 0xF) << (4 * e);
-        hi32 |= (uint32_t)(q1 & 0xF) << (4 * e);
-      }
+    for (int e = 0; e < 8; e++) {
+      lo32 |= (uint32_t)(q[e] & 0xF) << (4 * e);
+      hi32 |= (uint32_t)(q[8 + e] & 0xF) << (4 * e);
     }
     *reinterpret_cast<uint2*>(p.xq + (size_t)m * (p.K / 2) + (size_t)tid * 8) = make_uint2(lo32, hi32);
   }
