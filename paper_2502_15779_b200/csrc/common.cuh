@@ -22,7 +22,7 @@ __device__ __forceinline__ __half lut_finish(float s, uint2 lut4, int S0, int S1
   return __float2half_rn(s * acc);
 }
 
-// q[e] = clamp(round-half-even(v[e] / s), -8, 7) for sixteen values, the quotient being the IEEE fp32
+// q[e] = clamp(round-half-even(v[e] / s), -8, 7) for NV values, the quotient being the IEEE fp32
 // division the definition asks for, without dividing in the common case. With rinv = 1 / s (correctly
 // rounded), t = v * rinv lies within 2^-23 |v / s| of the exact quotient and the IEEE quotient within half
 // an ulp of it; clamped to [-8, 7] (rounding and clamping commute: the bounds are integers) the two differ
@@ -30,11 +30,12 @@ __device__ __forceinline__ __half lut_finish(float s, uint2 lut4, int S0, int S1
 // Only then (and on exact ties) does the warp redo its values with the division itself; the vote keeps
 // the warp together. Rounding: adding 1.5 * 2^23 leaves the rounded integer in the low mantissa bits.
 // s > 0 and finite. Every lane of the warp must call.
-__device__ __forceinline__ void quantize_int4x16(const float (&v)[16], float s, int (&q)[16]) {
+template <int NV>
+__device__ __forceinline__ void quantize_int4(const float (&v)[NV], float s, int (&q)[NV]) {
   const float rinv = __frcp_rn(s);
   bool doubt = false;
 #pragma unroll
-  for (int e = 0; e < 16; e++) {
+  for (int e = 0; e < NV; e++) {
     const float t = fminf(fmaxf(__fmul_rn(v[e], rinv), -8.f), 7.f);
     const float biased = __fadd_rn(t, 12582912.f);
     q[e] = __float_as_int(biased) - 0x4B400000;
@@ -42,7 +43,7 @@ __device__ __forceinline__ void quantize_int4x16(const float (&v)[16], float s, 
   }
   if (__any_sync(0xffffffffu, doubt)) {
 #pragma unroll
-    for (int e = 0; e < 16; e++) q[e] = max(-8, min(7, __float2int_rn(__fdiv_rn(v[e], s))));
+    for (int e = 0; e < NV; e++) q[e] = max(-8, min(7, __float2int_rn(__fdiv_rn(v[e], s))));
   }
 }
 

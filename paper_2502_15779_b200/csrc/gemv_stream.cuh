@@ -294,7 +294,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     int q[16];
     int tsum = 0;
     if (sc != 0.f) {   // the same for the whole CTA; threads beyond the token hold zeros
-      quantize_int4x16(v, sc, q);
+      quantize_int4<16>(v, sc, q);
     } else {
 #pragma unroll
       for (int e = 0; e < 16; e++) q[e] = 0;

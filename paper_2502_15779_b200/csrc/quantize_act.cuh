@@ -242,16 +242,17 @@ __global__ void __launch_bounds__(1024) quantize_act_kernel(const QuantParams p)
   const float s = __half2float(s16);
   if (rank == 0 && tid == 0) p.scale[m] = s16;
 
+  int q[8];
+  if (s != 0.f) {   // the same for the whole cluster; threads beyond the slice hold zeros
+    quantize_int4<8>(v, s, q);
+  } else {
+#pragma unroll
+    for (int e = 0; e < 8; e++) q[e] = 0;
+  }
   if (mine) {
     uint32_t packed = 0;
-    if (s != 0.f) {
 #pragma unroll
-      for (int e = 0; e < 8; e++) {
-        int q = __float2int_rn(__fdiv_rn(v[e], s));
-        q = max(-8, min(7, q));
-        packed |= (uint32_t)(q & 0xF) << (4 * e);
-      }
-    }
+    for (int e = 0; e < 8; e++) packed |= (uint32_t)(q[e] & 0xF) << (4 * e);
     *reinterpret_cast<uint32_t*>(p.xq + (size_t)m * (p.K / 2) + base / 2) = packed;
   }
 }
@@ -365,7 +366,7 @@ __global__ void __launch_bounds__(512) quantize_act_wide_kernel(const QuantParam
   if (tid == 0) p.scale[m] = __float2half_rn(s);
   int q[16];
   if (s != 0.f) {   // the same for the whole CTA; threads beyond the token hold zeros
-    quantize_int4x16(v, s, q);
+    quantize_int4<16>(v, s, q);
   } else {
 #pragma unroll
     for (int e = 0; e < 16; e++) q[e] = 0;
