@@ -130,6 +130,13 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
   return v;
 }
+// the same with the A operand read as signed bytes
+__device__ __forceinline__ void mma_s8s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
 __device__ __forceinline__ uint2 lds64(uint32_t addr) {
   uint2 v;
   asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
@@ -409,6 +416,10 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   // operand separate the b0 and b1 planes and a mask is saved.
   constexpr bool kSign3 = (MODE == kModeDp4a);
   int accP[NTD][2][2];   // [token][row][unsigned, signed]
+  // The same on the tensor cores (per-row grid): the operand masked at bits 6,7 goes through one MMA that
+  // reads it as unsigned and one that reads it as signed bytes.
+  constexpr bool kSign3M = (MODE == kModeMma && !GRP);
+  int accPu[4], accPs[4];
   auto zero_acc = [&]() {
 #pragma unroll
     for (int f = 0; f < (NF_M == 0 ? 1 : NF_M); f++)
@@ -428,6 +439,8 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     for (int a = 0; a < NTD; a++)
 #pragma unroll
       for (int r = 0; r < 2; r++) { accP[a][r][0] = 0; accP[a][r][1] = 0; }
+#pragma unroll
+    for (int r = 0; r < 4; r++) { accPu[r] = 0; accPs[r] = 0; }
   };
   zero_acc();
 
@@ -515,8 +528,16 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
           const uint32_t av0[3] = {v0 & m0, v0 & m1, and3(v0, v0s, m1)};
           const uint32_t av1[3] = {v1 & m0, v1 & m1, and3(v1, v1s, m1)};
 #pragma unroll
-          for (int f = 0; f < NF_M; f++)
+          for (int f = 0; f < NF_M; f++) {
+            if (kSign3M && pp == 3 && f < 2) continue;
             mma_u8s8(accM[f][pp >> 1], au0[f], av0[f], au1[f], av1[f], bM[pp][0], bM[pp][1]);
+          }
+          if (kSign3M && pp == 3) {
+            const uint32_t k3 = 0xC0C0C0C0u;
+            const uint32_t ku0 = u0 & k3, kv0 = v0 & k3, ku1 = u1 & k3, kv1 = v1 & k3;
+            mma_u8s8(accPu, ku0, kv0, ku1, kv1, bM[3][0], bM[3][1]);
+            mma_s8s8(accPs, ku0, kv0, ku1, kv1, bM[3][0], bM[3][1]);
+          }
           if (kSign3 && pp == 3) {
             const uint32_t k3 = 0xC0C0C0C0u;
 #pragma unroll
@@ -691,6 +712,10 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
         T1[r] = (accM[0][0][r] >> 2) + (accM[0][1][r] >> 6);
         T2[r] = (accM[1][0][r] >> 3) + (accM[1][1][r] >> 7);
         T3[r] = (accM[2][0][r] >> 3) + (accM[2][1][r] >> 7);
+        if constexpr (kSign3M) {
+          T1[r] += (accPu[r] + accPs[r]) >> 7;
+          T2[r] += (accPu[r] - accPs[r]) >> 8;
+        }
       }
     } else {
 #pragma unroll
