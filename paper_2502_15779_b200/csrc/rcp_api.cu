@@ -78,7 +78,7 @@ long long phase_cost(int gpc, int nchunk) {
   const int KS = rcp::kCWarps / gpc;
   const int stages = (nchunk + KS - 1) / KS;
   const int per_sched = (gpc * KS + 3) / 4;
-  return (long long)stages * per_sched * 504 + 2500;
+  return (long long)stages * per_sched * 504 + 2000;
 }
 
 // A phase with the quotients the kernel would otherwise divide for.
