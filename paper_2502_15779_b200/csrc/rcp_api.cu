@@ -3,6 +3,7 @@
 
 #include <algorithm>
 #include <cmath>
+#include <cstring>
 #include <mutex>
 #include <utility>
 
@@ -225,18 +226,40 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   if (!enc) return cuda_fail(cudaErrorNotSupported);
   const StreamPlan pl = make_plan(M, N, K, sm_count(), grouped, fa ? (size_t)4 * K : 0);
   if (pl.stages < 2 || pl.smem > kSmemMax) return RCP_ERR_SHAPE;
-  rcp::GemvMaps maps;
-  const cuuint64_t gdim[2] = {(cuuint64_t)(K / 16), (cuuint64_t)N};
-  const cuuint64_t gstride[1] = {(cuuint64_t)(K / 4)};
-  const cuuint32_t estr[2] = {1, 1};
-  for (int i = 0; i < rcp::kMaxPhases; i++) {
-    const int gpc = i < pl.nphase ? pl.phase[i].gpc : 1;
-    const cuuint32_t box[2] = {(cuuint32_t)rcp::kChunkWords, (cuuint32_t)(16 * gpc)};
-    const CUresult r = enc(&maps.m[i], CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t*>(words), gdim, gstride,
-                           box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue);
+  // Tensor maps of the phases in use (the others repeat the first). Encoding one costs the host about a
+  // microsecond, so the maps of the last few (weights, shape, boxes) combinations are remembered per thread.
+  struct MapKey { const void* words; int N, K, nphase, gpc[rcp::kMaxPhases]; };
+  struct MapSlot { MapKey key; rcp::GemvMaps maps; bool used; };
+  constexpr int kMapSlots = 16;
+  thread_local MapSlot map_cache[kMapSlots] = {};
+  thread_local int map_next = 0;
+  MapKey key = {};
+  key.words = words; key.N = N; key.K = K; key.nphase = pl.nphase;
+  for (int i = 0; i < pl.nphase; i++) key.gpc[i] = pl.phase[i].gpc;
+  const rcp::GemvMaps* cached = nullptr;
+  for (int i = 0; i < kMapSlots; i++)
+    if (map_cache[i].used && std::memcmp(&map_cache[i].key, &key, sizeof(MapKey)) == 0) { cached = &map_cache[i].maps; break; }
+  if (!cached) {
+    MapSlot& slot = map_cache[map_next];
+    map_next = (map_next + 1) % kMapSlots;
+    slot.used = false;
+    const cuuint64_t gdim[2] = {(cuuint64_t)(K / 16), (cuuint64_t)N};
+    const cuuint64_t gstride[1] = {(cuuint64_t)(K / 4)};
+    const cuuint32_t estr[2] = {1, 1};
+    for (int i = 0; i < rcp::kMaxPhases; i++) {
+      if (i >= pl.nphase && i > 0) { slot.maps.m[i] = slot.maps.m[0]; continue; }
+      const int gpc = i < pl.nphase ? pl.phase[i].gpc : 1;
+      const cuuint32_t box[2] = {(cuuint32_t)rcp::kChunkWords, (cuuint32_t)(16 * gpc)};
+      const CUresult r = enc(&slot.maps.m[i], CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t*>(words), gdim,
+                             gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+      if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue);
+    }
+    slot.key = key;
+    slot.used = true;
+    cached = &slot.maps;
   }
+  const rcp::GemvMaps& maps = *cached;
   rcp::GemvParams gp;
   gp.lut = static_cast<const uint2*>(lut_f16);
   gp.xq = xq;
