@@ -81,7 +81,9 @@ int rcp_quantize_act(const void* x_f16, int M, int K, int had_block, float clip_
  *                    with dp4a, two tokens per launch.
  *   RCP_GEMV_MMA     streaming kernel with the masked code planes as the A operand of int8 mma.sync,
  *                    up to eight tokens per launch (fewer when K is so long that their expanded
- *                    activations would not fit in shared memory); for one or two tokens the b0*b1
+ *                    activations would not fit in shared memory); nine to sixteen tokens go in one
+ *                    launch (two MMA column tiles fed from the same masks) while M * K <= 80 KiB,
+ *                    else in launches of eight at most; for one or two tokens the b0*b1
  *                    plane is computed with dp4a beside the tensor cores.
  *   RCP_GEMV_MMA_ONLY  as RCP_GEMV_MMA with all three planes on the tensor cores for every M.
  * The streaming kernel: persistent CTAs, weights through a TMA/mbarrier shared-memory ring, 16-row

@@ -183,7 +183,8 @@ __device__ __forceinline__ void dp4a_s8s8(int& d, uint32_t a, uint32_t b) {
 
 // MODE  kModeMma: all three planes on the tensor cores; kModeHybrid: b0 and b1 planes on the tensor
 //       cores, the b0*b1 plane on dp4a; kModeDp4a: everything on dp4a (CUDA cores only)
-// MTOK  tokens, fixed at compile time for the dp4a modes (1 or 2); 0 = run-time, up to 8 (kModeMma)
+// MTOK  tokens, fixed at compile time for the dp4a modes (1 or 2); kModeMma: 0 = run-time, up to 8
+//       (one MMA column tile), 16 = run-time, 9 to 16 (two column tiles fed from the same masks)
 // GRP   one grid per group of 128 weights instead of one per row (kModeHybrid has no such form)
 // FQ    one token of 4096 or 8192 activations under one rotation block: the activations arrive as
 //       fp16 and every CTA rotates and quantizes them itself (Appendix A.2, Section 4.4), in the
@@ -201,7 +202,9 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   uint8_t* const gen = smem_raw + (base - raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t = lane & 3;
-  const int M = (MTOK > 0) ? MTOK : p.M;
+  const int M = (MTOK > 0 && MODE != kModeMma) ? MTOK : p.M;
+  constexpr bool kTwoTiles = (MODE == kModeMma && MTOK == 16);   // tokens 8..15 in a second set of accumulators
+  static_assert(!(kTwoTiles && (GRP || FQ)), "two column tiles: per-row grid, quantized activations only");
   const int ncol = M;
   const int stages = p.stages;
   const uint32_t full0 = base + p.off_bar, empty0 = full0 + 8 * kMaxStages;
@@ -220,11 +223,11 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   const int b = blockIdx.x;
   // Launched with programmatic stream serialization: the next kernel may start as CTAs retire.
   asm volatile("griddepcontrol.launch_dependents;");
-  int* const s_T0tot = reinterpret_cast<int*>(s_scale + 24);   // [8]: sum of q per token, behind scales and maxima
+  int* const s_T0tot = reinterpret_cast<int*>(s_scale + 32);   // [16]: sum of q per token, behind scales and maxima
   // The producer warp sets up the ring's barriers and only announces that (bar.arrive): its first
   // requests go out without waiting for anybody. The consumer warps wait for the announcement.
   if (warp != kCWarps) {
-    if (tid < 8) s_T0tot[tid] = 0;
+    if (tid < kMaxTokens) s_T0tot[tid] = 0;
     asm volatile("bar.sync 3, %0;" ::"n"(kGThreads) : "memory");
   }
 
@@ -291,7 +294,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     constexpr int NT = kCWarps * 32;
     const int W = p.K / 16;                                           // 256 or 512 words: one per thread
     float* const qbuf = reinterpret_cast<float*>(gen + p.off_qbuf);   // [16][W]
-    float* const s_amax = s_scale + 8;                                // [16 warps] behind the scales
+    float* const s_amax = s_scale + 16;                               // [16 warps] behind the scales
     float v[16];
     const float sc = rotate_token_words<NT>(p.x, W, p.inv_sqrt_b, p.clip_ratio, qbuf, s_amax, v);
     if (tid == 0) {
@@ -353,16 +356,29 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   {
     const int W = p.K / 16;
     const int total = ncol * p.nchunk * 16;
+    // the two words of unit u (zeros past the end of the row or of the units)
+    auto load_unit = [&](int u) {
+      const int pair = u >> 4;
+      const int col = (int)(((uint32_t)pair * (uint32_t)p.inv_nchunk) >> 20), ch = pair - col * p.nchunk;   // pair / nchunk
+      const int lo = u & 3, hi = (u >> 2) & 3;
+      const int wx = ch * kChunkWords + (kRelabel ? 8 * hi + 2 * lo : 8 * lo + 2 * hi);   // word index in the row
+      uint4 x = make_uint4(0, 0, 0, 0);
+      if (u < total && wx < W) x = __ldg(reinterpret_cast<const uint4*>(p.xq + (size_t)col * (p.K / 2)) + (wx >> 1));
+      return x;
+    };
+    // per-row grid: the next unit's words are fetched while this one is expanded (the group-wise
+    // kernels have no registers to spare for that)
+    uint4 x_next = make_uint4(0, 0, 0, 0);
+    if constexpr (!GRP) x_next = load_unit(warp * 32 + lane);
     for (int u0 = warp * 32; u0 < total; u0 += kCWarps * 32) {
       const int u = u0 + lane;
       int tsum = 0;
       const int pair = u >> 4;
       const int col = (int)(((uint32_t)pair * (uint32_t)p.inv_nchunk) >> 20), ch = pair - col * p.nchunk;   // pair / nchunk
+      const uint4 x = GRP ? load_unit(u) : x_next;
+      if constexpr (!GRP) x_next = load_unit(u + kCWarps * 32);
       if (u < total) {
         const int lo = u & 3, hi = (u >> 2) & 3;   // lo: 16-byte slot t of the column block; hi: 2 i + pr, or the group
-        const int wx = ch * kChunkWords + (kRelabel ? 8 * hi + 2 * lo : 8 * lo + 2 * hi);   // word index in the row
-        uint4 x = make_uint4(0, 0, 0, 0);
-        if (wx < W) x = __ldg(reinterpret_cast<const uint4*>(p.xq + (size_t)col * (p.K / 2)) + (wx >> 1));
         uint32_t q[4][2];
 #pragma unroll
         for (int w = 0; w < 2; w++) {
@@ -410,6 +426,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   constexpr int NF_D = (MODE == kModeDp4a) ? 3 : (MODE == kModeHybrid ? 1 : 0);  // planes on dp4a
   constexpr int NTD = (NF_D == 0) ? 1 : MTOK;
   int accM[NF_M == 0 ? 1 : NF_M][2][4];
+  int accN[kTwoTiles ? 3 : 1][1][4];   // second column tile
   int accD[NTD][2][NF_D == 0 ? 1 : NF_D][2];
   // kModeDp4a: position 3 sits in bits 6 and 7 of a byte. One mask keeps both; read as unsigned
   // bytes they weigh 64 b0 + 128 b1, read as signed bytes 64 b0 - 128 b1, so two dp4a on the same
@@ -418,7 +435,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   int accP[NTD][2][2];   // [token][row][unsigned, signed]
   // The same on the tensor cores (per-row grid): the operand masked at bits 6,7 goes through one MMA that
   // reads it as unsigned and one that reads it as signed bytes.
-  constexpr bool kSign3M = (MODE == kModeMma && !GRP);
+  constexpr bool kSign3M = (MODE == kModeMma && !GRP && !kTwoTiles);   // two tiles: no registers for its accumulators
   int accPu[4], accPs[4];
   auto zero_acc = [&]() {
 #pragma unroll
@@ -441,23 +458,27 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
       for (int r = 0; r < 2; r++) { accP[a][r][0] = 0; accP[a][r][1] = 0; }
 #pragma unroll
     for (int r = 0; r < 4; r++) { accPu[r] = 0; accPs[r] = 0; }
+#pragma unroll
+    for (int f = 0; f < (kTwoTiles ? 3 : 1); f++)
+#pragma unroll
+      for (int r = 0; r < 4; r++) accN[f][0][r] = 0;
   };
   zero_acc();
 
   // (row, token) entries this lane emits.
-  // kModeMma:   lane (g,t) owns tokens 2t, 2t+1 for rows g and g+8.
+  // kModeMma:   lane (g,t) owns tokens 2t, 2t+1 (and 8+2t, 9+2t with two column tiles) for rows g and g+8.
   // dp4a modes: MMA columns repeat the tokens (column c carries token c % MTOK); dp4a partial sums
   //             are reduced over the quad and lane t==0 owns tokens 0..MTOK-1 for rows g and g+8.
-  constexpr int NE = (MODE == kModeMma) ? 4 : 2 * NTD;
+  constexpr int NE = (MODE == kModeMma) ? (kTwoTiles ? 8 : 4) : 2 * NTD;
   int etok[NE], err[NE], T0v[NE];
 #pragma unroll
   for (int e = 0; e < NE; e++) {
-    if constexpr (MODE == kModeMma) { etok[e] = 2 * t + (e & 1); err[e] = e >> 1; }
+    if constexpr (MODE == kModeMma) { etok[e] = 8 * (e >> 2) + 2 * t + (e & 1); err[e] = (e >> 1) & 1; }
     else { etok[e] = (t == 0) ? (e >> 1) : kMaxTokens; err[e] = e & 1; }
     T0v[e] = 0;
   }
   // T0 of the tokens this lane emits (added up while the activations were expanded)
-  if constexpr (!GRP) {
+  if constexpr (!GRP && !kTwoTiles) {   // two tiles: read when needed, the registers are taken
 #pragma unroll
     for (int e = 0; e < NE; e++) if (etok[e] < M) T0v[e] = s_T0tot[etok[e]];
   }
@@ -476,6 +497,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     else if (col >= M) col = M - 1;
     bM_lane = (uint32_t)(col * 64 + t * 16);
   }
+  const uint32_t bN_lane = (uint32_t)(min(8 + g, M - 1) * 64 + t * 16);   // column of the second tile
 #pragma unroll
   for (int tok = 0; tok < NTD; tok++) bD_lane[tok] = (uint32_t)(tok * 64 + t * 16);
 
@@ -515,22 +537,38 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
             bM[2][0] = y.x; bM[2][1] = y.y; bM[3][0] = y.z; bM[3][1] = y.w;
           }
         }
+        uint32_t bN[4][2];
+        if constexpr (kTwoTiles) {
+          const uint4 x = lds128(b_ptr + bN_lane + b_off);
+          const uint4 y = lds128(b_ptr + bN_lane + b_off + half_stride);
+          bN[0][0] = x.x; bN[0][1] = x.y; bN[1][0] = x.z; bN[1][1] = x.w;
+          bN[2][0] = y.x; bN[2][1] = y.y; bN[3][0] = y.z; bN[3][1] = y.w;
+        }
         const uint32_t u0 = uw[2 * pr], u1 = uw[2 * pr + 1], v0 = vw[2 * pr], v1 = vw[2 * pr + 1];
         const uint32_t u0s = u0 + u0, u1s = u1 + u1, v0s = v0 + v0, v1s = v1 + v1;  // b0 moved onto b1's bit
 #pragma unroll
         for (int po = 0; po < 4; po++) {
           // positions in the order 0, 2, 1, 3: consecutive iterations feed different accumulators
           const int pp = ((po & 1) << 1) | (po >> 1);
-          const uint32_t m0 = 0x01010101u << (2 * pp), m1 = m0 << 1;
+          // Two column tiles: positions 2 and 3 are moved down onto the bits of 0 and 1 first, so that all
+          // four positions add into one set of accumulators (there are no registers for two sets per tile).
+          const bool down = kTwoTiles && pp >= 2;
+          const uint32_t m0 = 0x01010101u << (2 * (down ? pp - 2 : pp)), m1 = m0 << 1;
+          const uint32_t w_u0 = down ? u0 >> 4 : u0, w_u1 = down ? u1 >> 4 : u1;
+          const uint32_t w_v0 = down ? v0 >> 4 : v0, w_v1 = down ? v1 >> 4 : v1;
+          const uint32_t s_u0 = down ? w_u0 + w_u0 : u0s, s_u1 = down ? w_u1 + w_u1 : u1s;
+          const uint32_t s_v0 = down ? w_v0 + w_v0 : v0s, s_v1 = down ? w_v1 + w_v1 : v1s;
           // the three planes of the four words: b0, b1, b0*b1 (the last two scaled by 2)
-          const uint32_t au0[3] = {u0 & m0, u0 & m1, and3(u0, u0s, m1)};
-          const uint32_t au1[3] = {u1 & m0, u1 & m1, and3(u1, u1s, m1)};
-          const uint32_t av0[3] = {v0 & m0, v0 & m1, and3(v0, v0s, m1)};
-          const uint32_t av1[3] = {v1 & m0, v1 & m1, and3(v1, v1s, m1)};
+          const uint32_t au0[3] = {w_u0 & m0, w_u0 & m1, and3(w_u0, s_u0, m1)};
+          const uint32_t au1[3] = {w_u1 & m0, w_u1 & m1, and3(w_u1, s_u1, m1)};
+          const uint32_t av0[3] = {w_v0 & m0, w_v0 & m1, and3(w_v0, s_v0, m1)};
+          const uint32_t av1[3] = {w_v1 & m0, w_v1 & m1, and3(w_v1, s_v1, m1)};
 #pragma unroll
           for (int f = 0; f < NF_M; f++) {
             if (kSign3M && pp == 3 && f < 2) continue;
-            mma_u8s8(accM[f][pp >> 1], au0[f], av0[f], au1[f], av1[f], bM[pp][0], bM[pp][1]);
+            const int half = kTwoTiles ? 0 : pp >> 1;
+            mma_u8s8(accM[f][half], au0[f], av0[f], au1[f], av1[f], bM[pp][0], bM[pp][1]);
+            if constexpr (kTwoTiles) mma_u8s8(accN[f][0], au0[f], av0[f], au1[f], av1[f], bN[pp][0], bN[pp][1]);
           }
           if (kSign3M && pp == 3) {
             const uint32_t k3 = 0xC0C0C0C0u;
@@ -717,6 +755,14 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
           T2[r] += (accPu[r] - accPs[r]) >> 8;
         }
       }
+      if constexpr (kTwoTiles) {
+#pragma unroll
+        for (int r = 0; r < 4; r++) {
+          T1[4 + r] = accN[0][0][r] >> 2;   // one set of accumulators: accM[.][1] stayed zero above
+          T2[4 + r] = accN[1][0][r] >> 3;
+          T3[4 + r] = accN[2][0][r] >> 3;
+        }
+      }
     } else {
 #pragma unroll
       for (int tok = 0; tok < NTD; tok++)
@@ -756,7 +802,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
       const int row = row_first + g + 8 * err[e];
       if (etok[e] < M && row < p.N) {
         const int S3 = T3[e], S1 = T1[e] - T3[e], S2 = T2[e] - T3[e];
-        const int S0 = T0v[e] - S1 - S2 - S3;
+        const int S0 = (kTwoTiles ? s_T0tot[etok[e]] : T0v[e]) - S1 - S2 - S3;
         p.y[(size_t)etok[e] * p.N + row] = lut_finish(s_scale[etok[e]], lut_g[err[e]], S0, S1, S2, S3);
       }
     }

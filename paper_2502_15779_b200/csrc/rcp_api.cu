@@ -65,9 +65,15 @@ struct StreamPlan {
 
 constexpr size_t kSmemMax = 232448;            // 227 KB of dynamic shared memory per CTA on sm_100
 constexpr size_t kExpandBudget = 128 * 1024;   // expanded activations (one byte per code and token) per CTA
+constexpr size_t kExpandBudgetTwoTiles = 80 * 1024;   // the same with 9 to 16 tokens (their reduction buffers are larger)
 
 // Tokens one launch can take: their expanded activations must fit beside a ring of three stages.
+// cap 16: the tensor-core kernel with two column tiles takes 9 to 16 tokens at once where they fit.
 int tokens_per_pass(int M, int K, int cap) {
+  if (cap > 8) {
+    if (M > 8 && (size_t)M * K <= kExpandBudgetTwoTiles) return M;
+    cap = 8;
+  }
   int m = std::min(M, cap);
   while (m > 1 && (size_t)m * K > kExpandBudget) m--;
   return m;
@@ -148,12 +154,12 @@ StreamPlan make_plan(int M, int N, int K, int sms, bool grouped = false, size_t 
   // row groups x 3 planes, or (group-wise grid) one fp32 term per warp
   const size_t t0c_bytes = grouped ? (size_t)(M + 1) * pl.nchunk * 16 : (((size_t)M * pl.nchunk * 4) + 15) / 16 * 16;
   const size_t red_bytes = grouped ? (size_t)2 * rcp::kCWarps * 16 * M * 4 : (size_t)2 * 8 * 16 * M * 3 * 4;
-  const size_t misc = 128 + t0c_bytes + 128 + red_bytes + qbuf;
+  const size_t misc = 128 + t0c_bytes + 256 + red_bytes + qbuf;
   pl.stages = (int)std::min<size_t>(rcp::kMaxStages, (kSmemMax - 1024 - misc - bs_bytes) / rcp::kStageBytes);
   size_t off = (size_t)pl.stages * rcp::kStageBytes;
   pl.off_bar = (int)off; off += 128;
   pl.off_T0c = (int)off; off += t0c_bytes;
-  pl.off_scale = (int)off; off += 128;   // 8 scales, then 16 per-warp maxima of the fused quantizer
+  pl.off_scale = (int)off; off += 256;   // 16 scales, 16 per-warp maxima of the fused quantizer, 16 token totals
   pl.off_red = (int)off; off += red_bytes;
   pl.off_bs = (int)off; off += bs_bytes;
   pl.off_qbuf = (int)off; off += qbuf;
@@ -219,7 +225,7 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
                   int M, int N, int K, void* y_f16, void* workspace, cudaStream_t st, bool grouped = false,
                   const FusedAct* fa = nullptr) {
   if (mode != rcp::kModeMma && M > 2) return RCP_ERR_VARIANT;
-  if (M > 8) return RCP_ERR_VARIANT;
+  if (M > 8 && (grouped || fa || M > rcp::kMaxTokens)) return RCP_ERR_VARIANT;
   if (grouped && (mode == rcp::kModeHybrid || K % 128)) return RCP_ERR_VARIANT;
   if (fa && (mode != rcp::kModeDp4a || !fused_ok(M, K, fa->B))) return RCP_ERR_VARIANT;
   EncodeTiledFn enc = encode_tiled_fn();
@@ -301,7 +307,7 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   if (mode == rcp::kModeDp4a)
     return M == 1 ? launch_stream_t<rcp::kModeDp4a, 1>(maps, gp, pl, st)
                   : launch_stream_t<rcp::kModeDp4a, 2>(maps, gp, pl, st);
-  return launch_stream_t<rcp::kModeMma, 0>(maps, gp, pl, st);
+  return M > 8 ? launch_stream_t<rcp::kModeMma, 16>(maps, gp, pl, st) : launch_stream_t<rcp::kModeMma, 0>(maps, gp, pl, st);
 }
 
 // All M tokens: as many launches as it takes for the expanded activations to fit (`cap` tokens at most each).
@@ -487,7 +493,7 @@ int rcp_gemv_plan(int M, int N, int K, int sms, int* out, int cap) {
   if (!out && cap > 0) return RCP_ERR_NULL;
   if (M < 1 || M > rcp::kMaxTokens || N < 1 || !k_ok(K)) return RCP_ERR_SHAPE;
   if (sms <= 0) sms = 148;
-  const int mp = tokens_per_pass(M, K, 8);
+  const int mp = tokens_per_pass(M, K, 16);
   const StreamPlan pl = make_plan(mp, N, K, sms);
   int v[6 + 5 * rcp::kMaxPhases];
   int n = 0;
@@ -535,10 +541,10 @@ int rcp_gemv_w2a4_variant(int variant, const uint32_t* words, const void* lut_f1
     }
     case RCP_GEMV_MMA:
       // tensor-core path; for one or two tokens the b0*b1 plane goes to dp4a (FMA pipe) instead
-      return launch_stream_passes(M <= 2 ? rcp::kModeHybrid : rcp::kModeMma, 8, words, lut_f16, xq, scale_f16, M, N, K,
+      return launch_stream_passes(M <= 2 ? rcp::kModeHybrid : rcp::kModeMma, 16, words, lut_f16, xq, scale_f16, M, N, K,
                                   y_f16, workspace, st);
     case RCP_GEMV_MMA_ONLY:
-      return launch_stream_passes(rcp::kModeMma, 8, words, lut_f16, xq, scale_f16, M, N, K, y_f16, workspace, st);
+      return launch_stream_passes(rcp::kModeMma, 16, words, lut_f16, xq, scale_f16, M, N, K, y_f16, workspace, st);
     case RCP_GEMV_DP4A:
       // CUDA-core path: two tokens per launch
       return launch_stream_passes(rcp::kModeDp4a, 2, words, lut_f16, xq, scale_f16, M, N, K, y_f16, workspace, st);
@@ -617,7 +623,7 @@ int rcp_linear_w2a4_launches(int M, int K, int had_block, int group) {
   const int B = had_block <= 1 ? 1 : had_block;
   if (fused_ok(M, K, B) && (group == 0 || group == 128)) return 1;
   if (group != 0 && group != 128) return 2;
-  const int cap = group == 0 ? (M == 1 ? 2 : 8) : (M <= 2 ? 2 : 8);   // tokens per launch of the variant AUTO picks
+  const int cap = group == 0 ? (M == 1 ? 2 : 16) : (M <= 2 ? 2 : 8);   // tokens per launch of the variant AUTO picks
   const int mp = tokens_per_pass(M, K, cap);
   return 1 + (M + mp - 1) / mp;
 }

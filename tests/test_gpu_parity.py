@@ -110,6 +110,9 @@ def _check_gemv(N, K, B, M, kind, variant, seed, rows=None):
     assert np.array_equal(words_np(words)[sel], w_ref)
     ref = oracle.gemv_w2a4(w_ref, f16_bits(lut)[sel], qa["xq"], qa["scale"])
     assert np.array_equal(S.cpu().numpy()[:, sel, :], ref["S"])
+    # y_dbg comes from the kernel that exported the S_c just checked. Every variant finishes its own integer
+    # sums with the same fp32 steps, so equal bits here mean the variant's S_c are the exact ones as well.
+    assert torch.equal(y.view(torch.int16), y_dbg.view(torch.int16)), "variant's sums differ from the exported S_c"
     for out in (y, y_dbg):
         got = out.float().cpu().numpy().astype(np.float64)[:, sel]
         err = np.abs(got - ref["y"])
@@ -123,6 +126,9 @@ SMALL = [
     (1, 64, 64, 1), (8, 64, 1, 1), (16, 128, 128, 1), (17, 192, 64, 3), (100, 320, 64, 2), (129, 512, 512, 1),
     (127, 1024, 128, 16), (300, 2048, 2048, 1), (256, 4096, 4096, 4), (130, 11008, 128, 1), (64, 28672, 128, 1),
     (40, 14336, 128, 16), (33, 8192, 8192, 8), (2048, 2048, 2048, 1), (513, 1088, 64, 5), (1000, 2560, 128, 7),
+    # 9 to 16 tokens in one launch (two column tiles) where they fit, in two launches where they do not
+    (2500, 4096, 4096, 9), (5000, 2048, 128, 13), (300, 6144, 128, 13), (70, 5120, 64, 16), (70, 5184, 64, 16),
+    (37965, 512, 128, 16), (2369, 1024, 1024, 12),
 ]
 
 

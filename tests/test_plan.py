@@ -46,8 +46,10 @@ def check(L, M, N, K, sms=148):
     assert len(p["phases"]) <= 6
     assert p["nchunk"] == -(-K // 512)
     assert p["stages"] >= 2 and p["smem"] <= 232448
-    assert 1 <= p["tokens"] <= 8 and p["tokens"] * p["launches"] >= M
+    assert 1 <= p["tokens"] <= 16 and p["tokens"] * p["launches"] >= M
     assert p["tokens"] == 1 or p["tokens"] * K <= 128 * 1024   # expanded activations fit
+    if p["tokens"] > 8:   # one launch with two column tiles: all the tokens, and a tighter budget
+        assert p["tokens"] == M and p["launches"] == 1 and M * K <= 80 * 1024 and p["stages"] >= 3
     return p
 
 
@@ -73,8 +75,13 @@ def test_plan_examples(L):
     assert p["phases"][-1] == (16, 1216, 2368, 148, 1)
     assert p["phases"][0][0] == 8 and p["phases"][0][2] == 8 * 148
     assert sum(t * r for _, _, t, _, r in p["phases"][:-1]) == 1216
-    # sixteen tokens go in two launches of eight; long K cuts the tokens per launch further
-    assert (check(L, 16, 4096, 4096)["tokens"], check(L, 16, 4096, 4096)["launches"]) == (8, 2)
+    # nine to sixteen tokens go in one launch while their expanded activations stay within 80 KB, otherwise
+    # in launches of eight at most; long K cuts the tokens per launch further
+    assert (check(L, 16, 4096, 4096)["tokens"], check(L, 16, 4096, 4096)["launches"]) == (16, 1)
+    assert (check(L, 16, 4096, 5120)["tokens"], check(L, 16, 4096, 5120)["launches"]) == (16, 1)
+    assert (check(L, 10, 4096, 8192)["tokens"], check(L, 10, 4096, 8192)["launches"]) == (10, 1)
+    assert (check(L, 16, 4096, 5184)["tokens"], check(L, 16, 4096, 5184)["launches"]) == (8, 2)
+    assert (check(L, 16, 4096, 11008)["tokens"], check(L, 16, 4096, 11008)["launches"]) == (8, 2)
     assert check(L, 8, 8192, 28672)["tokens"] == 4
     assert check(L, 16, 64, 65536)["tokens"] == 2
 
