@@ -248,3 +248,33 @@ def ldp_export(w_f16_bits, sb, sg, s1, s2, G):
     if rc:
         raise ValueError(f"orc_ldp_export failed: {rc}")
     return dict(codes=codes, lut=lut)
+
+
+def gemv_w2a16(words, lut_bits, x_f16_bits):
+    """Weight-only GEMV by its definition. Returns dict(y float64 [M][N], labsx float64 [M][N], labs float64 [N])."""
+    words = _c(words, np.uint32)
+    lut = _c(lut_bits, np.uint16)
+    x = _c(x_f16_bits, np.uint16)
+    N, W = words.shape
+    K = W * 16
+    M = x.shape[0]
+    assert x.shape == (M, K) and lut.shape == (N, 4)
+    y = np.empty((M, N), dtype=np.float64)
+    labsx = np.empty((M, N), dtype=np.float64)
+    labs = np.empty((N,), dtype=np.float64)
+    rc = lib().orc_gemv_w2a16(_p(words), _p(lut), _p(x), C.c_int(M), C.c_int(N), C.c_int(K), _p(y), _p(labsx), _p(labs))
+    if rc:
+        raise ValueError(f"orc_gemv_w2a16 failed: {rc}")
+    return dict(y=y, labsx=labsx, labs=labs)
+
+
+def split_act16(x_f16_bits):
+    """Base-64 fixed-point digits of fp16 activations. Returns dict(digits int8 [M][4][K], unit float64 [M][4])."""
+    x = _c(x_f16_bits, np.uint16)
+    M, K = x.shape
+    digits = np.empty((M, 4, K), dtype=np.int8)
+    unit = np.empty((M, 4), dtype=np.float64)
+    rc = lib().orc_split_act16(_p(x), C.c_int(M), C.c_int(K), _p(digits), _p(unit))
+    if rc:
+        raise ValueError(f"orc_split_act16 failed: {rc}")
+    return dict(digits=digits, unit=unit)

@@ -27,6 +27,10 @@
 // partitioning quantizer: hand-computed fixture, the uniform initial point == the textbook
 // asymmetric 2-bit quantizer, the range ends and bin centres the paper states, monotone codes,
 // the sum form of the dequantizer == LUT lookup.
+// Weight-only variant: equals the W2A4 oracle when the activations are integers times a power of
+// two; affine grid == plain matrix product; brute force; the fixed-point digits reproduce the
+// activations (exactly for elements within 2^-11 of the token's maximum, to half a unit otherwise)
+// and a hand-written case.
 // fp16 output y: the paper prints no worked numeric GEMV example, so y is pinned only by the
 // mathematical identities above, not by a printed value.
 #include <cstdint>
@@ -534,6 +538,85 @@ int orc_ldp_export(const uint16_t* w_f16, const float* sb, const float* sg, cons
         codes[(size_t)n * K + (size_t)j * G + k] = (uint8_t)code;
       }
     }
+  return 0;
+}
+
+// ---------------------------------------------------------------------------------------
+// Weight-only variant (Section 5, "W2-only setting", Table "W2_inference": the GEMV with the
+// 2-bit codes and the dequantization grid of Section 4.4 but activations left in 16-bit floating
+// point). The plain definition, in double, the sum over k taken in order:
+//   y[m][n]    = sum_k LUT[n][code[n][k]] * x[m][k]
+//   labsx[m][n] = sum_k |LUT[n][code[n][k]]| * |x[m][k]|     (magnitude the tolerance refers to)
+//   labs[n]    = sum_k |LUT[n][code[n][k]]|
+// x is fp16 [M][K]. Returns 0; -1 bad shape.
+// ---------------------------------------------------------------------------------------
+int orc_gemv_w2a16(const uint32_t* words, const uint16_t* lut_f16, const uint16_t* x_f16, int M, int N, int K,
+                   double* y, double* labsx, double* labs) {
+  if (M < 1 || N < 1 || K < 16 || K % 16) return -1;
+  uint8_t* codes = (uint8_t*)std::malloc((size_t)K);
+  for (int n = 0; n < N; n++) {
+    orc_unpack_weights(words + (size_t)n * (K / 16), 1, K, codes);
+    double L[4];
+    for (int c = 0; c < 4; c++) L[c] = (double)orc_f16_to_f32(lut_f16[(size_t)n * 4 + c]);
+    double la = 0.0;
+    for (int k = 0; k < K; k++) la += std::fabs(L[codes[k]]);
+    if (labs) labs[n] = la;
+    for (int m = 0; m < M; m++) {
+      double acc = 0.0, mag = 0.0;
+      for (int k = 0; k < K; k++) {
+        const double xv = (double)orc_f16_to_f32(x_f16[(size_t)m * K + k]);
+        acc += L[codes[k]] * xv;
+        mag += std::fabs(L[codes[k]]) * std::fabs(xv);
+      }
+      y[(size_t)m * N + n] = acc;
+      if (labsx) labsx[(size_t)m * N + n] = mag;
+    }
+  }
+  std::free(codes);
+  return 0;
+}
+
+// Block fixed point of a token of fp16 activations, as base-64 digits (an encoding chosen by this
+// implementation of the weight-only variant, not by the paper: it lets 16-bit activations run
+// through exact 8-bit integer dot products). Per token m, with E = floor(log2(max_k |x[m][k]|))
+// (E = 0 for an all-zero token):
+//   X[k]   = round-half-even( x[m][k] * 2^(21 - E) )              an integer, |X| < 2^22
+//   X[k]   = sum_{d=0..3} 64^d * q_d[k],  q_0..q_2 in [-32, 31] taken least significant first,
+//            q_3 what remains (within [-16, 16])
+//   unit_d = 2^(E - 21) * 64^d
+// digits int8 [M][4][K] (digit-major per token), unit double [M][4]. Returns 0; -1 bad shape;
+// -2 if an activation is not finite.
+int orc_split_act16(const uint16_t* x_f16, int M, int K, int8_t* digits, double* unit) {
+  if (M < 1 || K < 1) return -1;
+  for (int m = 0; m < M; m++) {
+    double amax = 0.0;
+    for (int k = 0; k < K; k++) {
+      const double v = std::fabs((double)orc_f16_to_f32(x_f16[(size_t)m * K + k]));
+      if (!(v <= 65504.0)) return -2;
+      if (v > amax) amax = v;
+    }
+    int E = 0;
+    if (amax > 0.0) {
+      int e2 = 0;
+      (void)std::frexp(amax, &e2);   // amax = f * 2^e2 with f in [0.5, 1)
+      E = e2 - 1;
+    }
+    for (int d = 0; d < 4; d++) unit[(size_t)m * 4 + d] = std::ldexp(1.0, E - 21 + 6 * d);
+    for (int k = 0; k < K; k++) {
+      const double v = (double)orc_f16_to_f32(x_f16[(size_t)m * K + k]);
+      long long X = (long long)std::nearbyint(std::ldexp(v, 21 - E));   // default rounding mode: half to even
+      for (int d = 0; d < 4; d++) {
+        long long q;
+        if (d < 3) {
+          q = ((X + 32) % 64 + 64) % 64 - 32;   // the residue of X in [-32, 31]
+          X = (X - q) / 64;
+        } else {
+          q = X;
+        }
+        digits[((size_t)m * 4 + d) * K + k] = (int8_t)q;
+      }
+    }
+  }
   return 0;
 }
 

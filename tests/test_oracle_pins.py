@@ -586,3 +586,95 @@ def test_ldp_degenerate_unit_and_planted_mistakes():
     assert not np.array_equal(a["codes"], b["codes"]) and not np.array_equal(a["lut"], c["lut"])
     with pytest.raises((ValueError, AssertionError)):
         oracle.ldp_export(f16_bits(w), one, one, one, one, 48)
+
+
+# ----------------------------------------------------------------------------- weight-only variant
+def _problem16(N, K, M, seed, kind="uniform"):
+    codes, lut = synth.make_layer(N, K, 1, kind, seed)
+    x = synth.make_activations(M, K, seed)
+    return codes.numpy(), lut, oracle.pack_weights(codes.numpy()), x
+
+
+def test_w2a16_brute_force_small_and_planted_mistakes():
+    codes, lut, words, x = _problem16(16, 32, 2, seed=5)
+    r = oracle.gemv_w2a16(words, f16_bits(lut), f16_bits(x))
+    lutf, xf = lut.numpy().astype(np.float64), x.numpy().astype(np.float64)
+    for m in range(2):
+        for n in range(16):
+            acc = mag = 0.0
+            for k in range(32):
+                acc += lutf[n, codes[n, k]] * xf[m, k]
+                mag += abs(lutf[n, codes[n, k]]) * abs(xf[m, k])
+            assert r["y"][m, n] == pytest.approx(acc, rel=1e-14, abs=0)
+            assert r["labsx"][m, n] == pytest.approx(mag, rel=1e-14)
+    assert np.allclose(r["labs"], np.abs(np.take_along_axis(lutf, codes.astype(np.int64), axis=1)).sum(axis=1), rtol=1e-14)
+    # reversed activations or a reversed code order change the result
+    r_rev = oracle.gemv_w2a16(words, f16_bits(lut), f16_bits(x.flip(1).contiguous()))
+    assert not np.allclose(r["y"], r_rev["y"], rtol=1e-6)
+    rev = oracle.pack_weights(np.ascontiguousarray(codes.reshape(16, 2, 16)[:, :, ::-1].reshape(16, 32)))
+    assert not np.allclose(r["y"], oracle.gemv_w2a16(rev, f16_bits(lut), f16_bits(x))["y"], rtol=1e-6)
+
+
+def test_w2a16_equals_the_w2a4_oracle_on_integer_activations():
+    # activations that are int4 values times a power of two: both definitions describe the same product
+    N, K, M = 40, 512, 3
+    codes, lut, words, qa = _problem(N, K, M, seed=31, kind="rotated_laplace", B=64)
+    s = np.array([0.25, 2.0 ** -9, 8.0])
+    x = torch.tensor(qa["q"].astype(np.float64) * s[:, None], dtype=torch.float16)
+    assert np.array_equal(x.numpy().astype(np.float64), qa["q"] * s[:, None])      # exact in fp16
+    r4 = oracle.gemv_w2a4(words, f16_bits(lut), qa["xq"], f16_bits(torch.tensor(s, dtype=torch.float16)))
+    r16 = oracle.gemv_w2a16(words, f16_bits(lut), f16_bits(x))
+    assert np.allclose(r16["y"], r4["y"], rtol=1e-11, atol=1e-13)
+    # and the magnitude sums: sum_k |L||x| >= s * sum_c |L_c||S_c| (no cancellation inside a code's sum)
+    assert np.all(r16["labsx"] >= (r4["tol"] - 1e-5) / 2e-3 * (1 - 1e-12))
+
+
+def test_w2a16_affine_grid_is_a_plain_matrix_product_and_matches_dense_dequantization():
+    N, K, M = 48, 320, 2
+    codes, lut, words, x = _problem16(N, K, M, seed=12)
+    a, d = 0.125, 0.03125
+    lut_aff = torch.tensor([[a + c * d for c in range(4)]] * N, dtype=torch.float16)
+    xf = x.numpy().astype(np.float64)
+    r = oracle.gemv_w2a16(words, f16_bits(lut_aff), f16_bits(x))
+    assert np.allclose(r["y"], a * xf.sum(axis=1)[:, None] + d * (xf @ codes.astype(np.float64).T), rtol=1e-11, atol=1e-12)
+    Wd = np.take_along_axis(lut.numpy().astype(np.float64), codes.astype(np.int64), axis=1)
+    r2 = oracle.gemv_w2a16(words, f16_bits(lut), f16_bits(x))
+    assert np.allclose(r2["y"], xf @ Wd.T, rtol=1e-10, atol=1e-12)
+    assert np.allclose(r2["labsx"], np.abs(xf) @ np.abs(Wd).T, rtol=1e-12)
+
+
+def test_split16_hand_cases_from_fixture():
+    rows = [ln.split() for ln in open(os.path.join(GOLD, "split16_hand_cases.txt")) if ln.strip() and not ln.startswith("#")]
+    x = torch.tensor([[float(r[0]) for r in rows]], dtype=torch.float16)
+    assert np.array_equal(x.numpy().astype(np.float64)[0], [float(r[0]) for r in rows])   # the fixture's x are fp16 values
+    sp = oracle.split_act16(f16_bits(x))
+    want = np.array([[int(v) for v in r[2:6]] for r in rows], dtype=np.int8).T       # [4][K]
+    assert np.array_equal(sp["digits"][0], want)
+    assert np.array_equal(sp["unit"][0], [2.0 ** -21, 2.0 ** -15, 2.0 ** -9, 2.0 ** -3])
+
+
+def test_split16_digits_reproduce_the_activations():
+    rng = np.random.default_rng(4)
+    toks = [synth.make_activations(1, 1024, 9).numpy()[0].astype(np.float64),
+            rng.standard_normal(1024) * 1e-3, rng.standard_normal(1024) * 200.0,
+            np.concatenate([[65504.0, -65504.0, 2.0 ** -24, -2.0 ** -14], rng.standard_normal(1020)]),
+            np.concatenate([[2.0 ** -24 * 3], np.zeros(1023)]),        # a token of subnormals only
+            np.zeros(1024)]
+    x = torch.tensor(np.stack(toks), dtype=torch.float16)
+    xf = x.numpy().astype(np.float64)
+    sp = oracle.split_act16(f16_bits(x))
+    dg, unit = sp["digits"].astype(np.int64), sp["unit"]
+    assert dg[:, :3].min() >= -32 and dg[:, :3].max() <= 31 and np.abs(dg[:, 3]).max() <= 16
+    for m in range(x.shape[0]):
+        amax = np.abs(xf[m]).max()
+        E = int(np.floor(np.log2(amax))) if amax > 0 else 0
+        assert np.array_equal(unit[m], 2.0 ** (E - 21 + 6 * np.arange(4)))
+        X = dg[m, 0] + 64 * dg[m, 1] + 4096 * dg[m, 2] + 262144 * dg[m, 3]
+        rec = X * 2.0 ** (E - 21)
+        assert np.all(np.abs(rec - xf[m]) <= 2.0 ** (E - 22))                        # half a unit at most
+        big = np.abs(xf[m]) >= 2.0 ** (E - 11)                                       # 11 significant bits fit above the unit
+        assert np.array_equal(rec[big], xf[m][big])
+        assert np.array_equal(X, np.rint(xf[m] * 2.0 ** (21 - E)).astype(np.int64))   # numpy rounds half to even
+    assert not dg[5].any()
+    with pytest.raises(ValueError):
+        oracle.split_act16(np.array([[0x7C00, 0]], dtype=np.uint16))
