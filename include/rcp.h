@@ -92,6 +92,29 @@ int rcp_quantize_act(const void* x_f16, int M, int K, int had_block, float clip_
 enum { RCP_GEMV_AUTO = 0, RCP_GEMV_SIMPLE = 1, RCP_GEMV_DP4A = 2, RCP_GEMV_MMA = 3, RCP_GEMV_MMA_ONLY = 4 };
 
 /*
+ * Weight-only form of the LUT GEMV (Section 5, the W2-only setting of Table "W2_inference": the codes
+ * and the dequantization grid of Section 4.4, activations left in 16-bit floating point):
+ *   y[m][n] = sum_k lut[n][ code[n][k] ] * x[m][k]
+ * The activations go through the integer kernels as block fixed point (an encoding of this library,
+ * the paper has none): per token, with E = floor(log2(max_k |x[m][k]|)), X = round-half-even(x * 2^(21-E))
+ * is split into four base-64 digits q0..q3 (q0..q2 in [-32, 31]); each digit plane is one int8 "token" of
+ * the tensor-core GEMV, whose exact integer per-code sums are weighted by the grid and the digit's unit
+ * 2^(E-21) * 64^d and added in fp32. Elements within 2^-11 of the token's largest magnitude are taken
+ * exactly, smaller ones to within 2^(E-22); so |y - exact| <= 2^(E-22) * sum_k |lut[n][code]| plus the
+ * fp32 finish and the fp16 rounding of y.
+ *   words, lut_f16   DEVICE, as for rcp_gemv_w2a4 (per-row grid).
+ *   x_f16            DEVICE fp16 [M][K], finite; 16-byte aligned.
+ *   M                1..16 (two tokens per launch, four while 16 * K <= 80 KiB); K % 64 == 0, K <= 32768.
+ *   y_f16            DEVICE fp16 [M][N], written.
+ *   digits           DEVICE int8 [M][4][K], written: the digit planes (16-byte aligned).
+ *   unit             DEVICE fp32 [M][4], written: the unit of each digit plane.
+ *   workspace        as for rcp_gemv_w2a4.
+ * Asynchronous on `stream`; returns RCP_OK or a negative status (RCP_ERR_SHAPE for K above 32768).
+ */
+int rcp_gemv_w2a16(const uint32_t* words, const void* lut_f16, const void* x_f16, int M, int N, int K, void* y_f16,
+                   int8_t* digits, float* unit, void* workspace, void* stream);
+
+/*
  * Bytes of caller-provided scratch rcp_gemv_w2a4 needs for this shape (0 on bad shapes). The scratch
  * holds a status word that a kernel sets if one of its bounded waits ever gives up (0 = fine). It
  * must be zero-filled once after allocation; every successful call leaves it zero-filled, so one

@@ -62,6 +62,8 @@ def lib():
         L.rcp_linear_w2a4_host.argtypes = [vp, i, i, i, C.c_float, vp, vp, i, vp, vp, vp, vp, vp, vp, vp]
         L.rcp_gemv_w2a4_static.restype = i
         L.rcp_gemv_w2a4_static.argtypes = [vp, vp, vp, vp, i, i, i, vp, vp]
+        L.rcp_gemv_w2a16.restype = i
+        L.rcp_gemv_w2a16.argtypes = [vp, vp, vp, i, i, i, vp, vp, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -196,6 +198,32 @@ def rcp_gemv_w2a4_grouped(words, lut, xq, scale, group=128, y=None, workspace=No
         _check("rcp_gemv_w2a4_grouped",
                lib().rcp_gemv_w2a4_grouped_variant(v, _ptr(words), _ptr(lut), group, _ptr(xq), _ptr(scale), M, N, K,
                                                    _ptr(y), _ptr(workspace), _ptr(S_dbg), _stream(words)))
+    return y
+
+
+def rcp_gemv_w2a16(words, lut, x, y=None, digits=None, unit=None, workspace=None):
+    """Weight-only form: words int32 [N][K/16], lut fp16 [N][4], x fp16 [M][K] -> y fp16 [M][N].
+    digits int8 [M][4][K] and unit fp32 [M][4] receive the fixed-point form of x the kernels used."""
+    _dev(words, torch.int32, "words")
+    _dev(lut, torch.float16, "lut")
+    _dev(x, torch.float16, "x")
+    N, W = words.shape
+    K = W * 16
+    M = x.shape[0]
+    if x.shape != (M, K) or lut.shape != (N, 4):
+        raise ValueError("shape mismatch between words, lut and x")
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.float16, device=words.device)
+    if digits is None:
+        digits = torch.empty((M, 4, K), dtype=torch.int8, device=words.device)
+    if unit is None:
+        unit = torch.empty((M, 4), dtype=torch.float32, device=words.device)
+    if workspace is None:
+        workspace = make_workspace(M, N, K, words.device)
+    with _on(words):
+        _check("rcp_gemv_w2a16",
+               lib().rcp_gemv_w2a16(_ptr(words), _ptr(lut), _ptr(x), M, N, K, _ptr(y), _ptr(digits), _ptr(unit),
+                                    _ptr(workspace), _stream(words)))
     return y
 
 

@@ -22,6 +22,17 @@ __device__ __forceinline__ __half lut_finish(float s, uint2 lut4, int S0, int S1
   return __float2half_rn(s * acc);
 }
 
+// L0*S0 + L1*S1 + L2*S2 + L3*S3 alone, in the same order and arithmetic.
+__device__ __forceinline__ float lut_sum(uint2 lut4, int S0, int S1, int S2, int S3) {
+  const __half2 l01 = *reinterpret_cast<const __half2*>(&lut4.x);
+  const __half2 l23 = *reinterpret_cast<const __half2*>(&lut4.y);
+  float acc = __half2float(__low2half(l01)) * (float)S0;
+  acc = fmaf(__half2float(__high2half(l01)), (float)S1, acc);
+  acc = fmaf(__half2float(__low2half(l23)), (float)S2, acc);
+  acc = fmaf(__half2float(__high2half(l23)), (float)S3, acc);
+  return acc;
+}
+
 // q[e] = clamp(round-half-even(v[e] / s), -8, 7) for NV values, the quotient being the IEEE fp32
 // division the definition asks for, without dividing in the common case. With rinv = 1 / s (correctly
 // rounded), t = v * rinv lies within 2^-23 |v / s| of the exact quotient and the IEEE quotient within half

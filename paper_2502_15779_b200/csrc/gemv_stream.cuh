@@ -70,6 +70,7 @@ struct GemvParams {
   const uint2* lut;
   const uint8_t* xq;
   const __half* scale;
+  const float* unit;     // A16: fp32 unit of each digit column (scale unused)
   __half* y;
   int32_t* status;      // optional: receives a code when a bounded wait gives up
   int M, N, K;
@@ -193,7 +194,10 @@ __device__ __forceinline__ void dp4a_s8s8(int& d, uint32_t a, uint32_t b) {
 //       it costs less than a kernel of its own. A thread takes one word (16 consecutive activations):
 //       strides 1..8 in registers, 16..256 by lane exchanges, 512 and up through shared memory, one
 //       thread per (lane, element) column over the warps.
-template <int MODE, int MTOK, bool GRP, bool FQ = false>
+// A16   weight-only form: the "tokens" are the four base-64 fixed-point digits of up to two (MTOK 16: four)
+//       fp16 tokens, one signed byte per element (p.xq is [4 tokens][K] bytes, p.unit their fp32 units, p.M
+//       the number of digit columns); the digits of a token are combined in fp32 when its rows are finished.
+template <int MODE, int MTOK, bool GRP, bool FQ = false, bool A16 = false>
 __global__ void __launch_bounds__(kGThreads, 1)
 gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -205,6 +209,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   const int M = (MTOK > 0 && MODE != kModeMma) ? MTOK : p.M;
   constexpr bool kTwoTiles = (MODE == kModeMma && MTOK == 16);   // tokens 8..15 in a second set of accumulators
   static_assert(!(kTwoTiles && (GRP || FQ)), "two column tiles: per-row grid, quantized activations only");
+  static_assert(!A16 || (MODE == kModeMma && !GRP && !FQ), "digit columns: tensor-core mode, per-row grid");
   const int ncol = M;
   const int stages = p.stages;
   const uint32_t full0 = base + p.off_bar, empty0 = full0 + 8 * kMaxStages;
@@ -366,20 +371,45 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
       if (u < total && wx < W) x = __ldg(reinterpret_cast<const uint4*>(p.xq + (size_t)col * (p.K / 2)) + (wx >> 1));
       return x;
     };
+    // digit columns: the 16 bytes of word wx + w of unit u
+    auto load_unit_bytes = [&](int u, int w) {
+      const int pair = u >> 4;
+      const int col = (int)(((uint32_t)pair * (uint32_t)p.inv_nchunk) >> 20), ch = pair - col * p.nchunk;
+      const int lo = u & 3, hi = (u >> 2) & 3;
+      const int wx = ch * kChunkWords + 8 * lo + 2 * hi + w;
+      uint4 x = make_uint4(0, 0, 0, 0);
+      if (u < total && wx < W) x = __ldg(reinterpret_cast<const uint4*>(p.xq + (size_t)col * p.K) + wx);
+      return x;
+    };
     // per-row grid: the next unit's words are fetched while this one is expanded (the group-wise
     // kernels have no registers to spare for that)
     uint4 x_next = make_uint4(0, 0, 0, 0);
-    if constexpr (!GRP) x_next = load_unit(warp * 32 + lane);
+    if constexpr (!GRP && !A16) x_next = load_unit(warp * 32 + lane);
     for (int u0 = warp * 32; u0 < total; u0 += kCWarps * 32) {
       const int u = u0 + lane;
       int tsum = 0;
       const int pair = u >> 4;
       const int col = (int)(((uint32_t)pair * (uint32_t)p.inv_nchunk) >> 20), ch = pair - col * p.nchunk;   // pair / nchunk
-      const uint4 x = GRP ? load_unit(u) : x_next;
-      if constexpr (!GRP) x_next = load_unit(u + kCWarps * 32);
+      const uint4 x = (GRP || A16) ? (A16 ? make_uint4(0, 0, 0, 0) : load_unit(u)) : x_next;
+      if constexpr (!GRP && !A16) x_next = load_unit(u + kCWarps * 32);
       if (u < total) {
         const int lo = u & 3, hi = (u >> 2) & 3;   // lo: 16-byte slot t of the column block; hi: 2 i + pr, or the group
         uint32_t q[4][2];
+        if constexpr (A16) {
+#pragma unroll
+          for (int w = 0; w < 2; w++) {
+            const uint4 d = load_unit_bytes(u, w);   // bytes 4b..4b+3 of d: the digits that meet byte b of the weight word
+            tsum = __dp4a((int)d.x, 0x01010101, tsum); tsum = __dp4a((int)d.y, 0x01010101, tsum);
+            tsum = __dp4a((int)d.z, 0x01010101, tsum); tsum = __dp4a((int)d.w, 0x01010101, tsum);
+            // 4 x 4 byte transpose: position p gathers byte p of each of the four
+            const uint32_t t01 = __byte_perm(d.x, d.y, 0x5140), t23 = __byte_perm(d.z, d.w, 0x5140);
+            const uint32_t s01 = __byte_perm(d.x, d.y, 0x7362), s23 = __byte_perm(d.z, d.w, 0x7362);
+            q[0][w] = (__byte_perm(t01, t23, 0x5410) << 2) & 0xFCFCFCFCu;   // even positions carry 4 q (|q| <= 32)
+            q[1][w] = __byte_perm(t01, t23, 0x7632);
+            q[2][w] = (__byte_perm(s01, s23, 0x5410) << 2) & 0xFCFCFCFCu;
+            q[3][w] = __byte_perm(s01, s23, 0x7632);
+          }
+        } else
 #pragma unroll
         for (int w = 0; w < 2; w++) {
           const uint32_t lo32 = w ? x.z : x.x, hi32 = w ? x.w : x.y;   // codes 0..7 and 8..15 of the word
@@ -415,7 +445,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
         if ((u & 12) == 0 && u < total) s_T0c[col * ng4 + ch * 4 + (u & 3)] = tsum;
       }
     }
-    if (tid < M) s_scale[tid] = __half2float(p.scale[tid]);
+    if (tid < M) s_scale[tid] = A16 ? p.unit[tid] : __half2float(p.scale[tid]);
     if constexpr (!GRP)
       for (int i = tid; i < 2 * 8 * 16 * M * 3; i += kCWarps * 32) s_red[i] = 0;
   }
@@ -797,13 +827,35 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     }
   };
   auto emit = [&](int row_first, const int (&T1)[NE], const int (&T2)[NE], const int (&T3)[NE]) {
+    if constexpr (A16) {
+      // Columns 4j..4j+3 are the digits of token j: lane t holds two of them, lane t ^ 1 the other two.
+      // y = (u_a D_a + u_b D_b) + (u_c D_c + u_d D_d) in fp32, D the grid-weighted sum of a digit column.
 #pragma unroll
-    for (int e = 0; e < NE; e++) {
-      const int row = row_first + g + 8 * err[e];
-      if (etok[e] < M && row < p.N) {
-        const int S3 = T3[e], S1 = T1[e] - T3[e], S2 = T2[e] - T3[e];
-        const int S0 = (kTwoTiles ? s_T0tot[etok[e]] : T0v[e]) - S1 - S2 - S3;
-        p.y[(size_t)etok[e] * p.N + row] = lut_finish(s_scale[etok[e]], lut_g[err[e]], S0, S1, S2, S3);
+      for (int e = 0; e < NE; e += 2) {
+        float v = 0.f;
+#pragma unroll
+        for (int h = 0; h < 2; h++) {
+          const int c = etok[e + h];
+          if (c < M) {
+            const int S3 = T3[e + h], S1 = T1[e + h] - T3[e + h], S2 = T2[e + h] - T3[e + h];
+            const int S0 = (kTwoTiles ? s_T0tot[c] : T0v[e + h]) - S1 - S2 - S3;
+            const float d = lut_sum(lut_g[err[e]], S0, S1, S2, S3);
+            v = h ? __fmaf_rn(s_scale[c], d, v) : __fmul_rn(s_scale[c], d);
+          }
+        }
+        v = __fadd_rn(v, __shfl_xor_sync(0xffffffffu, v, 1));   // both lanes add the same two numbers
+        const int row = row_first + g + 8 * err[e], tok = etok[e] >> 2;
+        if ((t & 1) == 0 && etok[e] < M && row < p.N) p.y[(size_t)tok * p.N + row] = __float2half_rn(v);
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < NE; e++) {
+        const int row = row_first + g + 8 * err[e];
+        if (etok[e] < M && row < p.N) {
+          const int S3 = T3[e], S1 = T1[e] - T3[e], S2 = T2[e] - T3[e];
+          const int S0 = (kTwoTiles ? s_T0tot[etok[e]] : T0v[e]) - S1 - S2 - S3;
+          p.y[(size_t)etok[e] * p.N + row] = lut_finish(s_scale[etok[e]], lut_g[err[e]], S0, S1, S2, S3);
+        }
       }
     }
   };

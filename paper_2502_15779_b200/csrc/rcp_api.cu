@@ -11,6 +11,7 @@
 #include "gemv_simple.cuh"
 #include "gemv_stream.cuh"
 #include "ldp_export.cuh"
+#include "split_act16.cuh"
 #include "pack.cuh"
 #include "quantize_act.cuh"
 
@@ -193,10 +194,10 @@ int sm_count() {
   return n;
 }
 
-template <int MODE, int MTOK, bool GRP = false, bool FQ = false>
+template <int MODE, int MTOK, bool GRP = false, bool FQ = false, bool A16 = false>
 int launch_stream_t(const rcp::GemvMaps& maps, const rcp::GemvParams& gp, const StreamPlan& pl, cudaStream_t st) {
   static bool attr_set = false;
-  auto kern = rcp::gemv_stream_kernel<MODE, MTOK, GRP, FQ>;
+  auto kern = rcp::gemv_stream_kernel<MODE, MTOK, GRP, FQ, A16>;
   if (!attr_set) {
     RCP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax));
     attr_set = true;
@@ -223,7 +224,9 @@ bool fused_ok(int M, int K, int B) { return M == 1 && B == K && (K == 4096 || K 
 
 int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const uint8_t* xq, const void* scale_f16,
                   int M, int N, int K, void* y_f16, void* workspace, cudaStream_t st, bool grouped = false,
-                  const FusedAct* fa = nullptr) {
+                  const FusedAct* fa = nullptr, const float* unit = nullptr) {
+  // unit: weight-only form; xq then holds M digit columns of K signed bytes (four per token), scale_f16 is unused
+  if (unit && (mode != rcp::kModeMma || grouped || fa || M % 4)) return RCP_ERR_VARIANT;
   if (mode != rcp::kModeMma && M > 2) return RCP_ERR_VARIANT;
   if (M > 8 && (grouped || fa || M > rcp::kMaxTokens)) return RCP_ERR_VARIANT;
   if (grouped && (mode == rcp::kModeHybrid || K % 128)) return RCP_ERR_VARIANT;
@@ -270,6 +273,7 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   gp.lut = static_cast<const uint2*>(lut_f16);
   gp.xq = xq;
   gp.scale = static_cast<const __half*>(scale_f16);
+  gp.unit = unit;
   gp.y = static_cast<__half*>(y_f16);
   gp.status = static_cast<int32_t*>(workspace);
   gp.M = M; gp.N = N; gp.K = K;
@@ -295,6 +299,9 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
     return grouped ? launch_stream_t<rcp::kModeDp4a, 1, true, true>(maps, gp, pl, st)
                    : launch_stream_t<rcp::kModeDp4a, 1, false, true>(maps, gp, pl, st);
   }
+  if (unit)
+    return M > 8 ? launch_stream_t<rcp::kModeMma, 16, false, false, true>(maps, gp, pl, st)
+                 : launch_stream_t<rcp::kModeMma, 0, false, false, true>(maps, gp, pl, st);
   if (grouped) {
     if (mode == rcp::kModeDp4a)
       return M == 1 ? launch_stream_t<rcp::kModeDp4a, 1, true>(maps, gp, pl, st)
@@ -559,6 +566,31 @@ int rcp_gemv_w2a4(const uint32_t* words, const void* lut_f16, const uint8_t* xq,
                   int M, int N, int K, void* y_f16, void* workspace, int32_t* S_dbg, void* stream) {
   return rcp_gemv_w2a4_variant(RCP_GEMV_AUTO, words, lut_f16, xq, scale_f16, M, N, K, y_f16, workspace,
                                S_dbg, stream);
+}
+
+int rcp_gemv_w2a16(const uint32_t* words, const void* lut_f16, const void* x_f16, int M, int N, int K, void* y_f16,
+                   int8_t* digits, float* unit, void* workspace, void* stream) {
+  if (!words || !lut_f16 || !x_f16 || !y_f16 || !digits || !unit) return RCP_ERR_NULL;
+  if (M < 1 || M > rcp::kMaxTokens || N < 1 || !k_ok(K)) return RCP_ERR_SHAPE;
+  if (!aligned16(words) || !aligned16(x_f16) || !aligned16(digits) || (reinterpret_cast<uintptr_t>(lut_f16) & 7u) ||
+      (reinterpret_cast<uintptr_t>(y_f16) & 1u) || (reinterpret_cast<uintptr_t>(unit) & 3u) ||
+      (reinterpret_cast<uintptr_t>(workspace) & 3u))
+    return RCP_ERR_ALIGN;
+  // digit columns per launch: sixteen (four tokens) or eight (two) where their expanded bytes fit, else four
+  const int cols = 4 * M;
+  const int cp = tokens_per_pass(std::min(cols, 16), K, 16) & ~3;
+  if (cp < 4) return RCP_ERR_SHAPE;   // K beyond 32768: the four digit planes of one token do not fit
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  RCP_CUDA(launch_overlapped(rcp::split_act16_kernel, dim3(M), dim3(rcp::kSplitThreads), 0, st,
+                             static_cast<const __half*>(x_f16), K, digits, unit));
+  for (int c0 = 0; c0 < cols; c0 += cp) {
+    const int cc = std::min(cp, cols - c0);
+    const int rc = launch_stream(rcp::kModeMma, words, lut_f16, reinterpret_cast<const uint8_t*>(digits) + (size_t)c0 * K,
+                                 nullptr, cc, N, K, static_cast<__half*>(y_f16) + (size_t)(c0 / 4) * N, workspace, st,
+                                 false, nullptr, unit + c0);
+    if (rc != RCP_OK) return rc;
+  }
+  return RCP_OK;
 }
 
 int rcp_gemv_w2a4_grouped_variant(int variant, const uint32_t* words, const void* lut_f16, int group,
