@@ -289,6 +289,27 @@ def per_shape_table(cfg, Ms, device, rcp, stream, variant, reps=3):
                 row.update({"grouped_bytes": nbytes_g, "grouped_us_per_call": round(us_g, 3),
                             "grouped_gbs": round(nbytes_g / us_g / 1e3, 1)})
                 del gg
+            if M <= 2 and L.K <= 32768:
+                # the weight-only form on the same weights: fp16 activations, split kernel + GEMV per call
+                dg = torch.empty(M, 4, L.K, dtype=torch.int8, device=device)
+                un = torch.empty(M, 4, dtype=torch.float32, device=device)
+
+                def body_a():
+                    for i in range(launches):
+                        c = i % copies
+                        rcp.rcp_gemv_w2a16(words[c], luts[c], x, y=y, digits=dg, unit=un, workspace=ws)
+                with torch.cuda.stream(stream):
+                    body_a()
+                stream.synchronize()
+                ga = capture(body_a, stream)
+                for _ in range(3):
+                    ga.replay()
+                stream.synchronize()
+                us_a = min(time_graph_replays([ga], [0], stream) for _ in range(reps)) * 1e3 / launches
+                nbytes_a = cfgs.gemv_w2a16_bytes(M, L.N, L.K)
+                row.update({"w2a16_bytes": nbytes_a, "w2a16_us_per_call": round(us_a, 3),
+                            "w2a16_gbs": round(nbytes_a / us_a / 1e3, 1)})
+                del ga
             rows.append(row)
         del words, luts, base, luts_g, lut_g
         torch.cuda.empty_cache()

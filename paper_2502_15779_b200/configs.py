@@ -67,3 +67,8 @@ def gemv_grouped_bytes(M: int, N: int, K: int, G: int) -> int:
 def quant_bytes(M: int, K: int) -> int:
     """Algorithmic bytes of one activation-quantization call: fp16 in, nibbles + fp16 scale out."""
     return 2 * M * K + M * K // 2 + 2 * M
+
+
+def gemv_w2a16_bytes(M: int, N: int, K: int) -> int:
+    """Algorithmic bytes of one weight-only GEMV call: packed codes + per-row LUT + fp16 activations + fp16 output."""
+    return N * K // 4 + 8 * N + 2 * M * K + 2 * M * N
