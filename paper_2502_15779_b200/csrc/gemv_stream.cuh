@@ -381,19 +381,25 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
       if (u < total && wx < W) x = __ldg(reinterpret_cast<const uint4*>(p.xq + (size_t)col * p.K) + wx);
       return x;
     };
-    // per-row grid: the next unit's words are fetched while this one is expanded (the group-wise
-    // kernels have no registers to spare for that)
+    // tensor-core kernels of the per-row grid (several tokens, so several units per thread): the next unit's
+    // words are fetched while this one is expanded. Measured: the one- and two-token kernels lose 1 % with
+    // it, the group-wise kernels have no registers to spare for it.
+    constexpr bool kPrefetch = !GRP && !A16 && MODE == kModeMma;
     uint4 x_next = make_uint4(0, 0, 0, 0);
-    if constexpr (!GRP && !A16) x_next = load_unit(warp * 32 + lane);
+    if constexpr (kPrefetch) x_next = load_unit(warp * 32 + lane);
     for (int u0 = warp * 32; u0 < total; u0 += kCWarps * 32) {
       const int u = u0 + lane;
       int tsum = 0;
       const int pair = u >> 4;
       const int col = (int)(((uint32_t)pair * (uint32_t)p.inv_nchunk) >> 20), ch = pair - col * p.nchunk;   // pair / nchunk
-      const uint4 x = (GRP || A16) ? (A16 ? make_uint4(0, 0, 0, 0) : load_unit(u)) : x_next;
-      if constexpr (!GRP && !A16) x_next = load_unit(u + kCWarps * 32);
+      uint4 x = x_next;
+      if constexpr (kPrefetch) x_next = load_unit(u + kCWarps * 32);
       if (u < total) {
         const int lo = u & 3, hi = (u >> 2) & 3;   // lo: 16-byte slot t of the column block; hi: 2 i + pr, or the group
+        if constexpr (!kPrefetch && !A16) {
+          const int wx = ch * kChunkWords + (kRelabel ? 8 * hi + 2 * lo : 8 * lo + 2 * hi);   // word index in the row
+          if (wx < W) x = __ldg(reinterpret_cast<const uint4*>(p.xq + (size_t)col * (p.K / 2)) + (wx >> 1));
+        }
         uint32_t q[4][2];
         if constexpr (A16) {
 #pragma unroll
