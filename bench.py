@@ -516,12 +516,12 @@ def main():
                               "frac": round(p_ach / peaks["hbm_gbs"], 4),
                               "note": "rcp_gemv_w2a4 launches alone, activations quantized beforehand"}
     del pgraphs
-    # Second bound: the kernel needs 245 warp instructions per KB of packed weights at one token (instruction
+    # Second bound: the kernel needs 249 warp instructions per KB of packed weights at one token (instruction
     # mix counted by ncu, profiles/gemv_stream_llama2_7b_M1_full.md) and an SM issues at most four per clock.
     if M == 1 and args.variant in ("auto", "dp4a") and clocks and clocks.get("sm_mhz"):
         sms = torch.cuda.get_device_properties(device).multi_processor_count
-        issue_gbs = 4.0 * sms * clocks["sm_mhz"] * 1e6 / 245.0 * 1024.0 / 1e9
-        roofline["issue_bound"] = {"warp_instructions_per_kb": 245, "peak": round(issue_gbs, 1), "unit": "GB/s",
+        issue_gbs = 4.0 * sms * clocks["sm_mhz"] * 1e6 / 249.0 * 1024.0 / 1e9
+        roofline["issue_bound"] = {"warp_instructions_per_kb": 249, "peak": round(issue_gbs, 1), "unit": "GB/s",
                                    "frac": round(achieved / issue_gbs, 4),
                                    "plain_gemv_frac": round(p_ach / issue_gbs, 4),
                                    "note": "4 warp instructions per clock per SM at the sampled SM clock"}
