@@ -125,9 +125,21 @@ class LayerSet:
             self.y.append(torch.empty(M, L.N, dtype=torch.float16, device=device))
             self.ws.append(rcp.make_workspace(M, L.N, L.K, device))
         self.copies = copies
+        self.digits = self.unit = None
+
+    def step_w2a16(self, copy):
+        """The same layer in the weight-only form (fp16 activations): split kernel + GEMV per linear."""
+        if self.digits is None:
+            self.digits = [torch.empty(self.M, 4, L.K, dtype=torch.int8, device=self.dev) for L in self.layers]
+            self.unit = [torch.empty(self.M, 4, dtype=torch.float32, device=self.dev) for L in self.layers]
+        for li, L in enumerate(self.layers):
+            self.rcp.rcp_gemv_w2a16(self.words[li][copy], self.luts[li][copy], self.x[li], y=self.y[li],
+                                    digits=self.digits[li], unit=self.unit[li], workspace=self.ws[li])
 
     def step(self, copy, variant="auto"):
         r = self.rcp
+        if variant == "w2a16":
+            return self.step_w2a16(copy)
         for li, L in enumerate(self.layers):
             if variant == "auto":
                 # the library's own chain: one kernel where that is faster, else quantizer + GEMV
@@ -408,7 +420,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2_70b", choices=list(cfgs.BY_KEY))
     ap.add_argument("--tokens", type=int, default=1)
-    ap.add_argument("--variant", default="auto", choices=["auto", "simple", "dp4a", "mma", "mma_only"])
+    ap.add_argument("--variant", default="auto", choices=["auto", "simple", "dp4a", "mma", "mma_only", "w2a16"],
+                    help="kernel variant of the W2A4 GEMV; w2a16 (only with --profile) runs the layer in the "
+                         "weight-only form instead, for the ncu summaries")
     ap.add_argument("--no-table", action="store_true", help="skip the per-shape table of the other configs")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle leg")
     ap.add_argument("--sample-seconds", type=float, default=12.0,
@@ -421,6 +435,8 @@ def main():
     if args.warmup < 3:
         args.warmup = 3
 
+    if args.variant == "w2a16" and (not args.profile or args.impl == "reference"):
+        ap.error("--variant w2a16 is a profiling aid: use it with --profile")
     if args.impl == "reference":
         run_reference(args, cfg, M)
         return
