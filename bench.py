@@ -153,14 +153,14 @@ class LayerSet:
     def launches_per_step(self, variant="auto"):
         r = self.rcp
         if variant == "auto":
-            return sum(r.rcp_linear_w2a4_launches(self.M, L.K, L.had_block) for L in self.layers)
+            return sum(r.rcp_linear_w2a4_launches(self.M, L.N, L.K, L.had_block) for L in self.layers)
         return sum(1 + -(-self.M // (8 if variant in ("mma", "mma_only") else 2)) for L in self.layers)
 
     def stream_kernels_only(self, copy, variant="auto"):
         """The launches of the streaming kernel a step makes, without the stand-alone quantizer launches."""
         r = self.rcp
         for li, L in enumerate(self.layers):
-            if variant == "auto" and r.rcp_linear_w2a4_launches(self.M, L.K, L.had_block) == 1:
+            if variant == "auto" and r.rcp_linear_w2a4_launches(self.M, L.N, L.K, L.had_block) == 1:
                 r.rcp_linear_w2a4(self.x[li], L.had_block, 1.0, self.words[li][copy], self.luts[li][copy], y=self.y[li],
                                   xq=self.xq[li], scale=self.scale[li], workspace=self.ws[li])
             else:
@@ -504,7 +504,7 @@ def main():
     gms = min(time_graph_replays(ggraphs, order, stream) for _ in range(3))
     g_launches = args.steps * (layer.launches_per_step(args.variant) -
                                sum(1 for L in layer.layers
-                                   if args.variant != "auto" or rcp.rcp_linear_w2a4_launches(M, L.K, L.had_block) > 1))
+                                   if args.variant != "auto" or rcp.rcp_linear_w2a4_launches(M, L.N, L.K, L.had_block) > 1))
     g_bytes_per_launch = layer.gemv_bytes() * args.steps / g_launches
     g_us = gms * 1e3 / g_launches
     achieved = g_bytes_per_launch / g_us / 1e3
@@ -523,7 +523,7 @@ def main():
     time_graph_replays(pgraphs, order[:8], stream)
     pms = min(time_graph_replays(pgraphs, order, stream) for _ in range(3))
     # had_block 1 never takes the single kernel: the count is the quantizer plus the GEMV launches
-    p_launches = args.steps * sum(rcp.rcp_linear_w2a4_launches(M, L.K, 1) - 1 if args.variant == "auto"
+    p_launches = args.steps * sum(rcp.rcp_linear_w2a4_launches(M, L.N, L.K, 1) - 1 if args.variant == "auto"
                                   else -(-M // (8 if args.variant in ("mma", "mma_only") else 2))
                                   for L in layer.layers)
     p_us = pms * 1e3 / p_launches

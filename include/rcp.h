@@ -80,8 +80,10 @@ int rcp_quantize_act(const void* x_f16, int M, int K, int had_block, float clip_
  *   RCP_GEMV_DP4A    streaming kernel, CUDA cores only: masked code planes times int8 activations
  *                    with dp4a, two tokens per launch.
  *   RCP_GEMV_MMA     streaming kernel with the masked code planes as the A operand of int8 mma.sync,
- *                    up to eight tokens per launch (fewer when K is so long that their expanded
- *                    activations would not fit in shared memory); nine to sixteen tokens go in one
+ *                    up to eight tokens per launch (when K is so long that their expanded activations
+ *                    would not fit in shared memory at once, the launch goes through K in up to eight
+ *                    parts, keeping the integer sums of its rows in shared memory in between; fewer
+ *                    tokens per launch only where even that does not fit); nine to sixteen tokens go in one
  *                    launch (two MMA column tiles fed from the same masks) while M * K <= 80 KiB,
  *                    else in launches of eight at most; for one or two tokens the b0*b1
  *                    plane is computed with dp4a beside the tensor cores.
@@ -104,12 +106,12 @@ enum { RCP_GEMV_AUTO = 0, RCP_GEMV_SIMPLE = 1, RCP_GEMV_DP4A = 2, RCP_GEMV_MMA =
  * fp32 finish and the fp16 rounding of y.
  *   words, lut_f16   DEVICE, as for rcp_gemv_w2a4 (per-row grid).
  *   x_f16            DEVICE fp16 [M][K], finite; 16-byte aligned.
- *   M                1..16 (two tokens per launch, four while 16 * K <= 80 KiB); K % 64 == 0, K <= 32768.
+ *   M                1..16 (two tokens per launch, four while 16 * K <= 80 KiB); K % 64 == 0.
  *   y_f16            DEVICE fp16 [M][N], written.
  *   digits           DEVICE int8 [M][4][K], written: the digit planes (16-byte aligned).
  *   unit             DEVICE fp32 [M][4], written: the unit of each digit plane.
  *   workspace        as for rcp_gemv_w2a4.
- * Asynchronous on `stream`; returns RCP_OK or a negative status (RCP_ERR_SHAPE for K above 32768).
+ * Asynchronous on `stream`; returns RCP_OK or a negative status.
  */
 int rcp_gemv_w2a16(const uint32_t* words, const void* lut_f16, const void* x_f16, int M, int N, int K, void* y_f16,
                    int8_t* digits, float* unit, void* workspace, void* stream);
@@ -127,7 +129,9 @@ size_t rcp_gemv_workspace_bytes(int M, int N, int K);
  * GPU). `sms` is the number of CTAs (one per SM; <= 0: 148). Writes up to `cap` ints to `out`:
  *   out[0] tokens per launch, out[1] launches, out[2] ring stages, out[3] shared-memory bytes,
  *   out[4] 128-byte chunks per row, out[5] number of phases, then per phase five ints:
- *   groups per CTA at most, first group, groups in the phase, CTAs taking part, repetitions.
+ *   groups per CTA at most, first group, groups in the phase, CTAs taking part, repetitions;
+ *   and one last int: the parts of K one launch goes through one after the other (1 unless several tokens
+ *   meet a K so long that their expanded activations do not fit in shared memory at once).
  * (A group is 16 consecutive output rows; see the kernel's description.) Returns the number of
  * ints the full description has, or a negative status.
  */
@@ -222,7 +226,7 @@ int rcp_linear_w2a4(const void* x_f16, int M, int K, int had_block, float clip_r
 
 /* Kernel launches one rcp_linear_w2a4 call makes for a shape (1: the single kernel; otherwise the
  * quantizer plus one GEMV launch per batch of tokens). Host only. Negative status on a bad shape. */
-int rcp_linear_w2a4_launches(int M, int K, int had_block, int group);
+int rcp_linear_w2a4_launches(int M, int N, int K, int had_block, int group);
 
 /*
  * One decode linear layer end to end with HOST activations (Section 4.4 data path: rotate and

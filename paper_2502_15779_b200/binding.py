@@ -57,7 +57,7 @@ def lib():
         L.rcp_linear_w2a4.restype = i
         L.rcp_linear_w2a4.argtypes = [vp, i, i, i, C.c_float, vp, vp, i, i, vp, vp, vp, vp, vp]
         L.rcp_linear_w2a4_launches.restype = i
-        L.rcp_linear_w2a4_launches.argtypes = [i, i, i, i]
+        L.rcp_linear_w2a4_launches.argtypes = [i, i, i, i, i]
         L.rcp_linear_w2a4_host.restype = i
         L.rcp_linear_w2a4_host.argtypes = [vp, i, i, i, C.c_float, vp, vp, i, vp, vp, vp, vp, vp, vp, vp]
         L.rcp_gemv_w2a4_static.restype = i
@@ -277,9 +277,9 @@ def rcp_linear_w2a4(x, had_block, clip_ratio, words, lut, group=0, y=None, xq=No
     return y
 
 
-def rcp_linear_w2a4_launches(M: int, K: int, had_block: int, group: int = 0) -> int:
+def rcp_linear_w2a4_launches(M: int, N: int, K: int, had_block: int, group: int = 0) -> int:
     """Kernel launches one rcp_linear_w2a4 call makes for a shape (host only)."""
-    n = int(lib().rcp_linear_w2a4_launches(M, K, int(had_block), int(group)))
+    n = int(lib().rcp_linear_w2a4_launches(M, N, K, int(had_block), int(group)))
     if n < 0:
         raise RcpError("rcp_linear_w2a4_launches", n, lib().rcp_status_str(n).decode(), 0)
     return n

@@ -75,7 +75,10 @@ struct GemvParams {
   int32_t* status;      // optional: receives a code when a bounded wait gives up
   int M, N, K;
   int ngrp;             // group-wise grid: groups of 128 weights per row (K / 128), lut is [N][ngrp]; else 0
-  int nchunk;           // 128-byte chunks per row, ceil(K / 512)
+  int nchunk;           // 128-byte chunks per row, ceil(K / 512); with nsplit > 1: per part of K
+  int nchunk_total;     // chunks per row over the whole K
+  int nsplit;           // parts of K gone through one after the other (tensor-core kernels of the per-row grid; else 1)
+  int off_part;         // nsplit > 1: partial sums of this CTA's rows between the parts
   int inv_nchunk;       // ceil(2^20 / nchunk): x / nchunk == (x * inv_nchunk) >> 20 for x < 2^20 / nchunk
   int nphase;
   GemvPhase phase[kMaxPhases];
@@ -197,7 +200,8 @@ __device__ __forceinline__ void dp4a_s8s8(int& d, uint32_t a, uint32_t b) {
 // A16   weight-only form: the "tokens" are the four base-64 fixed-point digits of up to two (MTOK 16: four)
 //       fp16 tokens, one signed byte per element (p.xq is [4 tokens][K] bytes, p.unit their fp32 units, p.M
 //       the number of digit columns); the digits of a token are combined in fp32 when its rows are finished.
-template <int MODE, int MTOK, bool GRP, bool FQ = false, bool A16 = false>
+// SPLIT K in parts (see below): the eight-column tensor-core kernels of the per-row grid, when asked to.
+template <int MODE, int MTOK, bool GRP, bool FQ = false, bool A16 = false, bool SPLIT = false>
 __global__ void __launch_bounds__(kGThreads, 1)
 gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -210,6 +214,14 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   constexpr bool kTwoTiles = (MODE == kModeMma && MTOK == 16);   // tokens 8..15 in a second set of accumulators
   static_assert(!(kTwoTiles && (GRP || FQ)), "two column tiles: per-row grid, quantized activations only");
   static_assert(!A16 || (MODE == kModeMma && !GRP && !FQ), "digit columns: tensor-core mode, per-row grid");
+  // Long K with several tokens: the expanded activations of the whole K do not fit in shared memory. The kernel
+  // then goes through K in nsplit parts: activations of the part expanded, every phase run over the part's
+  // chunks, the integer sums of this CTA's rows parked in shared memory until the last part finishes them. The
+  // plan is the same for every part, so the same lane meets the same sums again: nothing crosses warps.
+  // A form of its own, so that the kernels that never need it keep their code.
+  constexpr bool kSplit = SPLIT;
+  static_assert(!SPLIT || (MODE == kModeMma && MTOK == 0 && !GRP && !FQ), "K in parts: eight-column tensor-core kernels, per-row grid");
+  const int nsplit = kSplit ? p.nsplit : 1;
   const int ncol = M;
   const int stages = p.stages;
   const uint32_t full0 = base + p.off_bar, empty0 = full0 + 8 * kMaxStages;
@@ -255,10 +267,13 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     // whole grid: issued all at once, the stages of all CTAs share the bandwidth and even the first
     // one lands only when nearly all of them have.
     const long long t_start = clock64();
+    for (int kp = 0; kp < nsplit; kp++) {
+    const int chunk0 = kSplit ? kp * p.nchunk : 0;                                    // this part of K
+    const int nch = kSplit ? min(p.nchunk, p.nchunk_total - chunk0) : p.nchunk;
     for (int pi = 0; pi < p.nphase; pi++) {
       const GemvPhase ph = p.phase[pi];
       if (b >= ph.ncta) continue;
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.m[pi]) : "memory");
+      if (kp == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.m[pi]) : "memory");
       const int KS = ph.ks;
       const uint32_t box = (uint32_t)ph.gpc * kGroupBytes;
       const int lo = ph.q * b + min(b, ph.r);
@@ -277,14 +292,15 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
             while (clock64() < due) { }
           }
           const uint32_t bar = full0 + 8 * slot, dst = base + (uint32_t)slot * kStageBytes;
-          const int nbox = min(KS, p.nchunk - s * KS);
+          const int nbox = kSplit ? max(0, min(KS, nch - s * KS)) : min(KS, nch - s * KS);   // a short last part can leave a stage empty
           mbar_expect_tx(bar, (uint32_t)nbox * box);
           for (int j = 0; j < nbox; j++)
-            tma_load_2d(dst + (uint32_t)j * box, &maps.m[pi], (s * KS + j) * kChunkWords, row0, bar);
+            tma_load_2d(dst + (uint32_t)j * box, &maps.m[pi], (chunk0 + s * KS + j) * kChunkWords, row0, bar);
           issued++;
           if (++slot == stages) { slot = 0; phase ^= 1u; }
         }
       }
+    }
     }
     return;
   }
@@ -293,6 +309,14 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   // belong to the kernel before this one: wait for it.
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
+  // ring position, barrier parity and reduction-buffer parity carried from one part of K to the next
+  int slot_keep = 0, nred_keep = 0;
+  uint32_t phase_keep = 0;
+  int* const s_part = reinterpret_cast<int*>(gen + p.off_part);   // [group of this CTA][16 rows][M][3]
+  for (int kp = 0; kp < nsplit; kp++) {
+  const int chunk0 = kSplit ? kp * p.nchunk : 0;                                    // this part of K
+  const int nch = kSplit ? min(p.nchunk, p.nchunk_total - chunk0) : p.nchunk;
+  if (kp > 0) asm volatile("bar.sync 1, %0;" ::"n"(kCWarps * 32) : "memory");        // every warp is done with the last part's activations
   // ------------------------------------------------------------------ fused quantizer (consumer warps)
   if constexpr (FQ) {
     static_assert(!FQ || (MODE == kModeDp4a && MTOK == 1), "the fused quantizer serves the one-token kernels");
@@ -366,7 +390,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
       const int pair = u >> 4;
       const int col = (int)(((uint32_t)pair * (uint32_t)p.inv_nchunk) >> 20), ch = pair - col * p.nchunk;   // pair / nchunk
       const int lo = u & 3, hi = (u >> 2) & 3;
-      const int wx = ch * kChunkWords + (kRelabel ? 8 * hi + 2 * lo : 8 * lo + 2 * hi);   // word index in the row
+      const int wx = (chunk0 + ch) * kChunkWords + (kRelabel ? 8 * hi + 2 * lo : 8 * lo + 2 * hi);   // word index in the row
       uint4 x = make_uint4(0, 0, 0, 0);
       if (u < total && wx < W) x = __ldg(reinterpret_cast<const uint4*>(p.xq + (size_t)col * (p.K / 2)) + (wx >> 1));
       return x;
@@ -376,7 +400,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
       const int pair = u >> 4;
       const int col = (int)(((uint32_t)pair * (uint32_t)p.inv_nchunk) >> 20), ch = pair - col * p.nchunk;
       const int lo = u & 3, hi = (u >> 2) & 3;
-      const int wx = ch * kChunkWords + 8 * lo + 2 * hi + w;
+      const int wx = (chunk0 + ch) * kChunkWords + 8 * lo + 2 * hi + w;
       uint4 x = make_uint4(0, 0, 0, 0);
       if (u < total && wx < W) x = __ldg(reinterpret_cast<const uint4*>(p.xq + (size_t)col * p.K) + wx);
       return x;
@@ -397,7 +421,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
       if (u < total) {
         const int lo = u & 3, hi = (u >> 2) & 3;   // lo: 16-byte slot t of the column block; hi: 2 i + pr, or the group
         if constexpr (!kPrefetch && !A16) {
-          const int wx = ch * kChunkWords + (kRelabel ? 8 * hi + 2 * lo : 8 * lo + 2 * hi);   // word index in the row
+          const int wx = (chunk0 + ch) * kChunkWords + (kRelabel ? 8 * hi + 2 * lo : 8 * lo + 2 * hi);   // word index in the row
           if (wx < W) x = __ldg(reinterpret_cast<const uint4*>(p.xq + (size_t)col * (p.K / 2)) + (wx >> 1));
         }
         uint32_t q[4][2];
@@ -866,11 +890,27 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     }
   };
 
-  int slot = 0;
-  uint32_t phase = 0;
   int T1[NE], T2[NE], T3[NE];
+  // finishes the rows of a group, or (K in parts) parks their sums until the last part has added its share
+  auto finish = [&](int row_first, int gslot) {
+    if (kSplit && nsplit > 1) {
+#pragma unroll
+      for (int e = 0; e < NE; e++) {
+        if (etok[e] < M) {
+          int* d = s_part + ((gslot * 16 + g + 8 * err[e]) * M + etok[e]) * 3;
+          if (kp > 0) { T1[e] += d[0]; T2[e] += d[1]; T3[e] += d[2]; }
+          if (kp + 1 < nsplit) { d[0] = T1[e]; d[1] = T2[e]; d[2] = T3[e]; }
+        }
+      }
+      if (kp + 1 < nsplit) return;
+    }
+    emit(row_first, T1, T2, T3);
+  };
 
-  int nred = 0;   // phases with a shared-memory reduction so far (its two buffers alternate)
+  int slot = slot_keep;
+  uint32_t phase = phase_keep;
+  int nred = nred_keep;   // phases with a shared-memory reduction so far (its two buffers alternate)
+  int gbase = 0;   // groups of this CTA before the current repetition, the same count in every part
   for (int pi = 0; pi < p.nphase; pi++) {
     const GemvPhase ph = p.phase[pi];
     if (b >= ph.ncta) continue;
@@ -882,6 +922,8 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     const uint32_t a_off = (uint32_t)ks * ((uint32_t)ph.gpc * kGroupBytes) + (uint32_t)grp * kGroupBytes;
     for (int rp = 0; rp < ph.reps; rp++) {
       const int row_first = (ph.first + rp * ph.total + lo + grp) * 16;
+      const int gslot = gbase + grp;
+      gbase += hi - lo;
       uint32_t b_chunk = (uint32_t)ks * chunk_stride;
       int ch = ks;
       if constexpr (GRP) {
@@ -918,14 +960,14 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
           if (lane == 0 && p.status) atomicExch(p.status, 3);
           return;
         }
-        if (active && ch < p.nchunk) compute_chunk(base + (uint32_t)slot * kStageBytes + a_off, b_chunk);
+        if (active && ch < nch) compute_chunk(base + (uint32_t)slot * kStageBytes + a_off, b_chunk);
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + 8 * slot);   // this warp is done with the slot
         if (++slot == stages) { slot = 0; phase ^= 1u; }
       }
       collect(T1, T2, T3);
       if (KS == 1) {
-        if (active) emit(row_first, T1, T2, T3);
+        if (active) finish(row_first, gslot);
       } else {
         // the KS warps of a group add up in shared memory; the first of them finishes the rows
         int* const red = s_red + (nred & 1) * (8 * 16 * M * 3);
@@ -949,11 +991,13 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
               d[0] = 0; d[1] = 0; d[2] = 0;   // ready for the reduction after next
             }
           }
-          emit(row_first, T1, T2, T3);
+          finish(row_first, gslot);
         }
       }
     }
   }
+  slot_keep = slot; phase_keep = phase; nred_keep = nred;
+  }   // parts of K
 }
 
 }  // namespace rcp

@@ -58,9 +58,9 @@ __device__ int g_pack_bad;  // set by pack_weights_kernel when it meets a code a
 // ---------------------------------------------------------------------------------------------
 // Streaming GEMV: launch plan.
 struct StreamPlan {
-  int nchunk, nphase, stages, grid;
+  int nchunk, nchunk_total, nsplit, nphase, stages, grid;   // nchunk: chunks per row in one part of K
   rcp::GemvPhase phase[rcp::kMaxPhases];
-  int off_bar, off_T0c, off_scale, off_red, off_bs, off_qbuf;
+  int off_bar, off_T0c, off_scale, off_red, off_bs, off_qbuf, off_part;
   size_t smem;
 };
 
@@ -77,6 +77,27 @@ int tokens_per_pass(int M, int K, int cap) {
   }
   int m = std::min(M, cap);
   while (m > 1 && (size_t)m * K > kExpandBudget) m--;
+  return m;
+}
+
+// The tensor-core kernels of the per-row grid rather keep their (up to eight) tokens and go through K in
+// parts when the expanded activations of the whole K would not fit: the weights are then streamed once, not
+// once per launch. Falls back to fewer tokens when the sums parked between the parts leave no room for a
+// ring of three stages (very many rows per CTA). Returns the tokens per launch, *nsplit the parts of K.
+StreamPlan make_plan(int M, int N, int K, int sms, bool grouped = false, size_t qbuf = 0, int nsplit = 1);
+int tokens_and_parts(int M, int N, int K, int cap, int sms, int* nsplit) {
+  *nsplit = 1;
+  const int m = tokens_per_pass(M, K, cap);
+  if (cap < 8 || m > 8) return m;
+  const int want = std::min(M, 8);
+  if (m == want) return m;
+  for (int parts = (int)(((size_t)want * K + kExpandBudget - 1) / kExpandBudget); parts <= 8; parts++) {
+    const StreamPlan pl = make_plan(want, N, K, sms, false, 0, parts);
+    if (pl.stages >= 3 && pl.smem <= kSmemMax) {
+      *nsplit = pl.nsplit;
+      return want;
+    }
+  }
   return m;
 }
 
@@ -139,10 +160,14 @@ int plan_leftover(int rem, int sms, int nchunk, rcp::GemvPhase* out) {
 }
 
 // qbuf: bytes of staging for the fused quantizer's cross-warp rotation strides (0 if unused)
-StreamPlan make_plan(int M, int N, int K, int sms, bool grouped = false, size_t qbuf = 0) {
+// nsplit: parts of K the kernel goes through one after the other (tensor-core kernels of the per-row grid)
+StreamPlan make_plan(int M, int N, int K, int sms, bool grouped, size_t qbuf, int nsplit) {
   StreamPlan pl;
   pl.grid = sms;
-  pl.nchunk = (K / 16 + rcp::kChunkWords - 1) / rcp::kChunkWords;
+  pl.nchunk_total = (K / 16 + rcp::kChunkWords - 1) / rcp::kChunkWords;
+  pl.nsplit = std::max(1, std::min(nsplit, pl.nchunk_total));
+  pl.nchunk = (pl.nchunk_total + pl.nsplit - 1) / pl.nsplit;
+  pl.nsplit = (pl.nchunk_total + pl.nchunk - 1) / pl.nchunk;   // no empty part
   // Phases: first the groups left over when every CTA takes 16 per round, then the rounds.
   const int groups = (N + 15) / 16;
   const int per_round = sms * rcp::kCWarps;
@@ -155,8 +180,13 @@ StreamPlan make_plan(int M, int N, int K, int sms, bool grouped = false, size_t 
   // row groups x 3 planes, or (group-wise grid) one fp32 term per warp
   const size_t t0c_bytes = grouped ? (size_t)(M + 1) * pl.nchunk * 16 : (((size_t)M * pl.nchunk * 4) + 15) / 16 * 16;
   const size_t red_bytes = grouped ? (size_t)2 * rcp::kCWarps * 16 * M * 4 : (size_t)2 * 8 * 16 * M * 3 * 4;
-  const size_t misc = 128 + t0c_bytes + 256 + red_bytes + qbuf;
-  pl.stages = (int)std::min<size_t>(rcp::kMaxStages, (kSmemMax - 1024 - misc - bs_bytes) / rcp::kStageBytes);
+  // K in parts: the integer sums of every group this CTA owns wait in shared memory between the parts
+  int own_groups = 0;
+  for (int i = 0; i < pl.nphase; i++) own_groups += pl.phase[i].reps * (pl.phase[i].q + (pl.phase[i].r ? 1 : 0));
+  const size_t part_bytes = pl.nsplit > 1 ? (size_t)own_groups * 16 * M * 3 * 4 : 0;
+  const size_t misc = 128 + t0c_bytes + 256 + red_bytes + qbuf + part_bytes;
+  const size_t fixed = 1024 + misc + bs_bytes;
+  pl.stages = fixed >= kSmemMax ? 0 : (int)std::min<size_t>(rcp::kMaxStages, (kSmemMax - fixed) / rcp::kStageBytes);
   size_t off = (size_t)pl.stages * rcp::kStageBytes;
   pl.off_bar = (int)off; off += 128;
   pl.off_T0c = (int)off; off += t0c_bytes;
@@ -164,6 +194,7 @@ StreamPlan make_plan(int M, int N, int K, int sms, bool grouped = false, size_t 
   pl.off_red = (int)off; off += red_bytes;
   pl.off_bs = (int)off; off += bs_bytes;
   pl.off_qbuf = (int)off; off += qbuf;
+  pl.off_part = (int)off; off += part_bytes;
   pl.smem = off + 1024;
   return pl;
 }
@@ -194,10 +225,10 @@ int sm_count() {
   return n;
 }
 
-template <int MODE, int MTOK, bool GRP = false, bool FQ = false, bool A16 = false>
+template <int MODE, int MTOK, bool GRP = false, bool FQ = false, bool A16 = false, bool SPLIT = false>
 int launch_stream_t(const rcp::GemvMaps& maps, const rcp::GemvParams& gp, const StreamPlan& pl, cudaStream_t st) {
   static bool attr_set = false;
-  auto kern = rcp::gemv_stream_kernel<MODE, MTOK, GRP, FQ, A16>;
+  auto kern = rcp::gemv_stream_kernel<MODE, MTOK, GRP, FQ, A16, SPLIT>;
   if (!attr_set) {
     RCP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax));
     attr_set = true;
@@ -224,7 +255,8 @@ bool fused_ok(int M, int K, int B) { return M == 1 && B == K && (K == 4096 || K 
 
 int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const uint8_t* xq, const void* scale_f16,
                   int M, int N, int K, void* y_f16, void* workspace, cudaStream_t st, bool grouped = false,
-                  const FusedAct* fa = nullptr, const float* unit = nullptr) {
+                  const FusedAct* fa = nullptr, const float* unit = nullptr, int nsplit = 1) {
+  if (nsplit > 1 && (mode != rcp::kModeMma || grouped || fa || M > 8)) return RCP_ERR_VARIANT;
   // unit: weight-only form; xq then holds M digit columns of K signed bytes (four per token), scale_f16 is unused
   if (unit && (mode != rcp::kModeMma || grouped || fa || M % 4)) return RCP_ERR_VARIANT;
   if (mode != rcp::kModeMma && M > 2) return RCP_ERR_VARIANT;
@@ -233,7 +265,7 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   if (fa && (mode != rcp::kModeDp4a || !fused_ok(M, K, fa->B))) return RCP_ERR_VARIANT;
   EncodeTiledFn enc = encode_tiled_fn();
   if (!enc) return cuda_fail(cudaErrorNotSupported);
-  const StreamPlan pl = make_plan(M, N, K, sm_count(), grouped, fa ? (size_t)4 * K : 0);
+  const StreamPlan pl = make_plan(M, N, K, sm_count(), grouped, fa ? (size_t)4 * K : 0, nsplit);
   if (pl.stages < 2 || pl.smem > kSmemMax) return RCP_ERR_SHAPE;
   // Tensor maps of the phases in use (the others repeat the first). Encoding one costs the host about a
   // microsecond, so the maps of the last few (weights, shape, boxes) combinations are remembered per thread.
@@ -279,6 +311,9 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   gp.M = M; gp.N = N; gp.K = K;
   gp.ngrp = grouped ? K / 128 : 0;
   gp.nchunk = pl.nchunk;
+  gp.nchunk_total = pl.nchunk_total;
+  gp.nsplit = pl.nsplit;
+  gp.off_part = pl.off_part;
   gp.inv_nchunk = ((1 << 20) + pl.nchunk - 1) / pl.nchunk;
   gp.nphase = pl.nphase;
   for (int i = 0; i < rcp::kMaxPhases; i++) gp.phase[i] = i < pl.nphase ? pl.phase[i] : make_phase(1, 0, 0, 1, 0, pl.nchunk);
@@ -299,9 +334,11 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
     return grouped ? launch_stream_t<rcp::kModeDp4a, 1, true, true>(maps, gp, pl, st)
                    : launch_stream_t<rcp::kModeDp4a, 1, false, true>(maps, gp, pl, st);
   }
-  if (unit)
+  if (unit) {
+    if (pl.nsplit > 1) return launch_stream_t<rcp::kModeMma, 0, false, false, true, true>(maps, gp, pl, st);
     return M > 8 ? launch_stream_t<rcp::kModeMma, 16, false, false, true>(maps, gp, pl, st)
                  : launch_stream_t<rcp::kModeMma, 0, false, false, true>(maps, gp, pl, st);
+  }
   if (grouped) {
     if (mode == rcp::kModeDp4a)
       return M == 1 ? launch_stream_t<rcp::kModeDp4a, 1, true>(maps, gp, pl, st)
@@ -314,6 +351,7 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   if (mode == rcp::kModeDp4a)
     return M == 1 ? launch_stream_t<rcp::kModeDp4a, 1>(maps, gp, pl, st)
                   : launch_stream_t<rcp::kModeDp4a, 2>(maps, gp, pl, st);
+  if (pl.nsplit > 1) return launch_stream_t<rcp::kModeMma, 0, false, false, false, true>(maps, gp, pl, st);
   return M > 8 ? launch_stream_t<rcp::kModeMma, 16>(maps, gp, pl, st) : launch_stream_t<rcp::kModeMma, 0>(maps, gp, pl, st);
 }
 
@@ -321,14 +359,16 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
 int launch_stream_passes(int mode, int cap, const uint32_t* words, const void* lut_f16, const uint8_t* xq,
                          const void* scale_f16, int M, int N, int K, void* y_f16, void* workspace, cudaStream_t st,
                          bool grouped = false) {
-  const int mp = tokens_per_pass(M, K, cap);
+  int nsplit = 1;
+  const int mp = (grouped || cap < 8) ? tokens_per_pass(M, K, cap) : tokens_and_parts(M, N, K, cap, sm_count(), &nsplit);
   for (int m0 = 0; m0 < M; m0 += mp) {
     const int mm = std::min(mp, M - m0);
     int md = mode;
     if (md == rcp::kModeHybrid && mm > 2) md = rcp::kModeMma;
     const int rc = launch_stream(md, words, lut_f16, xq + (size_t)m0 * (K / 2),
                                  static_cast<const __half*>(scale_f16) + m0, mm, N, K,
-                                 static_cast<__half*>(y_f16) + (size_t)m0 * N, workspace, st, grouped);
+                                 static_cast<__half*>(y_f16) + (size_t)m0 * N, workspace, st, grouped, nullptr, nullptr,
+                                 md == rcp::kModeMma ? nsplit : 1);
     if (rc != RCP_OK) return rc;
   }
   return RCP_OK;
@@ -500,9 +540,10 @@ int rcp_gemv_plan(int M, int N, int K, int sms, int* out, int cap) {
   if (!out && cap > 0) return RCP_ERR_NULL;
   if (M < 1 || M > rcp::kMaxTokens || N < 1 || !k_ok(K)) return RCP_ERR_SHAPE;
   if (sms <= 0) sms = 148;
-  const int mp = tokens_per_pass(M, K, 16);
-  const StreamPlan pl = make_plan(mp, N, K, sms);
-  int v[6 + 5 * rcp::kMaxPhases];
+  int nsplit = 1;
+  const int mp = tokens_and_parts(M, N, K, 16, sms, &nsplit);
+  const StreamPlan pl = make_plan(mp, N, K, sms, false, 0, nsplit);
+  int v[7 + 5 * rcp::kMaxPhases];
   int n = 0;
   v[n++] = mp;
   v[n++] = (M + mp - 1) / mp;
@@ -514,6 +555,7 @@ int rcp_gemv_plan(int M, int N, int K, int sms, int* out, int cap) {
     v[n++] = pl.phase[i].gpc; v[n++] = pl.phase[i].first; v[n++] = pl.phase[i].total;
     v[n++] = pl.phase[i].ncta; v[n++] = pl.phase[i].reps;
   }
+  v[n++] = pl.nsplit;
   for (int i = 0; i < n && i < cap; i++) out[i] = v[i];
   return n;
 }
@@ -578,8 +620,9 @@ int rcp_gemv_w2a16(const uint32_t* words, const void* lut_f16, const void* x_f16
     return RCP_ERR_ALIGN;
   // digit columns per launch: sixteen (four tokens) or eight (two) where their expanded bytes fit, else four
   const int cols = 4 * M;
-  const int cp = tokens_per_pass(std::min(cols, 16), K, 16) & ~3;
-  if (cp < 4) return RCP_ERR_SHAPE;   // K beyond 32768: the four digit planes of one token do not fit
+  int nsplit = 1;
+  const int cp = tokens_and_parts(std::min(cols, 16), N, K, 16, sm_count(), &nsplit) & ~3;
+  if (cp < 4) return RCP_ERR_SHAPE;   // not even the four digit planes of one token fit (very many rows and a long K)
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   RCP_CUDA(launch_overlapped(rcp::split_act16_kernel, dim3(M), dim3(rcp::kSplitThreads), 0, st,
                              static_cast<const __half*>(x_f16), K, digits, unit));
@@ -587,7 +630,7 @@ int rcp_gemv_w2a16(const uint32_t* words, const void* lut_f16, const void* x_f16
     const int cc = std::min(cp, cols - c0);
     const int rc = launch_stream(rcp::kModeMma, words, lut_f16, reinterpret_cast<const uint8_t*>(digits) + (size_t)c0 * K,
                                  nullptr, cc, N, K, static_cast<__half*>(y_f16) + (size_t)(c0 / 4) * N, workspace, st,
-                                 false, nullptr, unit + c0);
+                                 false, nullptr, unit + c0, nsplit);
     if (rc != RCP_OK) return rc;
   }
   return RCP_OK;
@@ -650,13 +693,14 @@ int rcp_gemv_w2a4_static(const uint32_t* words, const void* lut_f16, const uint8
                                stream);
 }
 
-int rcp_linear_w2a4_launches(int M, int K, int had_block, int group) {
-  if (M < 1 || M > rcp::kMaxTokens || !k_ok(K)) return RCP_ERR_SHAPE;
+int rcp_linear_w2a4_launches(int M, int N, int K, int had_block, int group) {
+  if (M < 1 || M > rcp::kMaxTokens || N < 1 || !k_ok(K)) return RCP_ERR_SHAPE;
   const int B = had_block <= 1 ? 1 : had_block;
   if (fused_ok(M, K, B) && (group == 0 || group == 128)) return 1;
   if (group != 0 && group != 128) return 2;
   const int cap = group == 0 ? (M == 1 ? 2 : 16) : (M <= 2 ? 2 : 8);   // tokens per launch of the variant AUTO picks
-  const int mp = tokens_per_pass(M, K, cap);
+  int nsplit = 1;
+  const int mp = (group != 0 || cap < 8) ? tokens_per_pass(M, K, cap) : tokens_and_parts(M, N, K, cap, sm_count(), &nsplit);
   return 1 + (M + mp - 1) / mp;
 }
 

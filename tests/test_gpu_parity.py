@@ -129,6 +129,8 @@ SMALL = [
     # 9 to 16 tokens in one launch (two column tiles) where they fit, in two launches where they do not
     (2500, 4096, 4096, 9), (5000, 2048, 128, 13), (300, 6144, 128, 13), (70, 5120, 64, 16), (70, 5184, 64, 16),
     (37965, 512, 128, 16), (2369, 1024, 1024, 12),
+    # several tokens and a long K: one launch goes through K in parts (the last one shorter, or ending inside a chunk)
+    (64, 28672, 128, 8), (1000, 20480, 128, 7), (2400, 16448, 64, 8), (33, 65536, 128, 5), (300, 32768, 8192, 16),
 ]
 
 

@@ -50,7 +50,8 @@ def _check(N, K, M, seed, kind="rotated_laplace", x=None, rows=None):
 
 @pytest.mark.parametrize("N,K,M", [(1, 64, 1), (17, 192, 3), (100, 320, 2), (127, 1024, 4), (300, 2048, 1),
                                    (256, 4096, 4), (130, 11008, 1), (64, 28672, 2), (33, 8192, 5), (40, 32768, 1),
-                                   (513, 1088, 16), (2500, 4096, 3), (5000, 2048, 7), (2369, 5120, 4), (37965, 512, 2)])
+                                   (513, 1088, 16), (2500, 4096, 3), (5000, 2048, 7), (2369, 5120, 4), (37965, 512, 2),
+                                   (40, 65536, 2), (300, 28672, 3), (2400, 16448, 2)])
 def test_w2a16_small_and_ragged(N, K, M):
     _check(N, K, M, seed=N + K + M, kind="rotated_laplace" if K >= 512 else "uniform")
 
@@ -118,5 +119,5 @@ def test_w2a16_argument_errors():
     assert L.rcp_gemv_w2a16(None, p, p, 1, 16, 64, p, p, p, p, None) == -1
     assert L.rcp_gemv_w2a16(p, p, p, 0, 16, 64, p, p, p, p, None) == -2
     assert L.rcp_gemv_w2a16(p, p, p, 17, 16, 64, p, p, p, p, None) == -2
-    assert L.rcp_gemv_w2a16(p, p, p, 1, 16, 32832, p, p, p, p, None) == -2   # four digit planes of K > 32768 do not fit
+    assert L.rcp_gemv_w2a16(p, p, p, 1, 16, 65600, p, p, p, p, None) == -2   # K above the library's limit
     assert L.rcp_gemv_w2a16(p, p, p + 2, 1, 16, 64, p, p, p, p, None) == -3

@@ -22,7 +22,7 @@ def plan(L, M, N, K, sms=148):
     assert n >= 6, n
     v = list(buf[:n])
     phases = [tuple(v[6 + 5 * i: 11 + 5 * i]) for i in range(v[5])]
-    return dict(tokens=v[0], launches=v[1], stages=v[2], smem=v[3], nchunk=v[4], phases=phases)
+    return dict(tokens=v[0], launches=v[1], stages=v[2], smem=v[3], nchunk=v[4], phases=phases, parts=v[6 + 5 * v[5]])
 
 
 def check(L, M, N, K, sms=148):
@@ -44,10 +44,14 @@ def check(L, M, N, K, sms=148):
         nxt += total * reps
     assert nxt == groups, (nxt, groups)
     assert len(p["phases"]) <= 6
-    assert p["nchunk"] == -(-K // 512)
+    total_chunks = -(-K // 512)
+    assert 1 <= p["parts"] <= 8 and p["nchunk"] == -(-total_chunks // p["parts"])   # chunks per part of K
+    assert (p["parts"] - 1) * p["nchunk"] < total_chunks                             # no empty part
     assert p["stages"] >= 2 and p["smem"] <= 232448
     assert 1 <= p["tokens"] <= 16 and p["tokens"] * p["launches"] >= M
-    assert p["tokens"] == 1 or p["tokens"] * K <= 128 * 1024   # expanded activations fit
+    assert p["tokens"] == 1 or p["tokens"] * p["nchunk"] * 512 <= 128 * 1024   # expanded activations of a part fit
+    if p["parts"] > 1:
+        assert p["tokens"] == min(M, 8) and p["stages"] >= 3
     if p["tokens"] > 8:   # one launch with two column tiles: all the tokens, and a tighter budget
         assert p["tokens"] == M and p["launches"] == 1 and M * K <= 80 * 1024 and p["stages"] >= 3
     return p
@@ -82,8 +86,15 @@ def test_plan_examples(L):
     assert (check(L, 10, 4096, 8192)["tokens"], check(L, 10, 4096, 8192)["launches"]) == (10, 1)
     assert (check(L, 16, 4096, 5184)["tokens"], check(L, 16, 4096, 5184)["launches"]) == (8, 2)
     assert (check(L, 16, 4096, 11008)["tokens"], check(L, 16, 4096, 11008)["launches"]) == (8, 2)
-    assert check(L, 8, 8192, 28672)["tokens"] == 4
-    assert check(L, 16, 64, 65536)["tokens"] == 2
+    # long K: the launch keeps its eight tokens and goes through K in parts
+    p = check(L, 8, 8192, 28672)
+    assert (p["tokens"], p["launches"], p["parts"]) == (8, 1, 3)
+    p = check(L, 16, 64, 65536)
+    assert (p["tokens"], p["launches"], p["parts"]) == (8, 2, 6)
+    assert check(L, 1, 8192, 28672)["parts"] == 1 and check(L, 2, 64, 65536)["parts"] == 1
+    # so many rows per CTA that the parked sums leave no room for the ring: fewer tokens instead
+    p = check(L, 8, 300000, 28672)
+    assert p["parts"] == 1 and p["tokens"] == 4
 
 
 def test_plan_rejects_bad_shapes(L):
