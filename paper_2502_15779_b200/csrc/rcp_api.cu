@@ -90,7 +90,7 @@ int tokens_and_parts(int M, int N, int K, int cap, int sms, int* nsplit) {
   const int m = tokens_per_pass(M, K, cap);
   if (cap < 8 || m > 8) return m;
   const int want = std::min(M, 8);
-  if (m == want) return m;
+  if (m == want) return m;   // everything fits at once (measured: parts cost more than a ring of two stages does)
   for (int parts = (int)(((size_t)want * K + kExpandBudget - 1) / kExpandBudget); parts <= 8; parts++) {
     const StreamPlan pl = make_plan(want, N, K, sms, false, 0, parts);
     if (pl.stages >= 3 && pl.smem <= kSmemMax) {
