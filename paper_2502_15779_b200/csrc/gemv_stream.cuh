@@ -39,6 +39,7 @@
 
 #include "common.cuh"
 #include "quantize_act.cuh"
+#include "split_act16.cuh"
 
 namespace rcp {
 
@@ -71,6 +72,8 @@ struct GemvParams {
   const uint8_t* xq;
   const __half* scale;
   const float* unit;     // A16: fp32 unit of each digit column (scale unused)
+  float* unit_out;       // A16 with x set (one token): every CTA makes the digit planes itself (kept in shared
+                         // memory at off_qbuf); CTA 0 also stores them to xq_out ([4][K] bytes) and the units here
   __half* y;
   int32_t* status;      // optional: receives a code when a bounded wait gives up
   int M, N, K;
@@ -383,6 +386,55 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   // consecutive lanes: their sum of q is added to the token's total s_T0tot (per-row grid) or kept per group
   // of 128 in s_T0c (group-wise grid).
   {
+    // Weight-only form with the activations still in fp16: the digit planes of this CTA's copy are made
+    // here (the arithmetic of split_act16_kernel) and kept in shared memory.
+    uint8_t* const stg = gen + p.off_qbuf;   // [column][K] signed bytes
+    if constexpr (A16) {
+      if (p.x) {
+        // One token (the host asks for this form only then: with two, the stand-alone kernel in front was
+        // measured faster), its values held in registers between the two passes (up to four vectors of eight
+        // per thread: K <= 16384, which the host checks).
+        unsigned* const s_am = reinterpret_cast<unsigned*>(s_red);   // [16 warps]; s_red is cleared further down
+        const int nvec = p.K / 8;
+        uint4 xr[4];
+        unsigned amax = 0u;
+#pragma unroll
+        for (int r = 0; r < 4; r++) {
+          const int i = tid + r * (kCWarps * 32);
+          xr[r] = make_uint4(0, 0, 0, 0);
+          if (i < nvec) xr[r] = __ldg(reinterpret_cast<const uint4*>(p.x) + i);
+          amax = split_amax8(xr[r], amax);
+        }
+        amax = __reduce_max_sync(0xffffffffu, amax);
+        if (lane == 0) s_am[warp] = amax;
+        asm volatile("bar.sync 1, %0;" ::"n"(kCWarps * 32) : "memory");
+        amax = 0;
+#pragma unroll
+        for (int i = 0; i < kCWarps; i++) amax = max(amax, s_am[i]);
+        const int E = split_exponent(amax);
+        const float mult = __int_as_float((21 - E + 127) << 23);
+        if (tid < 4) {
+          const float un = __int_as_float((E - 21 + 6 * tid + 127) << 23);
+          s_scale[tid] = un;
+          if (b == 0 && p.unit_out) p.unit_out[tid] = un;
+        }
+#pragma unroll
+        for (int r = 0; r < 4; r++) {
+          const int i = tid + r * (kCWarps * 32);
+          if (i < nvec) {
+            uint32_t out[4][2];
+            split_digits8(xr[r], mult, out);
+#pragma unroll
+            for (int d = 0; d < 4; d++) {
+              const size_t at = (size_t)d * p.K + (size_t)i * 8;
+              *reinterpret_cast<uint2*>(stg + at) = make_uint2(out[d][0], out[d][1]);
+              if (b == 0 && p.xq_out) *reinterpret_cast<uint2*>(p.xq_out + at) = make_uint2(out[d][0], out[d][1]);
+            }
+          }
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(kCWarps * 32) : "memory");   // planes complete; s_red free to be cleared
+      }
+    }
     const int W = p.K / 16;
     const int total = ncol * p.nchunk * 16;
     // the two words of unit u (zeros past the end of the row or of the units)
@@ -402,7 +454,10 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
       const int lo = u & 3, hi = (u >> 2) & 3;
       const int wx = (chunk0 + ch) * kChunkWords + 8 * lo + 2 * hi + w;
       uint4 x = make_uint4(0, 0, 0, 0);
-      if (u < total && wx < W) x = __ldg(reinterpret_cast<const uint4*>(p.xq + (size_t)col * p.K) + wx);
+      if (u < total && wx < W) {
+        if (p.x) x = *(reinterpret_cast<const uint4*>(stg + (size_t)col * p.K) + wx);   // planes made above
+        else x = __ldg(reinterpret_cast<const uint4*>(p.xq + (size_t)col * p.K) + wx);
+      }
       return x;
     };
     // tensor-core kernels of the per-row grid (several tokens, so several units per thread): the next unit's
@@ -475,7 +530,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
         if ((u & 12) == 0 && u < total) s_T0c[col * ng4 + ch * 4 + (u & 3)] = tsum;
       }
     }
-    if (tid < M) s_scale[tid] = A16 ? p.unit[tid] : __half2float(p.scale[tid]);
+    if (tid < M && !(A16 && p.x)) s_scale[tid] = A16 ? p.unit[tid] : __half2float(p.scale[tid]);
     if constexpr (!GRP)
       for (int i = tid; i < 2 * 8 * 16 * M * 3; i += kCWarps * 32) s_red[i] = 0;
   }

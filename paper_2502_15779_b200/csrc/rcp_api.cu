@@ -251,12 +251,21 @@ struct FusedAct {
 // Shapes the in-kernel quantizer takes: one token of 4096 or 8192 elements under one rotation block.
 // Measured on B200: there the fused kernel beats the two kernels by 0.7 to 1.9 us a call; for shorter
 // tokens, block-wise rotation or two tokens the stand-alone quantizer (several CTAs per token) wins.
+// Weight-only form, activations still in fp16: the GEMV kernel makes the digit planes itself.
+struct SplitAct {
+  const void* x_f16;    // [tokens][K]
+  int8_t* digits_out;   // [tokens][4][K], written by CTA 0
+  float* unit_out;      // [tokens][4], written by CTA 0
+};
+
 bool fused_ok(int M, int K, int B) { return M == 1 && B == K && (K == 4096 || K == 8192); }
 
 int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const uint8_t* xq, const void* scale_f16,
                   int M, int N, int K, void* y_f16, void* workspace, cudaStream_t st, bool grouped = false,
-                  const FusedAct* fa = nullptr, const float* unit = nullptr, int nsplit = 1) {
+                  const FusedAct* fa = nullptr, const float* unit = nullptr, int nsplit = 1,
+                  const SplitAct* sa = nullptr) {
   if (nsplit > 1 && (mode != rcp::kModeMma || grouped || fa || M > 8)) return RCP_ERR_VARIANT;
+  if (sa && (mode != rcp::kModeMma || grouped || fa || unit || nsplit > 1 || M != 4 || K > 16384)) return RCP_ERR_VARIANT;
   // unit: weight-only form; xq then holds M digit columns of K signed bytes (four per token), scale_f16 is unused
   if (unit && (mode != rcp::kModeMma || grouped || fa || M % 4)) return RCP_ERR_VARIANT;
   if (mode != rcp::kModeMma && M > 2) return RCP_ERR_VARIANT;
@@ -265,7 +274,7 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   if (fa && (mode != rcp::kModeDp4a || !fused_ok(M, K, fa->B))) return RCP_ERR_VARIANT;
   EncodeTiledFn enc = encode_tiled_fn();
   if (!enc) return cuda_fail(cudaErrorNotSupported);
-  const StreamPlan pl = make_plan(M, N, K, sm_count(), grouped, fa ? (size_t)4 * K : 0, nsplit);
+  const StreamPlan pl = make_plan(M, N, K, sm_count(), grouped, fa ? (size_t)4 * K : (sa ? (size_t)M * K : 0), nsplit);
   if (pl.stages < 2 || pl.smem > kSmemMax) return RCP_ERR_SHAPE;
   // Tensor maps of the phases in use (the others repeat the first). Encoding one costs the host about a
   // microsecond, so the maps of the last few (weights, shape, boxes) combinations are remembered per thread.
@@ -323,7 +332,7 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   gp.off_bar = pl.off_bar; gp.off_T0c = pl.off_T0c; gp.off_scale = pl.off_scale; gp.off_red = pl.off_red;
   gp.off_bs = pl.off_bs;
   gp.off_qbuf = pl.off_qbuf;
-  gp.x = nullptr; gp.xq_out = nullptr; gp.scale_out = nullptr;
+  gp.x = nullptr; gp.xq_out = nullptr; gp.scale_out = nullptr; gp.unit_out = nullptr;
   gp.inv_sqrt_b = 1.f; gp.clip_ratio = 1.f;
   if (fa) {
     gp.x = static_cast<const __half*>(fa->x_f16);
@@ -333,6 +342,12 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
     gp.clip_ratio = fa->clip_ratio;
     return grouped ? launch_stream_t<rcp::kModeDp4a, 1, true, true>(maps, gp, pl, st)
                    : launch_stream_t<rcp::kModeDp4a, 1, false, true>(maps, gp, pl, st);
+  }
+  if (sa) {
+    gp.x = static_cast<const __half*>(sa->x_f16);
+    gp.xq_out = reinterpret_cast<uint8_t*>(sa->digits_out);
+    gp.unit_out = sa->unit_out;
+    return launch_stream_t<rcp::kModeMma, 0, false, false, true>(maps, gp, pl, st);
   }
   if (unit) {
     if (pl.nsplit > 1) return launch_stream_t<rcp::kModeMma, 0, false, false, true, true>(maps, gp, pl, st);
@@ -624,6 +639,15 @@ int rcp_gemv_w2a16(const uint32_t* words, const void* lut_f16, const void* x_f16
   const int cp = tokens_and_parts(std::min(cols, 16), N, K, 16, sm_count(), &nsplit) & ~3;
   if (cp < 4) return RCP_ERR_SHAPE;   // not even the four digit planes of one token fit (very many rows and a long K)
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // One token of up to 16384 elements: one kernel does both steps (every CTA splits its own copy of the
+  // activations, held in registers between the search for the largest magnitude and the digits, which costs
+  // less than a launch in front of it: measured 0.4 to 1.2 us a call; with two tokens the launch in front won).
+  if (M == 1 && nsplit == 1 && cp == cols && K <= 16384 &&
+      make_plan(cols, N, K, sm_count(), false, (size_t)cols * K, 1).stages >= 3) {
+    const SplitAct sa{x_f16, digits, unit};
+    return launch_stream(rcp::kModeMma, words, lut_f16, nullptr, nullptr, cols, N, K, y_f16, workspace, st, false,
+                         nullptr, nullptr, 1, &sa);
+  }
   RCP_CUDA(launch_overlapped(rcp::split_act16_kernel, dim3(M), dim3(rcp::kSplitThreads), 0, st,
                              static_cast<const __half*>(x_f16), K, digits, unit));
   for (int c0 = 0; c0 < cols; c0 += cp) {

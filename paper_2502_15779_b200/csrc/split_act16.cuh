@@ -11,6 +11,43 @@ namespace rcp {
 
 constexpr int kSplitThreads = 512;
 
+// floor(log2) of the largest magnitude of a token from its fp16 bit pattern (0 for an all-zero token)
+__device__ __forceinline__ int split_exponent(unsigned amax_bits) {
+  if (amax_bits >= 0x0400u) return (int)(amax_bits >> 10) - 15;        // normal
+  if (amax_bits > 0u) return (31 - __clz((int)amax_bits)) - 24;        // subnormal: mantissa * 2^-24
+  return 0;
+}
+// largest magnitude bit pattern among the eight fp16 values of v
+__device__ __forceinline__ unsigned split_amax8(uint4 v, unsigned amax) {
+  const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int j = 0; j < 4; j++) {
+    amax = max(amax, w[j] & 0x7FFFu);
+    amax = max(amax, (w[j] >> 16) & 0x7FFFu);
+  }
+  return amax;
+}
+// the four digit planes of eight consecutive fp16 values: out[d] = eight signed bytes of digit d
+__device__ __forceinline__ void split_digits8(uint4 v, float mult, uint32_t (&out)[4][2]) {
+  const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int d = 0; d < 4; d++) { out[d][0] = 0; out[d][1] = 0; }
+#pragma unroll
+  for (int j = 0; j < 8; j++) {
+    const __half h = __ushort_as_half((unsigned short)(j & 1 ? w[j >> 1] >> 16 : w[j >> 1] & 0xFFFFu));
+    int X = __float2int_rn(__fmul_rn(__half2float(h), mult));   // exact product, half-to-even
+#pragma unroll
+    for (int d = 0; d < 4; d++) {
+      int q = X;
+      if (d < 3) {
+        q = ((X + 32) & 63) - 32;   // residue in [-32, 31]
+        X = (X - q) >> 6;           // divisible: the shift is exact
+      }
+      out[d][j >> 2] |= (uint32_t)(q & 0xFF) << (8 * (j & 3));
+    }
+  }
+}
+
 // grid: one CTA per token. digits [M][4][K] int8, unit [M][4] fp32. K % 8 == 0, x 16-byte aligned.
 __global__ void __launch_bounds__(kSplitThreads) split_act16_kernel(const __half* __restrict__ x, int K,
                                                                      int8_t* __restrict__ digits,
@@ -23,45 +60,20 @@ __global__ void __launch_bounds__(kSplitThreads) split_act16_kernel(const __half
   const int nvec = K / 8;
   // largest magnitude: the bit patterns of finite fp16 magnitudes order like the values
   unsigned amax = 0;
-  for (int i = tid; i < nvec; i += kSplitThreads) {
-    const uint4 v = __ldg(xv + i);
-    const unsigned w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int j = 0; j < 4; j++) {
-      amax = max(amax, w[j] & 0x7FFFu);
-      amax = max(amax, (w[j] >> 16) & 0x7FFFu);
-    }
-  }
+  for (int i = tid; i < nvec; i += kSplitThreads) amax = split_amax8(__ldg(xv + i), amax);
   amax = __reduce_max_sync(0xffffffffu, amax);
   if ((tid & 31) == 0) s_max[tid >> 5] = amax;
   __syncthreads();
   amax = 0;
 #pragma unroll
   for (int i = 0; i < kSplitThreads / 32; i++) amax = max(amax, s_max[i]);
-  int E = 0;
-  if (amax >= 0x0400u) E = (int)(amax >> 10) - 15;          // normal
-  else if (amax > 0u) E = (31 - __clz((int)amax)) - 24;     // subnormal: mantissa * 2^-24
+  const int E = split_exponent(amax);
   const float mult = __int_as_float((21 - E + 127) << 23);  // 2^(21 - E), between 2^6 and 2^45
   if (tid < 4) unit[m * 4 + tid] = __int_as_float((E - 21 + 6 * tid + 127) << 23);
   int8_t* const dg = digits + (size_t)m * 4 * K;
   for (int i = tid; i < nvec; i += kSplitThreads) {
-    const uint4 v = __ldg(xv + i);
-    const unsigned w[4] = {v.x, v.y, v.z, v.w};
-    uint32_t out[4][2] = {};
-#pragma unroll
-    for (int j = 0; j < 8; j++) {
-      const __half h = __ushort_as_half((unsigned short)(j & 1 ? w[j >> 1] >> 16 : w[j >> 1] & 0xFFFFu));
-      int X = __float2int_rn(__fmul_rn(__half2float(h), mult));   // exact product, half-to-even
-#pragma unroll
-      for (int d = 0; d < 4; d++) {
-        int q = X;
-        if (d < 3) {
-          q = ((X + 32) & 63) - 32;   // residue in [-32, 31]
-          X = (X - q) >> 6;           // divisible: the shift is exact
-        }
-        out[d][j >> 2] |= (uint32_t)(q & 0xFF) << (8 * (j & 3));
-      }
-    }
+    uint32_t out[4][2];
+    split_digits8(__ldg(xv + i), mult, out);
 #pragma unroll
     for (int d = 0; d < 4; d++)
       *reinterpret_cast<uint2*>(dg + (size_t)d * K + (size_t)i * 8) = make_uint2(out[d][0], out[d][1]);
