@@ -106,7 +106,9 @@ enum { RCP_GEMV_AUTO = 0, RCP_GEMV_SIMPLE = 1, RCP_GEMV_DP4A = 2, RCP_GEMV_MMA =
  * fp32 finish and the fp16 rounding of y.
  *   words, lut_f16   DEVICE, as for rcp_gemv_w2a4 (per-row grid).
  *   x_f16            DEVICE fp16 [M][K], finite; 16-byte aligned.
- *   M                1..16 (two tokens per launch, four while 16 * K <= 80 KiB); K % 64 == 0.
+ *   M                1..16 (two tokens per launch, four while 16 * K <= 80 KiB; one token of up to 16384
+ *                    elements is split into its digits by the GEMV kernel itself, otherwise a small
+ *                    kernel in front does that); K % 64 == 0.
  *   y_f16            DEVICE fp16 [M][N], written.
  *   digits           DEVICE int8 [M][4][K], written: the digit planes (16-byte aligned).
  *   unit             DEVICE fp32 [M][4], written: the unit of each digit plane.
