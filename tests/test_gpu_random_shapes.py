@@ -69,6 +69,33 @@ def test_random_shape(N, K, M, variant, grouped, i):
         assert np.all(np.abs(got - ref["y"]) <= ref["tol"])
 
 
+@pytest.mark.parametrize("N,K,M,variant,grouped,i", [c for c in _cases(48, 20250215) if not c.values[4]][:20])
+def test_random_shape_weight_only(N, K, M, variant, grouped, i):
+    """The same sweep through the weight-only form (fp16 activations): digits bit for bit, y within the bound
+    its arithmetic gives."""
+    seed = 7000 + i
+    codes, lut = synth.make_layer(N, K, 64, "uniform", seed, device=DEV)
+    x = synth.make_activations(M, K, seed, device=DEV)
+    words = rcp.rcp_pack_weights(codes)
+    digits = torch.empty((M, 4, K), dtype=torch.int8, device=DEV)
+    unit = torch.empty((M, 4), dtype=torch.float32, device=DEV)
+    ws = rcp.make_workspace(M, N, K, DEV)
+    y = rcp.rcp_gemv_w2a16(words, lut, x, digits=digits, unit=unit, workspace=ws)
+    torch.cuda.synchronize()
+    assert int(ws.abs().max()) == 0
+    sp = oracle.split_act16(f16_bits(x))
+    assert np.array_equal(digits.cpu().numpy(), sp["digits"])
+    assert np.array_equal(unit.cpu().numpy().astype(np.float64), sp["unit"])
+    rows = np.arange(N) if N * K * M <= 1 << 24 else np.unique(np.concatenate(
+        [np.arange(64), np.arange(N - 64, N), np.random.default_rng(i).integers(0, N, size=256)]))
+    ref = oracle.gemv_w2a16(oracle.pack_weights(codes.cpu().numpy()[rows]), np.ascontiguousarray(f16_bits(lut)[rows]),
+                            f16_bits(x))
+    tol = (0.5 * sp["unit"][:, :1] * ref["labs"][None, :] + 2.0 ** -20 * ref["labsx"]
+           + 2.0 ** -11 * np.abs(ref["y"]) + 2.0 ** -24)
+    got = y.float().cpu().numpy().astype(np.float64)[:, rows]
+    assert np.all(np.isfinite(got)) and np.all(np.abs(got - ref["y"]) <= tol)
+
+
 @pytest.mark.parametrize("N,K,M,grouped", [(70, 65536, 1, False), (40, 65536, 8, False), (33, 65536, 2, True),
                                            (20, 65536, 5, True), (300000, 64, 1, False), (150000, 128, 3, True),
                                            (1, 64, 16, False), (1, 128, 16, True)])
