@@ -128,10 +128,13 @@ def test_extreme_shapes(N, K, M, grouped):
 
 
 @pytest.mark.parametrize("N,K,M,variant,grouped", [(4096, 4096, 1, "auto", False), (5000, 2048, 8, "auto", False),
-                                                   (3000, 11008, 2, "auto", True), (2600, 8192, 1, "linear", False)])
+                                                   (3000, 11008, 2, "auto", True), (2600, 8192, 1, "linear", False),
+                                                   (2500, 20480, 8, "auto", False), (5000, 4096, 16, "auto", False),
+                                                   (3000, 4096, 1, "w2a16", False), (2500, 20480, 2, "w2a16", False)])
 def test_many_launches_repeat_bit_for_bit(N, K, M, variant, grouped):
     """A few thousand back-to-back launches (the ring, its barriers and the phases restart every time): the
-    status word stays clear and every launch returns the same bits."""
+    status word stays clear and every launch returns the same bits. Covers the forms with shared-memory state of
+    their own as well: K in parts, two column tiles, the weight-only form with and without the split inside."""
     B = K if (K & (K - 1)) == 0 else 128
     if grouped:
         codes, lut = synth.make_layer_grouped(N, K, 128, B, "uniform", 77, device=DEV)
@@ -143,8 +146,13 @@ def test_many_launches_repeat_bit_for_bit(N, K, M, variant, grouped):
     ws = rcp.make_workspace(M, N, K, DEV)
     ys = [torch.empty(M, N, dtype=torch.float16, device=DEV) for _ in range(2)]
 
+    dg = torch.empty(M, 4, K, dtype=torch.int8, device=DEV)
+    un = torch.empty(M, 4, dtype=torch.float32, device=DEV)
+
     def launch(y):
-        if variant == "linear":
+        if variant == "w2a16":
+            rcp.rcp_gemv_w2a16(words, lut, x, y=y, digits=dg, unit=un, workspace=ws)
+        elif variant == "linear":
             rcp.rcp_linear_w2a4(x, B, 1.0, words, lut, y=y, xq=xq, scale=scale, workspace=ws)
         elif grouped:
             rcp.rcp_gemv_w2a4_grouped(words, lut, xq, scale, group=128, y=y, workspace=ws)
