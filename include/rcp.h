@@ -119,6 +119,15 @@ int rcp_gemv_w2a16(const uint32_t* words, const void* lut_f16, const void* x_f16
                    int8_t* digits, float* unit, void* workspace, void* stream);
 
 /*
+ * rcp_gemv_w2a16 with the integer sums exported, for parity tests (same section of the paper). S_dbg int32
+ * [4 M][N][4]: for digit plane d of token m, entry [4 m + d][n][c] is the sum of that plane's digits over the
+ * weights of row n whose code is c, taken from the checked instantiation of the kernel that runs anyway.
+ * S_dbg NULL: rcp_gemv_w2a16.
+ */
+int rcp_gemv_w2a16_checked(const uint32_t* words, const void* lut_f16, const void* x_f16, int M, int N, int K,
+                           void* y_f16, int8_t* digits, float* unit, void* workspace, int32_t* S_dbg, void* stream);
+
+/*
  * Bytes of caller-provided scratch rcp_gemv_w2a4 needs for this shape (0 on bad shapes). The scratch
  * holds a status word that a kernel sets if one of its bounded waits ever gives up (0 = fine). It
  * must be zero-filled once after allocation; every successful call leaves it zero-filled, so one
@@ -148,14 +157,18 @@ int rcp_gemv_plan(int M, int N, int K, int sms, int* out, int cap);
  *   words, lut_f16 are the constants of the layer: the kernel may start fetching them while earlier
  *              work on the stream is still running (programmatic dependent launch), so that work
  *              must not be writing them. xq, scale, y and workspace obey stream order as usual.
- *   S_dbg      NULL in production. Otherwise int32 [M][N][4] receives S_c (runs the SIMPLE variant).
+ *   S_dbg      NULL in production. Otherwise int32 [M][N][4] receives S_c, 16-byte aligned; this entry point
+ *              then runs the SIMPLE variant. (rcp_gemv_w2a4_variant with a streaming variant and S_dbg runs
+ *              the checked instantiation of that very kernel: the same code, which also stores the integer
+ *              sums it finishes its rows from. The production instantiations contain no such store.)
  * Never synchronizes.
  */
 int rcp_gemv_w2a4(const uint32_t* words, const void* lut_f16, const uint8_t* xq,
                   const void* scale_f16, int M, int N, int K, void* y_f16, void* workspace,
                   int32_t* S_dbg, void* stream);
 
-/* Same, with the kernel variant chosen by the caller (for benchmarks and profiles). */
+/* Same, with the kernel variant chosen by the caller (for benchmarks, profiles and the parity tests: with
+ * S_dbg set and a variant other than RCP_GEMV_AUTO, S_c comes from the chosen kernel itself). */
 int rcp_gemv_w2a4_variant(int variant, const uint32_t* words, const void* lut_f16,
                           const uint8_t* xq, const void* scale_f16, int M, int N, int K,
                           void* y_f16, void* workspace, int32_t* S_dbg, void* stream);
@@ -194,7 +207,9 @@ int rcp_ldp_export(const void* w_f16, const float* sig_beta, const float* sig_ga
  *   lut_f16    DEVICE fp16 [N][K/group][4], 8-byte aligned. A constant of the layer like `words`.
  *   group      a multiple of 16 that divides K. group == 128 runs the streaming kernels; any
  *              other size runs the plain kernel (correct, not tuned).
- *   S_dbg      NULL in production. Otherwise int32 [M][N][K/group][4] receives S_c (plain kernel).
+ *   S_dbg      NULL in production. Otherwise int32 [M][N][K/group][4] receives S_c (plain kernel; through
+ *              rcp_gemv_w2a4_grouped_variant with RCP_GEMV_DP4A or RCP_GEMV_MMA_ONLY: the checked
+ *              instantiation of that streaming kernel).
  * Everything else as for rcp_gemv_w2a4 (same workspace, same constraints on M, N, K). Returns
  * RCP_ERR_SHAPE for a bad group size. Never synchronizes.
  */
@@ -225,6 +240,17 @@ int rcp_gemv_w2a4_grouped_variant(int variant, const uint32_t* words, const void
 int rcp_linear_w2a4(const void* x_f16, int M, int K, int had_block, float clip_ratio,
                     const uint32_t* words, const void* lut_f16, int group, int N, void* y_f16,
                     uint8_t* xq, void* scale_f16, void* workspace, void* stream);
+
+/*
+ * rcp_linear_w2a4 with the exact integer sums exported, for parity tests (Section 4.4: the accumulation has
+ * to stay consistent with the grid, and the integer sums S_c are what shows it). Same arguments and results;
+ * S_dbg int32 [M][N][4] (group == 0) or [M][N][K/group][4] receives S_c from the checked instantiation of the
+ * kernel the call would run anyway (the single kernel with the quantizer inside, or the streaming GEMV behind
+ * the stand-alone quantizer; group sizes other than 128 take the plain kernel). S_dbg NULL: rcp_linear_w2a4.
+ */
+int rcp_linear_w2a4_checked(const void* x_f16, int M, int K, int had_block, float clip_ratio,
+                            const uint32_t* words, const void* lut_f16, int group, int N, void* y_f16,
+                            uint8_t* xq, void* scale_f16, void* workspace, int32_t* S_dbg, void* stream);
 
 /* Kernel launches one rcp_linear_w2a4 call makes for a shape (1: the single kernel; otherwise the
  * quantizer plus one GEMV launch per batch of tokens). Host only. Negative status on a bad shape. */

@@ -268,6 +268,21 @@ def gemv_w2a16(words, lut_bits, x_f16_bits):
     return dict(y=y, labsx=labsx, labs=labs)
 
 
+def percode_sums_i8(words, planes):
+    """Per-code sums of signed 8-bit activation planes: planes int8 [C][K] -> S int32 [C][N][4]."""
+    words = _c(words, np.uint32)
+    a = _c(planes, np.int8)
+    N, W = words.shape
+    K = W * 16
+    Cn = a.shape[0]
+    assert a.shape == (Cn, K)
+    S = np.empty((Cn, N, 4), dtype=np.int32)
+    rc = lib().orc_percode_sums_i8(_p(words), _p(a), C.c_int(Cn), C.c_int(N), C.c_int(K), _p(S))
+    if rc:
+        raise ValueError(f"orc_percode_sums_i8 failed: {rc}")
+    return S
+
+
 def split_act16(x_f16_bits):
     """Base-64 fixed-point digits of fp16 activations. Returns dict(digits int8 [M][4][K], unit float64 [M][4])."""
     x = _c(x_f16_bits, np.uint16)

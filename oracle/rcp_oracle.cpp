@@ -30,7 +30,8 @@
 // Weight-only variant: equals the W2A4 oracle when the activations are integers times a power of
 // two; affine grid == plain matrix product; brute force; the fixed-point digits reproduce the
 // activations (exactly for elements within 2^-11 of the token's maximum, to half a unit otherwise)
-// and a hand-written case.
+// and a hand-written case. Per-code sums of 8-bit planes: equal to the W2A4 oracle's S on int4 planes, a
+// pure-Python loop, sum_c S_c == sum_k a_k.
 // fp16 output y: the paper prints no worked numeric GEMV example, so y is pinned only by the
 // mathematical identities above, not by a printed value.
 #include <cstdint>
@@ -570,6 +571,26 @@ int orc_gemv_w2a16(const uint32_t* words, const uint16_t* lut_f16, const uint16_
       }
       y[(size_t)m * N + n] = acc;
       if (labsx) labsx[(size_t)m * N + n] = mag;
+    }
+  }
+  std::free(codes);
+  return 0;
+}
+
+// Per-code sums of signed 8-bit activation planes (Section 4.4: the accumulation respects the grid, one
+// sum per code). For plane j (a row of K signed bytes) and output row n:
+//   S[j][n][c] = sum over k with code[n][k] == c of a[j][k]
+// The weight-only form feeds the GEMV kernels the four digit planes of a token; this is what their
+// integer sums must equal. a int8 [C][K], S int32 [C][N][4]. Returns 0; -1 bad shape.
+int orc_percode_sums_i8(const uint32_t* words, const int8_t* a, int C, int N, int K, int32_t* S) {
+  if (C < 1 || N < 1 || K < 16 || K % 16) return -1;
+  uint8_t* codes = (uint8_t*)std::malloc((size_t)K);
+  for (int n = 0; n < N; n++) {
+    orc_unpack_weights(words + (size_t)n * (K / 16), 1, K, codes);
+    for (int j = 0; j < C; j++) {
+      long long Sc[4] = {0, 0, 0, 0};
+      for (int k = 0; k < K; k++) Sc[codes[k]] += (long long)a[(size_t)j * K + k];
+      for (int c = 0; c < 4; c++) S[((size_t)j * N + n) * 4 + c] = (int32_t)Sc[c];
     }
   }
   std::free(codes);

@@ -64,6 +64,10 @@ def lib():
         L.rcp_gemv_w2a4_static.argtypes = [vp, vp, vp, vp, i, i, i, vp, vp]
         L.rcp_gemv_w2a16.restype = i
         L.rcp_gemv_w2a16.argtypes = [vp, vp, vp, i, i, i, vp, vp, vp, vp, vp]
+        L.rcp_gemv_w2a16_checked.restype = i
+        L.rcp_gemv_w2a16_checked.argtypes = [vp, vp, vp, i, i, i, vp, vp, vp, vp, vp, vp]
+        L.rcp_linear_w2a4_checked.restype = i
+        L.rcp_linear_w2a4_checked.argtypes = [vp, i, i, i, C.c_float, vp, vp, i, i, vp, vp, vp, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -201,9 +205,10 @@ def rcp_gemv_w2a4_grouped(words, lut, xq, scale, group=128, y=None, workspace=No
     return y
 
 
-def rcp_gemv_w2a16(words, lut, x, y=None, digits=None, unit=None, workspace=None):
+def rcp_gemv_w2a16(words, lut, x, y=None, digits=None, unit=None, workspace=None, S_dbg=None):
     """Weight-only form: words int32 [N][K/16], lut fp16 [N][4], x fp16 [M][K] -> y fp16 [M][N].
-    digits int8 [M][4][K] and unit fp32 [M][4] receive the fixed-point form of x the kernels used."""
+    digits int8 [M][4][K] and unit fp32 [M][4] receive the fixed-point form of x the kernels used.
+    S_dbg int32 [4 M][N][4]: the per-code sums of every digit plane (checked instantiation of the kernel)."""
     _dev(words, torch.int32, "words")
     _dev(lut, torch.float16, "lut")
     _dev(x, torch.float16, "x")
@@ -222,8 +227,8 @@ def rcp_gemv_w2a16(words, lut, x, y=None, digits=None, unit=None, workspace=None
         workspace = make_workspace(M, N, K, words.device)
     with _on(words):
         _check("rcp_gemv_w2a16",
-               lib().rcp_gemv_w2a16(_ptr(words), _ptr(lut), _ptr(x), M, N, K, _ptr(y), _ptr(digits), _ptr(unit),
-                                    _ptr(workspace), _stream(words)))
+               lib().rcp_gemv_w2a16_checked(_ptr(words), _ptr(lut), _ptr(x), M, N, K, _ptr(y), _ptr(digits), _ptr(unit),
+                                            _ptr(workspace), _ptr(S_dbg), _stream(words)))
     return y
 
 
@@ -253,10 +258,13 @@ def rcp_gemv_w2a4_static(words, lut, xq, scale, y=None):
     return y
 
 
-def rcp_linear_w2a4(x, had_block, clip_ratio, words, lut, group=0, y=None, xq=None, scale=None, workspace=None):
+def rcp_linear_w2a4(x, had_block, clip_ratio, words, lut, group=0, y=None, xq=None, scale=None, workspace=None,
+                    S_dbg=None):
     """x fp16 [M][K] -> y fp16 [M][N]: activation quantization and LUT GEMV in one call (one kernel for
-    one or two tokens). lut fp16 [N][4] with group=0, [N][K/group][4] otherwise. xq / scale: optional
-    outputs on the one-kernel path, required staging otherwise (pass them to be safe)."""
+    one token of 4096 or 8192 under one rotation block). lut fp16 [N][4] with group=0, [N][K/group][4]
+    otherwise. xq / scale: optional outputs on the one-kernel path, required staging otherwise (pass them to
+    be safe). S_dbg int32 [M][N][4] ([M][N][K/group][4]): the integer sums, from the checked instantiation
+    of the kernel that runs anyway."""
     _dev(x, torch.float16, "x")
     _dev(words, torch.int32, "words")
     _dev(lut, torch.float16, "lut")
@@ -272,8 +280,9 @@ def rcp_linear_w2a4(x, had_block, clip_ratio, words, lut, group=0, y=None, xq=No
         workspace = make_workspace(M, N, K, words.device)
     with _on(words):
         _check("rcp_linear_w2a4",
-               lib().rcp_linear_w2a4(_ptr(x), M, K, int(had_block), float(clip_ratio), _ptr(words), _ptr(lut), group, N,
-                                     _ptr(y), _ptr(xq), _ptr(scale), _ptr(workspace), _stream(words)))
+               lib().rcp_linear_w2a4_checked(_ptr(x), M, K, int(had_block), float(clip_ratio), _ptr(words), _ptr(lut),
+                                             group, N, _ptr(y), _ptr(xq), _ptr(scale), _ptr(workspace), _ptr(S_dbg),
+                                             _stream(words)))
     return y
 
 

@@ -76,6 +76,8 @@ struct GemvParams {
                          // memory at off_qbuf); CTA 0 also stores them to xq_out ([4][K] bytes) and the units here
   __half* y;
   int32_t* status;      // optional: receives a code when a bounded wait gives up
+  int32_t* S_out;       // SDBG instantiations only: the exact per-code sums, [M][N][4] (group-wise: [M][N][ngrp][4];
+                        // digit columns: one "token" per column)
   int M, N, K;
   int ngrp;             // group-wise grid: groups of 128 weights per row (K / 128), lut is [N][ngrp]; else 0
   int nchunk;           // 128-byte chunks per row, ceil(K / 512); with nsplit > 1: per part of K
@@ -204,7 +206,10 @@ __device__ __forceinline__ void dp4a_s8s8(int& d, uint32_t a, uint32_t b) {
 //       fp16 tokens, one signed byte per element (p.xq is [4 tokens][K] bytes, p.unit their fp32 units, p.M
 //       the number of digit columns); the digits of a token are combined in fp32 when its rows are finished.
 // SPLIT K in parts (see below): the eight-column tensor-core kernels of the per-row grid, when asked to.
-template <int MODE, int MTOK, bool GRP, bool FQ = false, bool A16 = false, bool SPLIT = false>
+// SDBG  checked instantiation: the same kernel also stores the integer sums S_0..S_3 it finishes its rows
+//       from (p.S_out), so that a test can compare them with a reference bit for bit. The production
+//       instantiations (SDBG false) contain none of this.
+template <int MODE, int MTOK, bool GRP, bool FQ = false, bool A16 = false, bool SPLIT = false, bool SDBG = false>
 __global__ void __launch_bounds__(kGThreads, 1)
 gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -742,7 +747,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     }
   };
   // CUDA-core mode, after a chunk: this lane's sums are those of group t of the chunk
-  auto flush_grp_dp4a = [&](int ch, const uint2 (&lg)[NLG][2]) {
+  auto flush_grp_dp4a = [&](int ch, const uint2 (&lg)[NLG][2], int row_first) {
     if constexpr (GRP && MODE == kModeDp4a) {
       const int gi = ch * 4 + t;
 #pragma unroll
@@ -755,13 +760,19 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
           const int T0 = s_T0c[tok * ng4 + gi];
           const int S1 = a1 - a3, S2 = a2 - a3;
           yacc[tok * 2 + rr] += lut_dot(lg[0][rr], T0 - S1 - S2 - a3, S1, S2, a3);
+          if constexpr (SDBG) {
+            const int row = row_first + g + 8 * rr;
+            if (row < p.N && gi < p.ngrp)
+              *reinterpret_cast<int4*>(p.S_out + (((size_t)tok * p.N + row) * p.ngrp + gi) * 4) =
+                  make_int4(T0 - S1 - S2 - a3, S1, S2, a3);
+          }
         }
       zero_acc();
     }
   };
   // Tensor-core mode: one chunk = four groups, each read by the whole quad, finished after its
   // twelve MMAs.
-  auto compute_chunk_grp_mma = [&](uint32_t a_grp, uint32_t b_chunk, int ch, const uint2 (&lg)[NLG][2]) {
+  auto compute_chunk_grp_mma = [&](uint32_t a_grp, uint32_t b_chunk, int ch, const uint2 (&lg)[NLG][2], int row_first) {
     if constexpr (kRelabel) {
       const uint32_t a_row = a_grp + (uint32_t)(grow * 128 + ((t & 1) << 3));
       const uint32_t b_grp = base + (uint32_t)p.off_bs + b_chunk + bM_lane;
@@ -811,6 +822,18 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
           const float2 l01 = __half22float2(*reinterpret_cast<const __half2*>(&lgj[r >> 1].x));
           const float2 l23 = __half22float2(*reinterpret_cast<const __half2*>(&lgj[r >> 1].y));
           yacc[r] = fmaf(l01.x, S0, fmaf(l01.y, S1, fmaf(l23.x, S2, fmaf(l23.y, F3, yacc[r]))));
+          if constexpr (SDBG) {
+            // the same sums as integers: the accumulators hold 4 T1, 8 T2, 8 T3 (and 16 times that)
+            const int I1 = (accM[0][0][r] + (accM[0][1][r] >> 4)) >> 2;
+            const int I2 = (accM[1][0][r] + (accM[1][1][r] >> 4)) >> 3;
+            const int I3 = (accM[2][0][r] + (accM[2][1][r] >> 4)) >> 3;
+            const int tok = 2 * t + (r & 1), row = row_first + grow + 8 * (r >> 1);
+            if (tok < M && row < p.N && gi < p.ngrp) {
+              const int I0 = __float2int_rn(0.125f * ((r & 1) ? t0.y : t0.x)) - (I1 - I3) - (I2 - I3) - I3;
+              *reinterpret_cast<int4*>(p.S_out + (((size_t)tok * p.N + row) * p.ngrp + gi) * 4) =
+                  make_int4(I0, I1 - I3, I2 - I3, I3);
+            }
+          }
         }
       }
     }
@@ -925,6 +948,10 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
             const int S3 = T3[e + h], S1 = T1[e + h] - T3[e + h], S2 = T2[e + h] - T3[e + h];
             const int S0 = (kTwoTiles ? s_T0tot[c] : T0v[e + h]) - S1 - S2 - S3;
             const float d = lut_sum(lut_g[err[e]], S0, S1, S2, S3);
+            if constexpr (SDBG) {
+              const int row_s = row_first + g + 8 * err[e];
+              if (row_s < p.N) *reinterpret_cast<int4*>(p.S_out + ((size_t)c * p.N + row_s) * 4) = make_int4(S0, S1, S2, S3);
+            }
             v = h ? __fmaf_rn(s_scale[c], d, v) : __fmul_rn(s_scale[c], d);
           }
         }
@@ -940,6 +967,8 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
           const int S3 = T3[e], S1 = T1[e] - T3[e], S2 = T2[e] - T3[e];
           const int S0 = (kTwoTiles ? s_T0tot[etok[e]] : T0v[e]) - S1 - S2 - S3;
           p.y[(size_t)etok[e] * p.N + row] = lut_finish(s_scale[etok[e]], lut_g[err[e]], S0, S1, S2, S3);
+          if constexpr (SDBG)
+            *reinterpret_cast<int4*>(p.S_out + ((size_t)etok[e] * p.N + row) * 4) = make_int4(S0, S1, S2, S3);
         }
       }
     }
@@ -996,10 +1025,10 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
           if (active && ch < p.nchunk) {
             const uint32_t a_grp = base + (uint32_t)slot * kStageBytes + a_off;
             if constexpr (kRelabel) {
-              compute_chunk_grp_mma(a_grp, b_chunk, ch, lg_cur);
+              compute_chunk_grp_mma(a_grp, b_chunk, ch, lg_cur, row_first);
             } else {
               compute_chunk(a_grp, b_chunk);
-              flush_grp_dp4a(ch, lg_cur);
+              flush_grp_dp4a(ch, lg_cur, row_first);
             }
           }
           __syncwarp();

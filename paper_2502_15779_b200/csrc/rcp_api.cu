@@ -215,26 +215,44 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
+constexpr int kMaxDevices = 64;
+
+// SMs of the current device (remembered per device; 148 if the query fails)
 int sm_count() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-      n = 148;
-  }
-  return n;
+  static std::mutex mu;
+  static int n[kMaxDevices] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 148;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!n[dev] && cudaDeviceGetAttribute(&n[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n[dev] = 148;
+  return n[dev];
 }
 
-template <int MODE, int MTOK, bool GRP = false, bool FQ = false, bool A16 = false, bool SPLIT = false>
-int launch_stream_t(const rcp::GemvMaps& maps, const rcp::GemvParams& gp, const StreamPlan& pl, cudaStream_t st) {
-  static bool attr_set = false;
-  auto kern = rcp::gemv_stream_kernel<MODE, MTOK, GRP, FQ, A16, SPLIT>;
-  if (!attr_set) {
-    RCP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax));
-    attr_set = true;
+template <int MODE, int MTOK, bool GRP, bool FQ, bool A16, bool SPLIT, bool SDBG>
+int launch_stream_s(const rcp::GemvMaps& maps, const rcp::GemvParams& gp, const StreamPlan& pl, cudaStream_t st) {
+  // cudaFuncAttributeMaxDynamicSharedMemorySize belongs to the (kernel, device) pair: set once per device
+  static std::mutex mu;
+  static bool attr_set[kMaxDevices] = {};
+  auto kern = rcp::gemv_stream_kernel<MODE, MTOK, GRP, FQ, A16, SPLIT, SDBG>;
+  int dev = 0;
+  RCP_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return RCP_ERR_LIMIT;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (!attr_set[dev]) {
+      RCP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax));
+      attr_set[dev] = true;
+    }
   }
   RCP_CUDA(launch_overlapped(kern, dim3(pl.grid), dim3(rcp::kGThreads), pl.smem, st, maps, gp));
   return RCP_OK;
+}
+
+// gp.S_out set: the checked instantiation of the same kernel, which also stores its integer sums.
+template <int MODE, int MTOK, bool GRP = false, bool FQ = false, bool A16 = false, bool SPLIT = false>
+int launch_stream_t(const rcp::GemvMaps& maps, const rcp::GemvParams& gp, const StreamPlan& pl, cudaStream_t st) {
+  if (gp.S_out) return launch_stream_s<MODE, MTOK, GRP, FQ, A16, SPLIT, true>(maps, gp, pl, st);
+  return launch_stream_s<MODE, MTOK, GRP, FQ, A16, SPLIT, false>(maps, gp, pl, st);
 }
 
 // One launch: M tokens (their expanded activations fit in shared memory). grouped: lut_f16 is
@@ -263,7 +281,7 @@ bool fused_ok(int M, int K, int B) { return M == 1 && B == K && (K == 4096 || K 
 int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const uint8_t* xq, const void* scale_f16,
                   int M, int N, int K, void* y_f16, void* workspace, cudaStream_t st, bool grouped = false,
                   const FusedAct* fa = nullptr, const float* unit = nullptr, int nsplit = 1,
-                  const SplitAct* sa = nullptr) {
+                  const SplitAct* sa = nullptr, int32_t* S_out = nullptr) {
   if (nsplit > 1 && (mode != rcp::kModeMma || grouped || fa || M > 8)) return RCP_ERR_VARIANT;
   if (sa && (mode != rcp::kModeMma || grouped || fa || unit || nsplit > 1 || M != 4 || K > 16384)) return RCP_ERR_VARIANT;
   // unit: weight-only form; xq then holds M digit columns of K signed bytes (four per token), scale_f16 is unused
@@ -317,6 +335,7 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   gp.unit = unit;
   gp.y = static_cast<__half*>(y_f16);
   gp.status = static_cast<int32_t*>(workspace);
+  gp.S_out = S_out;
   gp.M = M; gp.N = N; gp.K = K;
   gp.ngrp = grouped ? K / 128 : 0;
   gp.nchunk = pl.nchunk;
@@ -373,7 +392,7 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
 // All M tokens: as many launches as it takes for the expanded activations to fit (`cap` tokens at most each).
 int launch_stream_passes(int mode, int cap, const uint32_t* words, const void* lut_f16, const uint8_t* xq,
                          const void* scale_f16, int M, int N, int K, void* y_f16, void* workspace, cudaStream_t st,
-                         bool grouped = false) {
+                         bool grouped = false, int32_t* S_out = nullptr) {
   int nsplit = 1;
   const int mp = (grouped || cap < 8) ? tokens_per_pass(M, K, cap) : tokens_and_parts(M, N, K, cap, sm_count(), &nsplit);
   for (int m0 = 0; m0 < M; m0 += mp) {
@@ -383,7 +402,8 @@ int launch_stream_passes(int mode, int cap, const uint32_t* words, const void* l
     const int rc = launch_stream(md, words, lut_f16, xq + (size_t)m0 * (K / 2),
                                  static_cast<const __half*>(scale_f16) + m0, mm, N, K,
                                  static_cast<__half*>(y_f16) + (size_t)m0 * N, workspace, st, grouped, nullptr, nullptr,
-                                 md == rcp::kModeMma ? nsplit : 1);
+                                 md == rcp::kModeMma ? nsplit : 1, nullptr,
+                                 S_out ? S_out + (size_t)m0 * N * 4 * (grouped ? K / 128 : 1) : nullptr);
     if (rc != RCP_OK) return rc;
   }
   return RCP_OK;
@@ -397,7 +417,6 @@ static __device__ __align__(256) unsigned char g_static_scratch[RCP_STATIC_SCRAT
 // stands for the symbol; the address a kernel can use comes from cudaGetSymbolAddress, asked once
 // per device with that device current and remembered afterwards.
 int static_scratch_address(void** out) {
-  constexpr int kMaxDevices = 64;
   static std::mutex mu;
   static void* addr[kMaxDevices] = {};
   int dev = 0;
@@ -591,7 +610,9 @@ int rcp_gemv_w2a4_variant(int variant, const uint32_t* words, const void* lut_f1
     return RCP_ERR_ALIGN;
   if (reinterpret_cast<uintptr_t>(workspace) & 3u) return RCP_ERR_ALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (S_dbg) variant = RCP_GEMV_SIMPLE;
+  // S_dbg without a variant of the caller's choice: the plain kernel. With one: the checked instantiation of
+  // that streaming kernel, which stores the sums it finishes its rows from.
+  if (S_dbg && variant == RCP_GEMV_AUTO) variant = RCP_GEMV_SIMPLE;
   // measured on B200: one token runs fastest on the CUDA cores alone, more tokens on the tensor cores
   if (variant == RCP_GEMV_AUTO) variant = (M == 1) ? RCP_GEMV_DP4A : RCP_GEMV_MMA_ONLY;
   switch (variant) {
@@ -606,12 +627,14 @@ int rcp_gemv_w2a4_variant(int variant, const uint32_t* words, const void* lut_f1
     case RCP_GEMV_MMA:
       // tensor-core path; for one or two tokens the b0*b1 plane goes to dp4a (FMA pipe) instead
       return launch_stream_passes(M <= 2 ? rcp::kModeHybrid : rcp::kModeMma, 16, words, lut_f16, xq, scale_f16, M, N, K,
-                                  y_f16, workspace, st);
+                                  y_f16, workspace, st, false, S_dbg);
     case RCP_GEMV_MMA_ONLY:
-      return launch_stream_passes(rcp::kModeMma, 16, words, lut_f16, xq, scale_f16, M, N, K, y_f16, workspace, st);
+      return launch_stream_passes(rcp::kModeMma, 16, words, lut_f16, xq, scale_f16, M, N, K, y_f16, workspace, st, false,
+                                  S_dbg);
     case RCP_GEMV_DP4A:
       // CUDA-core path: two tokens per launch
-      return launch_stream_passes(rcp::kModeDp4a, 2, words, lut_f16, xq, scale_f16, M, N, K, y_f16, workspace, st);
+      return launch_stream_passes(rcp::kModeDp4a, 2, words, lut_f16, xq, scale_f16, M, N, K, y_f16, workspace, st, false,
+                                  S_dbg);
     default:
       return RCP_ERR_VARIANT;
   }
@@ -625,9 +648,10 @@ int rcp_gemv_w2a4(const uint32_t* words, const void* lut_f16, const uint8_t* xq,
                                S_dbg, stream);
 }
 
-int rcp_gemv_w2a16(const uint32_t* words, const void* lut_f16, const void* x_f16, int M, int N, int K, void* y_f16,
-                   int8_t* digits, float* unit, void* workspace, void* stream) {
+int rcp_gemv_w2a16_checked(const uint32_t* words, const void* lut_f16, const void* x_f16, int M, int N, int K,
+                           void* y_f16, int8_t* digits, float* unit, void* workspace, int32_t* S_dbg, void* stream) {
   if (!words || !lut_f16 || !x_f16 || !y_f16 || !digits || !unit) return RCP_ERR_NULL;
+  if (!aligned16(S_dbg)) return RCP_ERR_ALIGN;
   if (M < 1 || M > rcp::kMaxTokens || N < 1 || !k_ok(K)) return RCP_ERR_SHAPE;
   if (!aligned16(words) || !aligned16(x_f16) || !aligned16(digits) || (reinterpret_cast<uintptr_t>(lut_f16) & 7u) ||
       (reinterpret_cast<uintptr_t>(y_f16) & 1u) || (reinterpret_cast<uintptr_t>(unit) & 3u) ||
@@ -646,7 +670,7 @@ int rcp_gemv_w2a16(const uint32_t* words, const void* lut_f16, const void* x_f16
       make_plan(cols, N, K, sm_count(), false, (size_t)cols * K, 1).stages >= 3) {
     const SplitAct sa{x_f16, digits, unit};
     return launch_stream(rcp::kModeMma, words, lut_f16, nullptr, nullptr, cols, N, K, y_f16, workspace, st, false,
-                         nullptr, nullptr, 1, &sa);
+                         nullptr, nullptr, 1, &sa, S_dbg);
   }
   RCP_CUDA(launch_overlapped(rcp::split_act16_kernel, dim3(M), dim3(rcp::kSplitThreads), 0, st,
                              static_cast<const __half*>(x_f16), K, digits, unit));
@@ -654,10 +678,15 @@ int rcp_gemv_w2a16(const uint32_t* words, const void* lut_f16, const void* x_f16
     const int cc = std::min(cp, cols - c0);
     const int rc = launch_stream(rcp::kModeMma, words, lut_f16, reinterpret_cast<const uint8_t*>(digits) + (size_t)c0 * K,
                                  nullptr, cc, N, K, static_cast<__half*>(y_f16) + (size_t)(c0 / 4) * N, workspace, st,
-                                 false, nullptr, unit + c0, nsplit);
+                                 false, nullptr, unit + c0, nsplit, nullptr, S_dbg ? S_dbg + (size_t)c0 * N * 4 : nullptr);
     if (rc != RCP_OK) return rc;
   }
   return RCP_OK;
+}
+
+int rcp_gemv_w2a16(const uint32_t* words, const void* lut_f16, const void* x_f16, int M, int N, int K, void* y_f16,
+                   int8_t* digits, float* unit, void* workspace, void* stream) {
+  return rcp_gemv_w2a16_checked(words, lut_f16, x_f16, M, N, K, y_f16, digits, unit, workspace, nullptr, stream);
 }
 
 int rcp_gemv_w2a4_grouped_variant(int variant, const uint32_t* words, const void* lut_f16, int group,
@@ -673,7 +702,7 @@ int rcp_gemv_w2a4_grouped_variant(int variant, const uint32_t* words, const void
   if (reinterpret_cast<uintptr_t>(workspace) & 3u) return RCP_ERR_ALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // the streaming kernels are built for the paper's group size; other sizes take the plain kernel
-  if (S_dbg || (variant == RCP_GEMV_AUTO && group != 128)) variant = RCP_GEMV_SIMPLE;
+  if (variant == RCP_GEMV_AUTO && (S_dbg || group != 128)) variant = RCP_GEMV_SIMPLE;
   if (variant == RCP_GEMV_AUTO) variant = (M <= 2) ? RCP_GEMV_DP4A : RCP_GEMV_MMA_ONLY;
   switch (variant) {
     case RCP_GEMV_SIMPLE: {
@@ -686,10 +715,12 @@ int rcp_gemv_w2a4_grouped_variant(int variant, const uint32_t* words, const void
     }
     case RCP_GEMV_MMA_ONLY:
       if (group != 128) return RCP_ERR_VARIANT;
-      return launch_stream_passes(rcp::kModeMma, 8, words, lut_f16, xq, scale_f16, M, N, K, y_f16, workspace, st, true);
+      return launch_stream_passes(rcp::kModeMma, 8, words, lut_f16, xq, scale_f16, M, N, K, y_f16, workspace, st, true,
+                                  S_dbg);
     case RCP_GEMV_DP4A:
       if (group != 128) return RCP_ERR_VARIANT;
-      return launch_stream_passes(rcp::kModeDp4a, 2, words, lut_f16, xq, scale_f16, M, N, K, y_f16, workspace, st, true);
+      return launch_stream_passes(rcp::kModeDp4a, 2, words, lut_f16, xq, scale_f16, M, N, K, y_f16, workspace, st, true,
+                                  S_dbg);
     default:
       return RCP_ERR_VARIANT;
   }
@@ -706,7 +737,13 @@ int rcp_gemv_w2a4_grouped(const uint32_t* words, const void* lut_f16, int group,
 
 int rcp_gemv_w2a4_static(const uint32_t* words, const void* lut_f16, const uint8_t* xq, const void* scale_f16,
                          int M, int N, int K, void* y_f16, void* stream) {
-  const size_t need = rcp_gemv_workspace_bytes(M, N, K);   // 0 on a bad shape: reported by the call below
+  // the same checks as rcp_gemv_w2a4, before anything is put on the stream
+  if (!words || !lut_f16 || !xq || !scale_f16 || !y_f16) return RCP_ERR_NULL;
+  if (M < 1 || M > rcp::kMaxTokens || N < 1 || !k_ok(K)) return RCP_ERR_SHAPE;
+  if (!aligned16(words) || !aligned16(xq) || (reinterpret_cast<uintptr_t>(lut_f16) & 7u) ||
+      (reinterpret_cast<uintptr_t>(y_f16) & 1u) || (reinterpret_cast<uintptr_t>(scale_f16) & 1u))
+    return RCP_ERR_ALIGN;
+  const size_t need = rcp_gemv_workspace_bytes(M, N, K);
   if (need > RCP_STATIC_SCRATCH_BYTES) return RCP_ERR_LIMIT;
   void* scratch = nullptr;
   const int rc = static_scratch_address(&scratch);
@@ -728,10 +765,11 @@ int rcp_linear_w2a4_launches(int M, int N, int K, int had_block, int group) {
   return 1 + (M + mp - 1) / mp;
 }
 
-int rcp_linear_w2a4(const void* x_f16, int M, int K, int had_block, float clip_ratio, const uint32_t* words,
-                    const void* lut_f16, int group, int N, void* y_f16, uint8_t* xq, void* scale_f16, void* workspace,
-                    void* stream) {
+int rcp_linear_w2a4_checked(const void* x_f16, int M, int K, int had_block, float clip_ratio, const uint32_t* words,
+                            const void* lut_f16, int group, int N, void* y_f16, uint8_t* xq, void* scale_f16,
+                            void* workspace, int32_t* S_dbg, void* stream) {
   if (!x_f16 || !words || !lut_f16 || !y_f16) return RCP_ERR_NULL;
+  if (!aligned16(S_dbg)) return RCP_ERR_ALIGN;
   if (M < 1 || M > rcp::kMaxTokens || N < 1 || !k_ok(K)) return RCP_ERR_SHAPE;
   const int B = had_block <= 1 ? 1 : had_block;
   if (B > 8192 || (B & (B - 1)) || K % B) return RCP_ERR_SHAPE;
@@ -745,14 +783,25 @@ int rcp_linear_w2a4(const void* x_f16, int M, int K, int had_block, float clip_r
   if (fused_ok(M, K, B) && (group == 0 || group == 128)) {
     const FusedAct fa{x_f16, B, clip_ratio, xq, scale_f16};
     return launch_stream(rcp::kModeDp4a, words, lut_f16, nullptr, nullptr, M, N, K, y_f16, workspace, st, group == 128,
-                         &fa);
+                         &fa, nullptr, 1, nullptr, S_dbg);
   }
   // otherwise the two kernels one after the other; they need the staging buffers
   if (!xq || !scale_f16) return RCP_ERR_NULL;
   int rc = rcp_quantize_act(x_f16, M, K, had_block, clip_ratio, xq, scale_f16, stream);
   if (rc != RCP_OK) return rc;
-  if (group == 0) return rcp_gemv_w2a4(words, lut_f16, xq, scale_f16, M, N, K, y_f16, workspace, nullptr, stream);
-  return rcp_gemv_w2a4_grouped(words, lut_f16, group, xq, scale_f16, M, N, K, y_f16, workspace, nullptr, stream);
+  // with S_dbg: the streaming kernel AUTO would pick, in its checked instantiation
+  if (group == 0)
+    return rcp_gemv_w2a4_variant(S_dbg ? (M == 1 ? RCP_GEMV_DP4A : RCP_GEMV_MMA_ONLY) : RCP_GEMV_AUTO, words, lut_f16, xq,
+                                 scale_f16, M, N, K, y_f16, workspace, S_dbg, stream);
+  return rcp_gemv_w2a4_grouped_variant(S_dbg && group == 128 ? (M <= 2 ? RCP_GEMV_DP4A : RCP_GEMV_MMA_ONLY) : RCP_GEMV_AUTO,
+                                       words, lut_f16, group, xq, scale_f16, M, N, K, y_f16, workspace, S_dbg, stream);
+}
+
+int rcp_linear_w2a4(const void* x_f16, int M, int K, int had_block, float clip_ratio, const uint32_t* words,
+                    const void* lut_f16, int group, int N, void* y_f16, uint8_t* xq, void* scale_f16, void* workspace,
+                    void* stream) {
+  return rcp_linear_w2a4_checked(x_f16, M, K, had_block, clip_ratio, words, lut_f16, group, N, y_f16, xq, scale_f16,
+                                 workspace, nullptr, stream);
 }
 
 int rcp_linear_w2a4_host(const void* x_host_f16, int M, int K, int had_block, float clip_ratio,

@@ -38,9 +38,16 @@ def _check(N, K, G, B, M, kind, variant, seed, rows=None, with_S=True):
     ref = oracle.gemv_w2a4_grouped(w_ref, np.ascontiguousarray(f16_bits(lut)[sel]), qa["xq"], qa["scale"], G)
     outs = [y]
     if with_S:
-        S = torch.full((M, N, K // G, 4), -12345, dtype=torch.int32, device=DEV)
-        outs.append(rcp.rcp_gemv_w2a4_grouped(words, lut, xq, scale, group=G, workspace=ws, S_dbg=S))
-        assert np.array_equal(S.cpu().numpy()[:, sel], ref["S"])
+        # the per-group sums from the checked instantiation of the kernel `variant` names; with auto, from the
+        # plain kernel and from the streaming kernel auto dispatches to
+        todo = [variant]
+        if variant == "auto" and G == 128:
+            todo.append("dp4a" if M <= 2 else "mma_only")
+        for v in todo:
+            S = torch.full((M, N, K // G, 4), -12345, dtype=torch.int32, device=DEV)
+            outs.append(rcp.rcp_gemv_w2a4_grouped(words, lut, xq, scale, group=G, workspace=ws, S_dbg=S, variant=v))
+            assert np.array_equal(S.cpu().numpy()[:, sel], ref["S"]), f"S_c of variant {v}"
+            del S
     for out in outs:
         got = out.float().cpu().numpy().astype(np.float64)[:, sel]
         err = np.abs(got - ref["y"])
@@ -129,4 +136,4 @@ def test_grouped_gemv_full_size_configs_sampled_rows(ci, N, K, B, M):
     rng = np.random.default_rng(N + K + M)
     rows = np.unique(np.concatenate([np.arange(min(N, 32)), np.arange(max(0, N - 32), N),
                                      rng.integers(0, N, size=min(N, 128))]))
-    _check(N, K, 128, B, M, "uniform", "auto", seed=2000 + ci, rows=rows, with_S=False)
+    _check(N, K, 128, B, M, "uniform", "auto", seed=2000 + ci, rows=rows)

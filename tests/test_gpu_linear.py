@@ -42,6 +42,11 @@ def _check(N, K, B, M, group, clip, seed, kind="uniform", rows=None, staging=Tru
     assert np.all(np.isfinite(got))
     err = np.abs(got - ref["y"])
     assert np.all(err <= ref["tol"]), f"max err/tol {np.max(err / ref['tol'])}"
+    # the integer sums of the kernel this call runs (checked instantiation), bit for bit
+    S = torch.full((M, N, K // group, 4) if group else (M, N, 4), -12345, dtype=torch.int32, device=DEV)
+    y3 = rcp.rcp_linear_w2a4(x, B, clip, words, lut, group=group, xq=xq, scale=scale, workspace=ws, S_dbg=S)
+    assert np.array_equal(S.cpu().numpy()[:, sel], ref["S"])
+    assert torch.equal(y.view(torch.int16), y3.view(torch.int16))
 
 
 CASES = [

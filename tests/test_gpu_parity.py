@@ -109,10 +109,16 @@ def _check_gemv(N, K, B, M, kind, variant, seed, rows=None):
     w_ref = oracle.pack_weights(codes_sel)
     assert np.array_equal(words_np(words)[sel], w_ref)
     ref = oracle.gemv_w2a4(w_ref, f16_bits(lut)[sel], qa["xq"], qa["scale"])
+    # S comes from the checked instantiation of the very kernel `variant` names (auto: the plain kernel)
     assert np.array_equal(S.cpu().numpy()[:, sel, :], ref["S"])
-    # y_dbg comes from the kernel that exported the S_c just checked. Every variant finishes its own integer
-    # sums with the same fp32 steps, so equal bits here mean the variant's S_c are the exact ones as well.
-    assert torch.equal(y.view(torch.int16), y_dbg.view(torch.int16)), "variant's sums differ from the exported S_c"
+    assert torch.equal(y.view(torch.int16), y_dbg.view(torch.int16)), "checked and production instantiation differ"
+    if variant == "auto":
+        # ... and from the streaming kernel that auto dispatches to for this token count
+        hot = "dp4a" if M == 1 else "mma_only"
+        S_hot = torch.full((M, N, 4), -12345, dtype=torch.int32, device=DEV)
+        y_hot = rcp.rcp_gemv_w2a4(words, lut, xq, scale, workspace=ws, S_dbg=S_hot, variant=hot)
+        assert np.array_equal(S_hot.cpu().numpy()[:, sel, :], ref["S"]), f"S_c of the {hot} kernel"
+        assert torch.equal(y.view(torch.int16), y_hot.view(torch.int16))
     for out in (y, y_dbg):
         got = out.float().cpu().numpy().astype(np.float64)[:, sel]
         err = np.abs(got - ref["y"])

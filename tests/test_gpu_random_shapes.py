@@ -67,6 +67,18 @@ def test_random_shape(N, K, M, variant, grouped, i):
         got = out.float().cpu().numpy().astype(np.float64)[:, rows]
         assert np.all(np.isfinite(got))
         assert np.all(np.abs(got - ref["y"]) <= ref["tol"])
+    # the integer sums of the kernel the variant names (auto: the plain kernel) and of the linear call's kernel
+    shape = (M, N, K // 128, 4) if grouped else (M, N, 4)
+    S1 = torch.full(shape, -12345, dtype=torch.int32, device=DEV)
+    S2 = torch.full(shape, -12345, dtype=torch.int32, device=DEV)
+    if grouped:
+        rcp.rcp_gemv_w2a4_grouped(words, lut, xq, scale, group=128, workspace=ws, variant=variant, S_dbg=S1)
+    else:
+        rcp.rcp_gemv_w2a4(words, lut, xq, scale, workspace=ws, variant=variant, S_dbg=S1)
+    rcp.rcp_linear_w2a4(x, B, 1.0, words, lut, group=128 if grouped else 0, xq=torch.empty_like(xq),
+                        scale=torch.empty_like(scale), workspace=ws, S_dbg=S2)
+    assert np.array_equal(S1.cpu().numpy()[:, rows], ref["S"])
+    assert np.array_equal(S2.cpu().numpy()[:, rows], ref["S"])
 
 
 @pytest.mark.parametrize("N,K,M,variant,grouped,i", [c for c in _cases(48, 20250215) if not c.values[4]][:20])
@@ -94,6 +106,10 @@ def test_random_shape_weight_only(N, K, M, variant, grouped, i):
            + 2.0 ** -11 * np.abs(ref["y"]) + 2.0 ** -24)
     got = y.float().cpu().numpy().astype(np.float64)[:, rows]
     assert np.all(np.isfinite(got)) and np.all(np.abs(got - ref["y"]) <= tol)
+    S = torch.full((4 * M, N, 4), -12345, dtype=torch.int32, device=DEV)
+    rcp.rcp_gemv_w2a16(words, lut, x, workspace=ws, S_dbg=S)
+    w_rows = oracle.pack_weights(codes.cpu().numpy()[rows])
+    assert np.array_equal(S.cpu().numpy()[:, rows], oracle.percode_sums_i8(w_rows, sp["digits"].reshape(4 * M, K)))
 
 
 @pytest.mark.parametrize("N,K,M,grouped", [(70, 65536, 1, False), (40, 65536, 8, False), (33, 65536, 2, True),

@@ -45,6 +45,11 @@ def _check(N, K, M, seed, kind="rotated_laplace", x=None, rows=None):
     err = np.abs(got - ref["y"])
     assert np.all(np.isfinite(got))
     assert np.all(err <= tol), f"max err/tol {np.max(err / tol)}"
+    # the per-code sums of every digit plane, from the checked instantiation of the same kernels
+    S = torch.full((4 * M, N, 4), -12345, dtype=torch.int32, device=DEV)
+    y3 = rcp.rcp_gemv_w2a16(words, lut, x, workspace=ws, S_dbg=S)
+    assert np.array_equal(S.cpu().numpy()[:, sel], oracle.percode_sums_i8(w_ref, sp["digits"].reshape(4 * M, K)))
+    assert torch.equal(y.view(torch.int16), y3.view(torch.int16))
     return err, tol, ref
 
 

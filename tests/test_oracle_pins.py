@@ -678,3 +678,33 @@ def test_split16_digits_reproduce_the_activations():
     assert not dg[5].any()
     with pytest.raises(ValueError):
         oracle.split_act16(np.array([[0x7C00, 0]], dtype=np.uint16))
+
+
+# ----------------------------------------------------------------------------- per-code sums of 8-bit planes
+def test_percode_sums_i8_brute_force_and_invariants():
+    rng = np.random.default_rng(41)
+    N, K, C = 7, 64, 3
+    codes = rng.integers(0, 4, size=(N, K), dtype=np.uint8)
+    planes = rng.integers(-128, 128, size=(C, K)).astype(np.int8)
+    S = oracle.percode_sums_i8(oracle.pack_weights(codes), planes)
+    ref = np.zeros((C, N, 4), dtype=np.int64)
+    for j in range(C):          # the definition as a plain loop
+        for n in range(N):
+            for k in range(K):
+                ref[j, n, int(codes[n, k])] += int(planes[j, k])
+    assert np.array_equal(S, ref)
+    # the four sums of a row add up to the plane's total, whatever the codes
+    assert np.array_equal(S.sum(axis=2), np.repeat(planes.astype(np.int64).sum(axis=1)[:, None], N, axis=1))
+    # a planted mistake (codes read in reversed order) is caught
+    bad = oracle.percode_sums_i8(oracle.pack_weights(codes[:, ::-1].copy()), planes)
+    assert not np.array_equal(bad, ref)
+
+
+def test_percode_sums_i8_equal_the_w2a4_sums_on_int4_planes():
+    N, K, M = 33, 512, 4
+    codes, lut = synth.make_layer(N, K, 128, "uniform", 3)
+    x = synth.make_activations(M, K, 3)
+    qa = oracle.quantize_act(f16_bits(x), 128, 1.0)
+    words = oracle.pack_weights(codes.numpy())
+    ref = oracle.gemv_w2a4(words, f16_bits(lut), qa["xq"], qa["scale"])
+    assert np.array_equal(oracle.percode_sums_i8(words, oracle.unpack_act(qa["xq"]).astype(np.int8)), ref["S"])
