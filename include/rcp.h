@@ -35,7 +35,7 @@ enum {
   RCP_ERR_SHAPE = -2,     /* K % 64 != 0, N < 1, M outside 1..16, bad had_block, ... */
   RCP_ERR_ALIGN = -3,     /* a pointer is not 16-byte aligned */
   RCP_ERR_CODE = -4,      /* rcp_pack_weights met a code above 3 */
-  RCP_ERR_WORKSPACE = -5, /* workspace missing */
+  RCP_ERR_WORKSPACE = -5, /* workspace missing (the streaming kernels report through it) */
   RCP_ERR_CUDA = -6,      /* a CUDA call failed; see rcp_last_cuda_error() */
   RCP_ERR_VARIANT = -7,   /* unknown kernel variant, or the variant does not support the shape */
   RCP_ERR_LIMIT = -8      /* size beyond a fixed capacity of the entry point */
@@ -51,7 +51,8 @@ int rcp_last_cuda_error(void);
  * Weight packing (Section 4.4: W_q is pre-computed offline and stored sub-byte packed along the
  * input channel). codes: uint8 [N][K], each in {0,1,2,3}. words: uint32 [N][K/16].
  * K % 64 == 0. Synchronizes the stream before returning so that RCP_ERR_CODE can be reported;
- * on RCP_ERR_CODE the contents of `words` are unspecified.
+ * on RCP_ERR_CODE the contents of `words` are unspecified. Calls from several host threads or on several
+ * streams may overlap (up to 64 in flight keep separate error flags).
  */
 int rcp_pack_weights(const uint8_t* codes, int N, int K, uint32_t* words, void* stream);
 
@@ -153,7 +154,10 @@ int rcp_gemv_plan(int M, int N, int K, int sms, int* out, int cap);
  *   S_c[m][n] = sum over k with code[n][k] == c of q[m][k]       (exact integers)
  *   y[m][n]   = fp16( scale[m] * sum_c lut[n][c] * S_c[m][n] )   (fp32 arithmetic)
  * Constraints: 1 <= M <= 16, N >= 1, K % 64 == 0, 64 <= K <= 65536.
- *   workspace  rcp_gemv_workspace_bytes(M,N,K) bytes, see above; NULL is accepted (no status word).
+ *   workspace  rcp_gemv_workspace_bytes(M,N,K) bytes, see above. Required (RCP_ERR_WORKSPACE without it): every
+ *              wait inside the streaming kernels is bounded, and a wait that gives up writes a non-zero code
+ *              into its first word (2: the weight producer, 3: a consumer warp) and ends the kernel; the
+ *              results of that call are then invalid. Only RCP_GEMV_SIMPLE (no waits) takes NULL.
  *   words, lut_f16 are the constants of the layer: the kernel may start fetching them while earlier
  *              work on the stream is still running (programmatic dependent launch), so that work
  *              must not be writing them. xq, scale, y and workspace obey stream order as usual.
@@ -175,9 +179,9 @@ int rcp_gemv_w2a4_variant(int variant, const uint32_t* words, const void* lut_f1
 
 /*
  * Export of a layer trained with learnable direct partitioning to the GEMV's inputs: 2-bit codes,
- * packed, and the four-entry grid of every quantization unit (Section 3.3: Eq. "partition", the
- * equation for t_i, Eq. "quant", Eq. "dequantgrid"; Section 3.4, Eq. "deqgrid"; clipping range of
- * Section 3.2). Offline, like rcp_pack_weights. A unit is `group` consecutive weights of a row:
+ * packed, and the four-entry grid of every quantization unit (Section 4.3: Eq. "partition", the
+ * equation for t_i, Eq. "quant", Eq. "dequantgrid"; Section 4.4, Eq. "deqgrid"; clipping range of
+ * Section 4.2). Offline, like rcp_pack_weights. A unit is `group` consecutive weights of a row:
  *   lo = sig_beta * min(W), hi = sig_gamma * max(W), h = hi - lo, W clipped to [lo, hi];
  *   p1 = sig_s1, p2 = (1 - p1) sig_s2, p3 = (1 - p1)(1 - sig_s2);
  *   t1 = p1/2, t2 = t1 + (p1 + p2)/2, t3 = t2 + (p2 + p3)/2;
@@ -191,7 +195,11 @@ int rcp_gemv_w2a4_variant(int variant, const uint32_t* words, const void* lut_f1
  *   words      DEVICE uint32 [N][K/16] (the format of rcp_pack_weights);
  *   lut_f16    DEVICE fp16 [N][K/group][4] (the lut of rcp_gemv_w2a4_grouped; of rcp_gemv_w2a4 when
  *              group == K).
- * Never synchronizes.
+ * Never synchronizes. The GEMV entry points treat words and lut_f16 as constants of the layer and may fetch
+ * them before earlier work on their stream has finished (see rcp_gemv_w2a4): let this call complete (stream or
+ * event synchronization) before the first GEMV or linear call that reads what it wrote, unless that call is on
+ * the same stream directly behind it -- this kernel never signals an early start, so the next kernel on the stream
+ * begins only when it has finished.
  */
 int rcp_ldp_export(const void* w_f16, const float* sig_beta, const float* sig_gamma,
                    const float* sig_s1, const float* sig_s2, int N, int K, int group,
@@ -199,7 +207,7 @@ int rcp_ldp_export(const void* w_f16, const float* sig_beta, const float* sig_ga
 
 /*
  * LUT GEMV with one grid per group of weights (Section 4.4: the dequantization grid has shape
- * H x N*4 for N groups per row; Appendix A.1: C = N*G; the table of quantization configurations
+ * H x N*4 for N groups per row; Appendix A.3: C = N*G; the table of quantization configurations
  * sets the weight group size G = 128). Weight k of row n takes its levels from lut[n][k / group]:
  *   S_c[m][n][j] = sum over k in [j*group, (j+1)*group) with code[n][k] == c of q[m][k]   (exact)
  *   y[m][n]      = fp16( scale[m] * sum_j sum_c lut[n][j][c] * S_c[m][n][j] )   (fp32 arithmetic;
@@ -302,6 +310,24 @@ int rcp_linear_w2a4_host(const void* x_host_f16, int M, int K, int had_block, fl
 #define RCP_STATIC_SCRATCH_BYTES 4096u
 int rcp_gemv_w2a4_static(const uint32_t* words, const void* lut_f16, const uint8_t* xq,
                          const void* scale_f16, int M, int N, int K, void* y_f16, void* stream);
+
+/*
+ * The status word of the built-in scratch array (the paper has no counterpart). rcp_gemv_w2a4 callers can look
+ * into their own workspace after a call; callers of rcp_gemv_w2a4_static cannot see the array, so this copies
+ * its first word to *status_host: 0 = every wait of the calls since the last clearing ended normally, 2 or 3 = a
+ * bounded wait gave up (see rcp_gemv_w2a4) and the results of that call are invalid. Synchronizes `stream`;
+ * allocates nothing.
+ */
+int rcp_gemv_w2a4_static_status(int32_t* status_host, void* stream);
+
+/*
+ * Self-test of the failure report (a test aid; the paper has no counterpart): launches one thread that waits,
+ * with the bounded wait of the GEMV kernels and a limit of `polls` polls (1 .. 2^20), on a barrier nobody
+ * arrives at. The wait runs out, the kernel writes code 3 into the first word of `workspace` (NULL: the
+ * built-in scratch array of rcp_gemv_w2a4_static) and returns; the context stays usable. Nothing faults and
+ * nothing hangs: the limit is the point. Asynchronous on `stream`.
+ */
+int rcp_selftest_wait_timeout(void* workspace, int polls, void* stream);
 
 #ifdef __cplusplus
 }

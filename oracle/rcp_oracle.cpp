@@ -382,7 +382,7 @@ void orc_dequant_weights(const uint32_t* words, const uint16_t* lut_f16, int N, 
 
 // ---------------------------------------------------------------------------------------
 // Group-wise LUT GEMV. Section 4.4 gives the dequantization grid the shape H x (N*4) with N
-// groups per input channel row, and Appendix A.1 sets C = N*G with group size G (128 in the
+// groups per input channel row, and Appendix A.3 sets C = N*G with group size G (128 in the
 // table of quantization configurations): weight k of row n takes its four levels from group
 // k / G. For token m, row n, group j:
 //   S_c[m][n][j] = sum over k in [jG, (j+1)G) with code[n][k] == c of q[m][k]   (exact integers)
@@ -468,9 +468,9 @@ void orc_percode_int_grouped(const uint16_t* lut_f16, const int32_t* S, int M, i
 }
 
 // ---------------------------------------------------------------------------------------
-// Learnable direct partitioning, export of a trained layer to the kernel's inputs (Section 3.3,
-// Eqs. "partition", the grid t_i, "quant", "dequantgrid" and Section 3.4 Eq. "deqgrid"; clipping
-// range from Section 3.2). One quantization unit = G consecutive weights of a row. Per unit, in
+// Learnable direct partitioning, export of a trained layer to the kernel's inputs (Section 4.3,
+// Eqs. "partition", the grid t_i, "quant", "dequantgrid" and Section 4.4 Eq. "deqgrid"; clipping
+// range from Section 4.2). One quantization unit = G consecutive weights of a row. Per unit, in
 // fp32 with one rounding per operation (the precision the export kernel works in):
 //   lo = sb * min(W_r), hi = sg * max(W_r), h = hi - lo      (sb, sg: the sigmoids of beta, gamma)
 //   W_rc = clip(W_r, lo, hi)

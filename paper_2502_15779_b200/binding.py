@@ -11,7 +11,8 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "librcp_w2a4.so")
+# RCP_W2A4_LIB names another build of the same library (the tests use it for the guarded build)
+LIB_PATH = os.environ.get("RCP_W2A4_LIB") or os.path.join(_HERE, "librcp_w2a4.so")
 
 GEMV_AUTO, GEMV_SIMPLE, GEMV_DP4A, GEMV_MMA, GEMV_MMA_ONLY = 0, 1, 2, 3, 4
 VARIANTS = {"auto": GEMV_AUTO, "simple": GEMV_SIMPLE, "dp4a": GEMV_DP4A, "mma": GEMV_MMA, "mma_only": GEMV_MMA_ONLY}
@@ -64,6 +65,10 @@ def lib():
         L.rcp_gemv_w2a4_static.argtypes = [vp, vp, vp, vp, i, i, i, vp, vp]
         L.rcp_gemv_w2a16.restype = i
         L.rcp_gemv_w2a16.argtypes = [vp, vp, vp, i, i, i, vp, vp, vp, vp, vp]
+        L.rcp_gemv_w2a4_static_status.restype = i
+        L.rcp_gemv_w2a4_static_status.argtypes = [vp, vp]
+        L.rcp_selftest_wait_timeout.restype = i
+        L.rcp_selftest_wait_timeout.argtypes = [vp, i, vp]
         L.rcp_gemv_w2a16_checked.restype = i
         L.rcp_gemv_w2a16_checked.argtypes = [vp, vp, vp, i, i, i, vp, vp, vp, vp, vp, vp]
         L.rcp_linear_w2a4_checked.restype = i

@@ -5,6 +5,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librcp_w2a4.so")
+LIB_CHECKED = os.path.join(HERE, "librcp_w2a4_checked.so")   # the guarded build (-DRCP_CHECKED), for tests
 SOURCES = ["rcp_api.cu"]
 
 
@@ -14,16 +15,29 @@ def _newest_source_mtime() -> float:
     return max(os.path.getmtime(p) for p in paths)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest_source_mtime():
-        return LIB
+def _compile(out: str, defines=(), verbose: bool = False) -> str:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "--shared", "-Xcompiler", "-fPIC", "-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES]
+           "--shared", "-Xcompiler", "-fPIC", "-o", out] + [f"-D{d}" for d in defines] + \
+          [os.path.join(CSRC, s) for s in SOURCES]
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
     subprocess.check_call(cmd)
-    return LIB
+    return out
+
+
+def build(force: bool = False, verbose: bool = False) -> str:
+    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest_source_mtime():
+        return LIB
+    return _compile(LIB, verbose=verbose)
+
+
+def build_checked(force: bool = False) -> str:
+    """The guarded build: the same sources with -DRCP_CHECKED (shared-memory addresses and TMA requests of the
+    streaming kernel checked against the host's layout; a violation is reported through the status word)."""
+    if not force and os.path.exists(LIB_CHECKED) and os.path.getmtime(LIB_CHECKED) >= _newest_source_mtime():
+        return LIB_CHECKED
+    return _compile(LIB_CHECKED, defines=("RCP_CHECKED",))
 
 
 if __name__ == "__main__":

@@ -41,6 +41,27 @@
 #include "quantize_act.cuh"
 #include "split_act16.cuh"
 
+// Guarded build (-DRCP_CHECKED): compute-sanitizer's stand-in. Every shared-memory address the streaming kernel
+// forms for the weight ring, the expanded activations, the reduction buffers and the parked sums, and every TMA
+// request, is checked against the area the host laid out; a violation skips the access and leaves 16 + the
+// number of the site in the status word (the largest such code wins) instead of faulting. The production build
+// compiles none of it.
+#ifdef RCP_CHECKED
+#define RCP_CK(cond, site) ((cond) ? true : (ck_fail(site), false))
+#define RCP_LDS128(addr, lo, hi, site) \
+  ([&]() -> uint4 { const uint32_t a__ = (addr); \
+     if (!RCP_CK(a__ >= (lo) && a__ + 16u <= (hi) && (a__ & 15u) == 0, site)) return make_uint4(0, 0, 0, 0); \
+     return lds128(a__); }())
+#define RCP_LDS64(addr, lo, hi, site) \
+  ([&]() -> uint2 { const uint32_t a__ = (addr); \
+     if (!RCP_CK(a__ >= (lo) && a__ + 8u <= (hi) && (a__ & 7u) == 0, site)) return make_uint2(0, 0); \
+     return lds64(a__); }())
+#else
+#define RCP_CK(cond, site) (true)
+#define RCP_LDS128(addr, lo, hi, site) lds128(addr)
+#define RCP_LDS64(addr, lo, hi, site) lds64(addr)
+#endif
+
 namespace rcp {
 
 constexpr int kCWarps = 16;                       // consumer warps
@@ -96,6 +117,7 @@ struct GemvParams {
   int stages;           // ring depth
   int ramp_clk;         // clocks between the first `stages` requests of a CTA
   int off_bar, off_T0c, off_scale, off_red, off_bs;   // shared-memory byte offsets from the aligned base
+  int bs_bytes, red_bytes, part_bytes;                // sizes of the areas at off_bs, off_red, off_part (guarded build)
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -120,14 +142,15 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait. Returns false after kSpinLimit polls.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kSpinLimit; i++) {
+// Bounded wait. Returns false after `limit` polls.
+__device__ __forceinline__ bool mbar_wait_n(uint32_t bar, uint32_t parity, uint32_t limit) {
+  for (uint32_t i = 0; i < limit; i++) {
     if (mbar_try(bar, parity)) return true;
     __nanosleep(64);   // leave the issue slots to the warps that have work
   }
   return false;
 }
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) { return mbar_wait_n(bar, parity, kSpinLimit); }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
@@ -180,6 +203,19 @@ __device__ __forceinline__ void dp4a_u8s8(int& d, uint32_t a, uint32_t b) {
 }
 __device__ __forceinline__ void dp4a_s8s8(int& d, uint32_t a, uint32_t b) {
   asm("dp4a.s32.s32 %0, %1, %2, %0;" : "+r"(d) : "r"(a), "r"(b));
+}
+
+// Self-test of the bounded wait and its report (a test aid, not part of the data path): one thread waits, with
+// the routine the GEMV kernels wait with and a limit of the caller's choice, on a barrier that nobody ever
+// arrives at. The wait gives up, the status word receives the consumer-side code, the kernel returns.
+__global__ void wait_timeout_kernel(int32_t* status, uint32_t polls) {
+  __shared__ __align__(8) unsigned long long bar_mem;
+  if (threadIdx.x == 0) {
+    const uint32_t bar = smem_u32(&bar_mem);
+    mbar_init(bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (!mbar_wait_n(bar, 0, polls)) atomicExch(status, 3);
+  }
 }
 
 // Expanded activations. A chunk is 32 words of a row; consumer lane t reads 16-byte chunk 2t+i of
@@ -244,6 +280,13 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   const int ng4 = 4 * p.nchunk;
   const int Mp = (M + 1) & ~1;
   uint8_t* const bs = gen + p.off_bs;
+#ifdef RCP_CHECKED
+  auto ck_fail = [&](int site) { if (p.status) atomicMax(p.status, 16 + site); };
+#endif
+  // areas of the layout (used by the guarded build's checks only)
+  const uint32_t ring_lo = base, ring_hi = base + (uint32_t)stages * kStageBytes;
+  const uint32_t bs_lo = base + (uint32_t)p.off_bs, bs_hi = bs_lo + (uint32_t)p.bs_bytes;
+  (void)ring_lo; (void)ring_hi; (void)bs_lo; (void)bs_hi;
 
   const int b = blockIdx.x;
   // Launched with programmatic stream serialization: the next kernel may start as CTAs retire.
@@ -302,8 +345,12 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
           const uint32_t bar = full0 + 8 * slot, dst = base + (uint32_t)slot * kStageBytes;
           const int nbox = kSplit ? max(0, min(KS, nch - s * KS)) : min(KS, nch - s * KS);   // a short last part can leave a stage empty
           mbar_expect_tx(bar, (uint32_t)nbox * box);
-          for (int j = 0; j < nbox; j++)
-            tma_load_2d(dst + (uint32_t)j * box, &maps.m[pi], (chunk0 + s * KS + j) * kChunkWords, row0, bar);
+          for (int j = 0; j < nbox; j++) {
+            const int xw = (chunk0 + s * KS + j) * kChunkWords;   // first word of the box: a multiple of 32, so 16-byte aligned
+            if (RCP_CK(dst + (uint32_t)(j + 1) * box <= ring_hi && ((dst + (uint32_t)j * box) & 1023u) == 0 && xw >= 0 &&
+                       xw < p.K / 16 && (xw & 3) == 0 && row0 >= 0 && row0 < p.N && pi < kMaxPhases, 1))
+              tma_load_2d(dst + (uint32_t)j * box, &maps.m[pi], xw, row0, bar);
+          }
           issued++;
           if (++slot == stages) { slot = 0; phase ^= 1u; }
         }
@@ -358,10 +405,12 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
                 ((uint32_t)((q[8 + pp] * m) & 0xFF) << 16) | ((uint32_t)((q[12 + pp] * m) & 0xFF) << 24);
       }
       uint8_t* dst = bs + (size_t)((ch * 4 + ((wi >> 1) & 3)) * 2) * 64 + (wi >> 3) * 16 + (wi & 1) * 4;
-      *reinterpret_cast<uint32_t*>(dst) = Q[0];
-      *reinterpret_cast<uint32_t*>(dst + 8) = Q[1];
-      *reinterpret_cast<uint32_t*>(dst + 64) = Q[2];
-      *reinterpret_cast<uint32_t*>(dst + 64 + 8) = Q[3];
+      if (RCP_CK(dst >= bs && dst + 64 + 12 <= bs + p.bs_bytes, 2)) {
+        *reinterpret_cast<uint32_t*>(dst) = Q[0];
+        *reinterpret_cast<uint32_t*>(dst + 8) = Q[1];
+        *reinterpret_cast<uint32_t*>(dst + 64) = Q[2];
+        *reinterpret_cast<uint32_t*>(dst + 64 + 8) = Q[3];
+      }
     }
     if (b == 0 && p.xq_out && tid < W) {
       uint32_t lo32 = 0, hi32 = 0;
@@ -518,8 +567,10 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
           q[3][w] = __byte_perm(n4[1], n4[3], 0x7531);
         }
         uint8_t* dst = bs + ((size_t)(((ch * 4 + hi) * 2) * ncol + col)) * 64 + lo * 16;
-        *reinterpret_cast<uint4*>(dst) = make_uint4(q[0][0], q[0][1], q[1][0], q[1][1]);
-        *reinterpret_cast<uint4*>(dst + (size_t)ncol * 64) = make_uint4(q[2][0], q[2][1], q[3][0], q[3][1]);
+        if (RCP_CK(dst >= bs && dst + (size_t)ncol * 64 + 16 <= bs + p.bs_bytes, 3)) {
+          *reinterpret_cast<uint4*>(dst) = make_uint4(q[0][0], q[0][1], q[1][0], q[1][1]);
+          *reinterpret_cast<uint4*>(dst + (size_t)ncol * 64) = make_uint4(q[2][0], q[2][1], q[3][0], q[3][1]);
+        }
       }
       if constexpr (!GRP) {
 #pragma unroll
@@ -627,8 +678,8 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     const uint32_t b_ptr = base + (uint32_t)p.off_bs + b_chunk;
 #pragma unroll
     for (int i = 0; i < 2; i++) {
-      const uint4 U = lds128(a_ptr + a_chunk[i]);
-      const uint4 V = lds128(a_ptr + 8 * 128 + a_chunk[i]);
+      const uint4 U = RCP_LDS128(a_ptr + a_chunk[i], ring_lo, ring_hi, 4);
+      const uint4 V = RCP_LDS128(a_ptr + 8 * 128 + a_chunk[i], ring_lo, ring_hi, 4);
       const uint32_t uw[4] = {U.x, U.y, U.z, U.w};
       const uint32_t vw[4] = {V.x, V.y, V.z, V.w};
 #pragma unroll
@@ -640,8 +691,8 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
         if constexpr (NF_D > 0) {
 #pragma unroll
           for (int tok = 0; tok < NTD; tok++) {
-            const uint4 x = lds128(b_ptr + bD_lane[tok] + b_off);
-            const uint4 y = lds128(b_ptr + bD_lane[tok] + b_off + half_stride);
+            const uint4 x = RCP_LDS128(b_ptr + bD_lane[tok] + b_off, bs_lo, bs_hi, 5);
+            const uint4 y = RCP_LDS128(b_ptr + bD_lane[tok] + b_off + half_stride, bs_lo, bs_hi, 5);
             bD[tok][0][0] = x.x; bD[tok][0][1] = x.y; bD[tok][1][0] = x.z; bD[tok][1][1] = x.w;
             bD[tok][2][0] = y.x; bD[tok][2][1] = y.y; bD[tok][3][0] = y.z; bD[tok][3][1] = y.w;
           }
@@ -651,16 +702,16 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
 #pragma unroll
             for (int pp = 0; pp < 4; pp++) { bM[pp][0] = bD[0][pp][0]; bM[pp][1] = bD[0][pp][1]; }
           } else {
-            const uint4 x = lds128(b_ptr + bM_lane + b_off);
-            const uint4 y = lds128(b_ptr + bM_lane + b_off + half_stride);
+            const uint4 x = RCP_LDS128(b_ptr + bM_lane + b_off, bs_lo, bs_hi, 6);
+            const uint4 y = RCP_LDS128(b_ptr + bM_lane + b_off + half_stride, bs_lo, bs_hi, 6);
             bM[0][0] = x.x; bM[0][1] = x.y; bM[1][0] = x.z; bM[1][1] = x.w;
             bM[2][0] = y.x; bM[2][1] = y.y; bM[3][0] = y.z; bM[3][1] = y.w;
           }
         }
         uint32_t bN[4][2];
         if constexpr (kTwoTiles) {
-          const uint4 x = lds128(b_ptr + bN_lane + b_off);
-          const uint4 y = lds128(b_ptr + bN_lane + b_off + half_stride);
+          const uint4 x = RCP_LDS128(b_ptr + bN_lane + b_off, bs_lo, bs_hi, 7);
+          const uint4 y = RCP_LDS128(b_ptr + bN_lane + b_off + half_stride, bs_lo, bs_hi, 7);
           bN[0][0] = x.x; bN[0][1] = x.y; bN[1][0] = x.z; bN[1][1] = x.w;
           bN[2][0] = y.x; bN[2][1] = y.y; bN[3][0] = y.z; bN[3][1] = y.w;
         }
@@ -779,11 +830,11 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
 #pragma unroll
       for (int j = 0; j < 4; j++) {
         const uint32_t a_sw = (uint32_t)(((2 * j + (t >> 1)) ^ (grow & 7)) << 4);
-        const uint2 U = lds64(a_row + a_sw);
-        const uint2 V = lds64(a_row + 8 * 128 + a_sw);
+        const uint2 U = RCP_LDS64(a_row + a_sw, ring_lo, ring_hi, 8);
+        const uint2 V = RCP_LDS64(a_row + 8 * 128 + a_sw, ring_lo, ring_hi, 8);
         const uint32_t b_ptr = b_grp + (uint32_t)(j * 2) * half_stride;
-        const uint4 x = lds128(b_ptr);
-        const uint4 y = lds128(b_ptr + half_stride);
+        const uint4 x = RCP_LDS128(b_ptr, bs_lo, bs_hi, 9);
+        const uint4 y = RCP_LDS128(b_ptr + half_stride, bs_lo, bs_hi, 9);
         const uint32_t bM[4][2] = {{x.x, x.y}, {x.z, x.w}, {y.x, y.y}, {y.z, y.w}};
         const uint32_t u0 = U.x, u1 = U.y, v0 = V.x, v1 = V.y;
         const uint32_t u0s = u0 + u0, u1s = u1 + u1, v0s = v0 + v0, v1s = v1 + v1;
@@ -854,7 +905,9 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
         nred++;
 #pragma unroll
         for (int e = 0; e < NE; e++)
-          if (active && etok[e] < M) red[(warp * 16 + g + 8 * err[e]) * M + etok[e]] = yacc[e];
+          if (active && etok[e] < M &&
+              RCP_CK(((nred - 1) & 1) * (kCWarps * 16 * M) + (warp * 16 + g + 8 * err[e]) * M + etok[e] < p.red_bytes / 4, 10))
+            red[(warp * 16 + g + 8 * err[e]) * M + etok[e]] = yacc[e];
         asm volatile("bar.sync 2, %0;" ::"n"(kCWarps * 32) : "memory");   // consumer warps only
         if (active && ks == 0) {
 #pragma unroll
@@ -982,6 +1035,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
       for (int e = 0; e < NE; e++) {
         if (etok[e] < M) {
           int* d = s_part + ((gslot * 16 + g + 8 * err[e]) * M + etok[e]) * 3;
+          if (!RCP_CK(gslot >= 0 && (((gslot * 16 + g + 8 * err[e]) * M + etok[e]) * 3 + 3) * 4 <= p.part_bytes, 11)) continue;
           if (kp > 0) { T1[e] += d[0]; T2[e] += d[1]; T3[e] += d[2]; }
           if (kp + 1 < nsplit) { d[0] = T1[e]; d[1] = T2[e]; d[2] = T3[e]; }
         }
@@ -1058,7 +1112,8 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
         nred++;
 #pragma unroll
         for (int e = 0; e < NE; e++) {
-          if (active && etok[e] < M) {
+          if (active && etok[e] < M &&
+              RCP_CK(grp < 8 && (((nred - 1) & 1) * (8 * 16 * M * 3) + ((grp * 16 + g + 8 * err[e]) * M + etok[e]) * 3 + 3) * 4 <= p.red_bytes, 12)) {
             int* d = red + ((grp * 16 + g + 8 * err[e]) * M + etok[e]) * 3;
             atomicAdd(d + 0, T1[e]);
             atomicAdd(d + 1, T2[e]);

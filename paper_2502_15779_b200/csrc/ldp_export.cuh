@@ -1,6 +1,6 @@
-// Export of a layer trained with learnable direct partitioning to the GEMV's inputs (Section 3.3:
-// Eq. "partition", the grid t_i, Eq. "quant", Eq. "dequantgrid"; Section 3.4 Eq. "deqgrid"; the
-// clipping range of Section 3.2). An offline, one-pass kernel: 2 bytes read and a quarter byte
+// Export of a layer trained with learnable direct partitioning to the GEMV's inputs (Section 4.3:
+// Eq. "partition", the grid t_i, Eq. "quant", Eq. "dequantgrid"; Section 4.4 Eq. "deqgrid"; the
+// clipping range of Section 4.2). An offline, one-pass kernel: 2 bytes read and a quarter byte
 // written per weight. One warp per quantization unit (G consecutive weights of a row): the range by
 // shuffles, the three thresholds and four levels in fp32 with one rounding per operation (so the
 // 2-bit decision is reproducible bit for bit), codes packed 16 to a word straight away.

@@ -2,15 +2,13 @@
 // per-token absmax symmetric int4 quantization -> nibble packing (Section 4.4 tensor formats).
 //
 // A token is one vector of K elements and the whole job is latency: a thread-block cluster of C
-// CTAs (1, 2, 4 or 8) shares it, each CTA a contiguous slice, every thread 8 consecutive
+// CTAs (1, 2, 4 or 8) shares it, each CTA whole rotation blocks, every thread 8 consecutive
 // elements. The butterfly strides run in ascending order: 1,2,4 inside the thread's registers,
-// 8..128 by warp shuffles, 256 up to the slice through the CTA's shared memory in radix-8 passes,
-// and the strides that span slices (a rotation block larger than a slice) across the cluster:
-// every CTA reads the partner slices through distributed shared memory and redoes the small
-// butterfly network over the ranks, keeping its own output. Each butterfly is one fp32 add and
-// one fp32 subtract (lower index first), then one fp32 multiply by 1/sqrt(B): the rounding order
-// is fixed, so the int4 decision is reproducible bit for bit. The token's absmax meets in
-// distributed shared memory as well.
+// 8..128 by warp shuffles, 256 and up through the CTA's shared memory in radix-8 passes. (A rotation
+// block never spans CTAs: one block over a token of 4096 or 8192 elements takes the one-CTA kernel
+// further down, shorter tokens fit one CTA.) Each butterfly is one fp32 add and one fp32 subtract
+// (lower index first), then one fp32 multiply by 1/sqrt(B): the rounding order is fixed, so the int4
+// decision is reproducible bit for bit. The token's absmax meets in distributed shared memory.
 #pragma once
 #include "common.cuh"
 
@@ -28,28 +26,14 @@ __device__ __forceinline__ float ld_cluster_f32(const float* local, uint32_t ran
   asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(raddr) : "memory");
   return v;
 }
-// the same for four consecutive floats (16-byte aligned)
-__device__ __forceinline__ float4 ld_cluster_f32x4(const float* local, uint32_t rank) {
-  const uint32_t laddr = (uint32_t)__cvta_generic_to_shared(local);
-  uint32_t raddr;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(raddr) : "r"(laddr), "r"(rank));
-  float4 v;
-  asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];"
-               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-               : "r"(raddr)
-               : "memory");
-  return v;
-}
 
 struct QuantParams {
   const __half* x;
   uint8_t* xq;
   __half* scale;
   int K, B, lgB;
-  int unit, nunits;     // cross == 1: the token is shared out in units of `unit` elements (a multiple of B and 64)
-  int slice;            // cross > 1: elements per CTA (a power of two, 256 .. 8192), K == B == cross * slice
-  int lg_local;         // B > 256: log2 of min(B, slice): strides below it stay inside the CTA
-  int cross;            // CTAs one rotation block is split over (1, 2, 4 or 8)
+  int unit, nunits;     // the token is shared out over the cluster in units of `unit` elements (a multiple of B and 64)
+  int lg_local;         // B > 256: log2 B, the strides that go through shared memory end below it
   float inv_sqrt_b, clip_ratio;
 };
 
@@ -69,15 +53,8 @@ __global__ void __launch_bounds__(1024) quantize_act_kernel(const QuantParams p)
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
   // this CTA's slice of the token
-  int start, len;
-  if (p.cross == 1) {
-    const int u0 = (int)((long long)p.nunits * rank / C), u1 = (int)((long long)p.nunits * (rank + 1) / C);
-    start = u0 * p.unit;
-    len = (u1 - u0) * p.unit;
-  } else {
-    start = (int)rank * p.slice;
-    len = p.slice;
-  }
+  const int u0 = (int)((long long)p.nunits * rank / C), u1 = (int)((long long)p.nunits * (rank + 1) / C);
+  const int start = u0 * p.unit, len = (u1 - u0) * p.unit;
   const int base = start + tid * 8;
   const bool mine = tid * 8 < len;
   const __half* xm = p.x + (size_t)m * p.K;
@@ -125,7 +102,7 @@ __global__ void __launch_bounds__(1024) quantize_act_kernel(const QuantParams p)
       }
     }
     if (B > 256) {
-      // strides 256 .. below min(B, slice): passes of up to three strides (radix 8) through shared
+      // strides 256 .. B/2: passes of up to three strides (radix 8) through shared
       // memory. A pass over strides s, 2s, .. (r = 2, 4 or 8 of them combined) works on tuples of r
       // elements s apart; the tuple index maps to an element index with shifts only:
       // element = ((tuple >> log2 s) << log2(r s)) | (tuple & (s - 1)), plus j s for the j-th member.
@@ -162,51 +139,8 @@ __global__ void __launch_bounds__(1024) quantize_act_kernel(const QuantParams p)
         __syncthreads();
         ls += lr;
       }
-      if constexpr (C > 1) {
-        if (p.cross > 1) {
-          // strides slice .. B/2: the partner elements sit at the same offset in the other CTAs of
-          // an aligned group of `cross` ranks; run the butterflies over the ranks, keep this rank's
-          cluster_sync_all();
-          const uint32_t g0 = rank & ~(uint32_t)(p.cross - 1), me = rank - g0;
-          float w[C][8];
 #pragma unroll
-          for (int r = 0; r < C; r++) {
-            float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
-            if (r < p.cross) {
-              a = ld_cluster_f32x4(&sbuf[tid * 8], g0 + r);
-              b = ld_cluster_f32x4(&sbuf[tid * 8 + 4], g0 + r);
-            }
-            w[r][0] = a.x; w[r][1] = a.y; w[r][2] = a.z; w[r][3] = a.w;
-            w[r][4] = b.x; w[r][5] = b.y; w[r][6] = b.z; w[r][7] = b.w;
-          }
-#pragma unroll
-          for (int e = 0; e < 8; e++) {
-#pragma unroll
-            for (int h = 1; h < C; h *= 2) {
-              if (h < p.cross) {
-#pragma unroll
-                for (int r = 0; r < C; r++) {
-                  if ((r & h) == 0) {
-                    const float u = w[r][e], z = w[r + h][e];
-                    w[r][e] = __fadd_rn(u, z);
-                    w[r + h][e] = __fsub_rn(u, z);
-                  }
-                }
-              }
-            }
-            float out = w[0][e];
-#pragma unroll
-            for (int r = 1; r < C; r++) out = (me == (uint32_t)r) ? w[r][e] : out;
-            v[e] = out;
-          }
-        } else {
-#pragma unroll
-          for (int e = 0; e < 8; e++) v[e] = sbuf[tid * 8 + e];
-        }
-      } else {
-#pragma unroll
-        for (int e = 0; e < 8; e++) v[e] = sbuf[tid * 8 + e];
-      }
+      for (int e = 0; e < 8; e++) v[e] = sbuf[tid * 8 + e];
     }
 #pragma unroll
     for (int e = 0; e < 8; e++) v[e] = __fmul_rn(v[e], p.inv_sqrt_b);

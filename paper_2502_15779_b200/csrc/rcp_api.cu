@@ -2,6 +2,7 @@
 #include "../../include/rcp.h"
 
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstring>
 #include <mutex>
@@ -53,7 +54,11 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 bool k_ok(int K) { return K >= 64 && K <= rcp::kMaxK && K % 64 == 0; }
 
-__device__ int g_pack_bad;  // set by pack_weights_kernel when it meets a code above 3
+// Set by pack_weights_kernel when it meets a code above 3. One slot per call in flight (calls from several host
+// threads or on several streams take different slots, so that none clears or reads another's flag).
+constexpr unsigned kPackSlots = 64;
+__device__ int g_pack_bad[kPackSlots];
+std::atomic<unsigned> g_pack_next{0};
 
 // ---------------------------------------------------------------------------------------------
 // Streaming GEMV: launch plan.
@@ -61,6 +66,7 @@ struct StreamPlan {
   int nchunk, nchunk_total, nsplit, nphase, stages, grid;   // nchunk: chunks per row in one part of K
   rcp::GemvPhase phase[rcp::kMaxPhases];
   int off_bar, off_T0c, off_scale, off_red, off_bs, off_qbuf, off_part;
+  int bs_bytes, red_bytes, part_bytes;
   size_t smem;
 };
 
@@ -195,6 +201,7 @@ StreamPlan make_plan(int M, int N, int K, int sms, bool grouped, size_t qbuf, in
   pl.off_bs = (int)off; off += bs_bytes;
   pl.off_qbuf = (int)off; off += qbuf;
   pl.off_part = (int)off; off += part_bytes;
+  pl.bs_bytes = (int)bs_bytes; pl.red_bytes = (int)red_bytes; pl.part_bytes = (int)part_bytes;
   pl.smem = off + 1024;
   return pl;
 }
@@ -350,6 +357,7 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   gp.ramp_clk = (int)((double)rcp::kStageBytes * pl.grid / 6.0e12 * 1.9e9);
   gp.off_bar = pl.off_bar; gp.off_T0c = pl.off_T0c; gp.off_scale = pl.off_scale; gp.off_red = pl.off_red;
   gp.off_bs = pl.off_bs;
+  gp.bs_bytes = pl.bs_bytes; gp.red_bytes = pl.red_bytes; gp.part_bytes = pl.part_bytes;
   gp.off_qbuf = pl.off_qbuf;
   gp.x = nullptr; gp.xq_out = nullptr; gp.scale_out = nullptr; gp.unit_out = nullptr;
   gp.inv_sqrt_b = 1.f; gp.clip_ratio = 1.f;
@@ -460,6 +468,7 @@ int rcp_pack_weights(const uint8_t* codes, int N, int K, uint32_t* words, void* 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int* bad = nullptr;
   RCP_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&bad), g_pack_bad));
+  bad += g_pack_next.fetch_add(1) % kPackSlots;
   RCP_CUDA(cudaMemsetAsync(bad, 0, sizeof(int), st));
   const size_t nwords = (size_t)N * (K / 16);
   const int block = 256;
@@ -517,35 +526,23 @@ int rcp_quantize_act(const void* x_f16, int M, int K, int had_block, float clip_
   qp.clip_ratio = clip_ratio;
   if (B == K && (K == 4096 || K == 8192)) {
     // one rotation block over a long token: one CTA of 512 threads per token (measured faster than a cluster)
-    qp.cross = 1; qp.slice = 0; qp.unit = K; qp.nunits = 1; qp.lg_local = qp.lgB;
+    qp.unit = K; qp.nunits = 1; qp.lg_local = qp.lgB;
     RCP_CUDA(launch_overlapped(rcp::quantize_act_wide_kernel, dim3((unsigned)M), dim3(512), (size_t)4 * K, st, qp));
     return RCP_OK;
   }
+  // whole rotation blocks per CTA (a block is at most 2048 elements here: longer single blocks went above,
+  // and B <= 8192 < K otherwise means at least two blocks)
   int C = 1;
   while (C < 8 && K / (2 * C) >= 2048) C *= 2;
-  int T;
-  if (B == K && B > 256) {
-    // one rotation block: split it over the cluster, the top strides go through distributed shared memory
-    qp.cross = C;
-    qp.slice = K / C;
-    qp.unit = K; qp.nunits = 1;
-    qp.lg_local = qp.lgB;
-    while ((1 << qp.lg_local) > qp.slice) qp.lg_local--;
-    T = qp.slice / 8;
-  } else {
-    // whole rotation blocks per CTA
-    qp.cross = 1;
-    qp.slice = 0;
-    qp.unit = std::max(B, 64);
-    qp.nunits = K / qp.unit;
-    qp.lg_local = qp.lgB;
-    C = std::min(C, qp.nunits);
-    while (C > 1 && (C & (C - 1))) C--;   // power of two
-    int per = (qp.nunits + C - 1) / C;
-    while ((long long)per * qp.unit > 8192 && C < 8) { C *= 2; per = (qp.nunits + C - 1) / C; }
-    if ((long long)per * qp.unit > 8192) return RCP_ERR_SHAPE;
-    T = (per * qp.unit / 8 + 31) / 32 * 32;
-  }
+  qp.unit = std::max(B, 64);
+  qp.nunits = K / qp.unit;
+  qp.lg_local = qp.lgB;
+  C = std::min(C, qp.nunits);
+  while (C > 1 && (C & (C - 1))) C--;   // power of two
+  int per = (qp.nunits + C - 1) / C;
+  while ((long long)per * qp.unit > 8192 && C < 8) { C *= 2; per = (qp.nunits + C - 1) / C; }
+  if ((long long)per * qp.unit > 8192) return RCP_ERR_SHAPE;
+  const int T = (per * qp.unit / 8 + 31) / 32 * 32;
   const size_t smem = B > 256 ? (size_t)T * 8 * sizeof(float) : 0;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)M * C);
@@ -615,6 +612,8 @@ int rcp_gemv_w2a4_variant(int variant, const uint32_t* words, const void* lut_f1
   if (S_dbg && variant == RCP_GEMV_AUTO) variant = RCP_GEMV_SIMPLE;
   // measured on B200: one token runs fastest on the CUDA cores alone, more tokens on the tensor cores
   if (variant == RCP_GEMV_AUTO) variant = (M == 1) ? RCP_GEMV_DP4A : RCP_GEMV_MMA_ONLY;
+  // the streaming kernels wait on barriers with a bound and report a wait that gave up through the workspace
+  if (variant != RCP_GEMV_SIMPLE && !workspace) return RCP_ERR_WORKSPACE;
   switch (variant) {
     case RCP_GEMV_SIMPLE: {
       const int block = 256;
@@ -651,6 +650,7 @@ int rcp_gemv_w2a4(const uint32_t* words, const void* lut_f16, const uint8_t* xq,
 int rcp_gemv_w2a16_checked(const uint32_t* words, const void* lut_f16, const void* x_f16, int M, int N, int K,
                            void* y_f16, int8_t* digits, float* unit, void* workspace, int32_t* S_dbg, void* stream) {
   if (!words || !lut_f16 || !x_f16 || !y_f16 || !digits || !unit) return RCP_ERR_NULL;
+  if (!workspace) return RCP_ERR_WORKSPACE;
   if (!aligned16(S_dbg)) return RCP_ERR_ALIGN;
   if (M < 1 || M > rcp::kMaxTokens || N < 1 || !k_ok(K)) return RCP_ERR_SHAPE;
   if (!aligned16(words) || !aligned16(x_f16) || !aligned16(digits) || (reinterpret_cast<uintptr_t>(lut_f16) & 7u) ||
@@ -704,6 +704,7 @@ int rcp_gemv_w2a4_grouped_variant(int variant, const uint32_t* words, const void
   // the streaming kernels are built for the paper's group size; other sizes take the plain kernel
   if (variant == RCP_GEMV_AUTO && (S_dbg || group != 128)) variant = RCP_GEMV_SIMPLE;
   if (variant == RCP_GEMV_AUTO) variant = (M <= 2) ? RCP_GEMV_DP4A : RCP_GEMV_MMA_ONLY;
+  if (variant != RCP_GEMV_SIMPLE && !workspace) return RCP_ERR_WORKSPACE;
   switch (variant) {
     case RCP_GEMV_SIMPLE: {
       const int block = 256;
@@ -754,6 +755,30 @@ int rcp_gemv_w2a4_static(const uint32_t* words, const void* lut_f16, const uint8
                                stream);
 }
 
+int rcp_gemv_w2a4_static_status(int32_t* status_host, void* stream) {
+  if (!status_host) return RCP_ERR_NULL;
+  void* scratch = nullptr;
+  const int rc = static_scratch_address(&scratch);
+  if (rc != RCP_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  RCP_CUDA(cudaMemcpyAsync(status_host, scratch, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  RCP_CUDA(cudaStreamSynchronize(st));
+  return RCP_OK;
+}
+
+int rcp_selftest_wait_timeout(void* workspace, int polls, void* stream) {
+  if (polls < 1 || polls > (1 << 20)) return RCP_ERR_SHAPE;
+  if (reinterpret_cast<uintptr_t>(workspace) & 3u) return RCP_ERR_ALIGN;
+  void* status = workspace;
+  if (!status) {
+    const int rc = static_scratch_address(&status);
+    if (rc != RCP_OK) return rc;
+  }
+  rcp::wait_timeout_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<int32_t*>(status), (uint32_t)polls);
+  RCP_CUDA(cudaGetLastError());
+  return RCP_OK;
+}
+
 int rcp_linear_w2a4_launches(int M, int N, int K, int had_block, int group) {
   if (M < 1 || M > rcp::kMaxTokens || N < 1 || !k_ok(K)) return RCP_ERR_SHAPE;
   const int B = had_block <= 1 ? 1 : had_block;
@@ -780,6 +805,7 @@ int rcp_linear_w2a4_checked(const void* x_f16, int M, int K, int had_block, floa
       (reinterpret_cast<uintptr_t>(workspace) & 3u))
     return RCP_ERR_ALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (!workspace) return RCP_ERR_WORKSPACE;
   if (fused_ok(M, K, B) && (group == 0 || group == 128)) {
     const FusedAct fa{x_f16, B, clip_ratio, xq, scale_f16};
     return launch_stream(rcp::kModeDp4a, words, lut_f16, nullptr, nullptr, M, N, K, y_f16, workspace, st, group == 128,

@@ -76,6 +76,41 @@ def test_exported_layer_through_the_gemv(N, K, G, M):
     assert np.corrcoef(got.ravel(), full.ravel())[0, 1] > 0.6
 
 
+@pytest.mark.parametrize("N,K,G,M", [(2500, 8192, 128, 1), (3000, 4096, 4096, 1), (700, 2048, 128, 4)])
+def test_export_directly_followed_by_the_linear_call_on_one_stream(N, K, G, M):
+    """The export kernel and the linear call back to back on one stream, nothing in between (the GEMV kernels
+    start fetching the weights before the kernel in front of them has finished only if that kernel signals an
+    early start, which the export kernel never does). Repeated, so that a stale read would show."""
+    w, sb, sg, s1, s2 = _inputs(N, K, G, 3 * N + M)
+    wd, sbd, sgd, s1d, s2d = (t.to(DEV) for t in (w, sb, sg, s1, s2))
+    x = synth.make_activations(M, K, 13, device=DEV)
+    B = K if G == K else 128
+    ref_q = oracle.ldp_export(f16_bits(w), sb.numpy(), sg.numpy(), s1.numpy(), s2.numpy(), G)
+    qa = oracle.quantize_act(f16_bits(x), B, 1.0)
+    w_ref = oracle.pack_weights(ref_q["codes"])
+    ref = (oracle.gemv_w2a4(w_ref, ref_q["lut"].reshape(N, 4), qa["xq"], qa["scale"]) if G == K
+           else oracle.gemv_w2a4_grouped(w_ref, ref_q["lut"], qa["xq"], qa["scale"], G))
+    words = torch.empty((N, K // 16), dtype=torch.int32, device=DEV)
+    lut = torch.empty((N, K // G, 4), dtype=torch.float16, device=DEV)
+    xq = torch.empty(M, K // 2, dtype=torch.uint8, device=DEV)
+    scale = torch.empty(M, dtype=torch.float16, device=DEV)
+    ws = rcp.make_workspace(M, N, K, DEV)
+    L = rcp.lib()
+    import ctypes as C
+    st = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    for rep in range(5):
+        words.fill_(-1)
+        lut.fill_(float("nan"))
+        torch.cuda.synchronize()
+        assert L.rcp_ldp_export(wd.data_ptr(), sbd.data_ptr(), sgd.data_ptr(), s1d.data_ptr(), s2d.data_ptr(), N, K, G,
+                                words.data_ptr(), lut.data_ptr(), st) == 0
+        y = rcp.rcp_linear_w2a4(x, B, 1.0, words, lut.reshape(N, 4) if G == K else lut, group=0 if G == K else G,
+                                xq=xq, scale=scale, workspace=ws)
+        torch.cuda.synchronize()
+        got = y.float().cpu().numpy().astype(np.float64)
+        assert np.all(np.isfinite(got)) and np.all(np.abs(got - ref["y"]) <= ref["tol"]), f"repetition {rep}"
+
+
 def test_ldp_export_argument_errors():
     L = rcp.lib()
     z = torch.zeros(4096, dtype=torch.int32, device=DEV)

@@ -166,6 +166,26 @@ def test_gemv_degenerate_inputs():
         assert np.all(got[1] == 0)
 
 
+def test_bounded_wait_gives_up_reports_and_leaves_the_context_usable():
+    """Failure report of the streaming kernels, without a fault or a hang: a thread waits with their bounded
+    wait (a short limit) on a barrier nobody arrives at, gives up, writes its code into the workspace and
+    returns. A GEMV on the same context afterwards works; a call without a workspace is refused."""
+    import ctypes as C
+    L = rcp.lib()
+    ws = torch.zeros(4, dtype=torch.int32, device=DEV)
+    stream = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    assert L.rcp_selftest_wait_timeout(C.c_void_p(ws.data_ptr()), 3000, stream) == 0
+    torch.cuda.synchronize()
+    assert ws.cpu().tolist() == [3, 0, 0, 0]
+    ws.zero_()
+    _check_gemv(300, 2048, 128, 2, "uniform", "mma_only", seed=5)
+    z = torch.zeros(4096, dtype=torch.int32, device=DEV)
+    p = z.data_ptr()
+    assert L.rcp_gemv_w2a4(p, p, p, p, 1, 16, 64, p, None, None, None) == -5
+    assert L.rcp_gemv_w2a4_variant(1, p, p, p, p, 1, 16, 64, p, None, None, None) == 0   # the plain kernel has no waits
+    torch.cuda.synchronize()
+
+
 def test_gemv_argument_errors():
     L = rcp.lib()
     z = torch.zeros(4096, dtype=torch.int32, device=DEV)

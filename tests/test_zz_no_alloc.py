@@ -4,7 +4,8 @@ synchronization an allocation brings). Its scratch is an array inside the librar
 caller buffer, so the checks here are the ones that matter to such a caller: called through the C
 ABI with nothing but inputs and outputs, it must give what rcp_gemv_w2a4 gives, also the second
 time, when the shared array still holds whatever the first call left behind; and bad arguments must
-come back as status codes with nothing launched.
+come back as status codes with nothing put on the stream. A bounded wait that gives up is reported through
+the array's status word, which such a caller reads with rcp_gemv_w2a4_static_status; the next call clears it.
 
 This file sorts after the other test files on purpose: a run that stops at the first failure has
 then already run everything else."""
@@ -65,11 +66,31 @@ def test_static_scratch_entry_reports_errors_and_wrapper_agrees():
     for (M, N, K) in [(1, 57344, 8192), (16, 600000, 64), (8, 8192, 28672)]:
         assert 0 < rcp.rcp_gemv_workspace_bytes(M, N, K) <= rcp.binding.STATIC_SCRATCH_BYTES
     assert L.rcp_status_str(-8) not in (None, b"")       # the text of RCP_ERR_LIMIT
-    # bad arguments are reported like the existing entry point reports them, and nothing is launched
+    # bad arguments are reported like the existing entry point reports them, before anything reaches the stream
     assert L.rcp_gemv_w2a4_static(p, p, p, p, 1, 16, 96, p, None) == -2
     assert L.rcp_gemv_w2a4_static(None, p, p, p, 1, 16, 64, p, None) == -1
+    assert L.rcp_gemv_w2a4_static(C.c_void_p(z.data_ptr() + 4), p, p, p, 1, 16, 64, p, None) == -3
     # the Python wrapper gives the same bits as the existing entry point
     words, lut, xq, scale = _inputs(64, 256, 128, 1, seed=3)
     y = rcp.rcp_gemv_w2a4_static(words, lut, xq, scale)
     ws = rcp.make_workspace(1, 64, 256, DEV)
     assert torch.equal(y.view(torch.int16), rcp.rcp_gemv_w2a4(words, lut, xq, scale, workspace=ws).view(torch.int16))
+
+
+def test_static_scratch_status_word_reports_a_wait_that_gave_up_and_the_next_call_clears_it():
+    """The built-in array is dirtied the way a real failure would dirty it: a kernel whose bounded wait runs out
+    (nobody arrives at its barrier) writes its code into the status word. The caller sees it through the status
+    accessor; the next rcp_gemv_w2a4_static call clears the word before its kernel and gives the right answer."""
+    L = rcp.lib()
+    st = C.c_int32(-1)
+    stream = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    assert L.rcp_selftest_wait_timeout(None, 2000, stream) == 0
+    assert L.rcp_gemv_w2a4_static_status(C.byref(st), stream) == 0
+    assert st.value == 3, "the wait must have given up and said so"
+    words, lut, xq, scale = _inputs(300, 1024, 128, 2, seed=11)
+    y = rcp.rcp_gemv_w2a4_static(words, lut, xq, scale)
+    ws = rcp.make_workspace(2, 300, 1024, DEV)
+    assert torch.equal(y.view(torch.int16), rcp.rcp_gemv_w2a4(words, lut, xq, scale, workspace=ws).view(torch.int16))
+    assert L.rcp_gemv_w2a4_static_status(C.byref(st), stream) == 0
+    assert st.value == 0
+    assert L.rcp_selftest_wait_timeout(None, 0, stream) == -2
