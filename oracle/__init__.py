@@ -250,6 +250,91 @@ def ldp_export(w_f16_bits, sb, sg, s1, s2, G):
     return dict(codes=codes, lut=lut)
 
 
+def pack_weights3(codes):
+    """3-bit codes u8 [N][K] -> (words2 uint32 [N][K/16], words1 uint32 [N][K/32])."""
+    codes = _c(codes, np.uint8)
+    N, K = codes.shape
+    w2 = np.empty((N, K // 16), dtype=np.uint32)
+    w1 = np.empty((N, K // 32), dtype=np.uint32)
+    rc = lib().orc_pack_weights3(_p(codes), C.c_int(N), C.c_int(K), _p(w2), _p(w1))
+    if rc:
+        raise ValueError(f"orc_pack_weights3 failed: {rc}")
+    return w2, w1
+
+
+def unpack_weights3(words2, words1):
+    w2 = _c(words2, np.uint32)
+    w1 = _c(words1, np.uint32)
+    N, W = w2.shape
+    codes = np.empty((N, W * 16), dtype=np.uint8)
+    lib().orc_unpack_weights3(_p(w2), _p(w1), C.c_int(N), C.c_int(W * 16), _p(codes))
+    return codes
+
+
+def gemv_w3a4(words2, words1, lut_bits, xq, scale_bits, G=None):
+    """W3A4 GEMV. lut uint16 [N][K/G][8] (or [N][8] with G None = one grid per row).
+    Returns dict(S int32 [M][N][K/G][8], y float64 [M][N], tol float64 [M][N])."""
+    w2 = _c(words2, np.uint32)
+    w1 = _c(words1, np.uint32)
+    lut = _c(lut_bits, np.uint16)
+    xq = _c(xq, np.uint8)
+    scale = _c(scale_bits, np.uint16)
+    N, W = w2.shape
+    K = W * 16
+    M = xq.shape[0]
+    if G is None:
+        G = K
+    NG = K // G
+    lut = lut.reshape(N, NG, 8)
+    assert xq.shape == (M, K // 2) and w1.shape == (N, K // 32) and scale.shape == (M,)
+    S = np.empty((M, N, NG, 8), dtype=np.int32)
+    y = np.empty((M, N), dtype=np.float64)
+    tol = np.empty((M, N), dtype=np.float64)
+    rc = lib().orc_gemv_w3a4(_p(w2), _p(w1), _p(lut), _p(xq), _p(scale), C.c_int(M), C.c_int(N), C.c_int(K), C.c_int(G),
+                             _p(S), _p(y), _p(tol))
+    if rc:
+        raise ValueError(f"orc_gemv_w3a4 failed: {rc}")
+    return dict(S=S, y=y, tol=tol)
+
+
+def gemv_w3a4_direct_int(words2, words1, lut_bits, xq, G=None):
+    w2 = _c(words2, np.uint32)
+    w1 = _c(words1, np.uint32)
+    lut = _c(lut_bits, np.uint16)
+    xq = _c(xq, np.uint8)
+    N, W = w2.shape
+    K = W * 16
+    M = xq.shape[0]
+    if G is None:
+        G = K
+    acc = np.empty((M, N), dtype=np.int64)
+    rc = lib().orc_gemv_w3a4_direct_int(_p(w2), _p(w1), _p(lut), _p(xq), C.c_int(M), C.c_int(N), C.c_int(K), C.c_int(G),
+                                        _p(acc))
+    if rc:
+        raise ValueError(f"orc_gemv_w3a4_direct_int failed: {rc}")
+    return acc
+
+
+def nf3_export(w_f16_bits, sb, sg, s1, table, zero_index, G):
+    """3-bit export with a learnable centre. w uint16 [N][K]; sb, sg, s1 float32 [N][K/G]; table float32 [8]
+    ascending with table[zero_index] == 0. Returns dict(codes u8 [N][K], lut uint16 [N][K/G][8])."""
+    w = _c(w_f16_bits, np.uint16)
+    N, K = w.shape
+    assert K % G == 0
+    arrs = [_c(a, np.float32) for a in (sb, sg, s1)]
+    for a in arrs:
+        assert a.shape == (N, K // G)
+    t = _c(table, np.float32)
+    assert t.shape == (8,)
+    codes = np.empty((N, K), dtype=np.uint8)
+    lut = np.empty((N, K // G, 8), dtype=np.uint16)
+    rc = lib().orc_nf3_export(_p(w), _p(arrs[0]), _p(arrs[1]), _p(arrs[2]), _p(t), C.c_int(int(zero_index)), C.c_int(N),
+                              C.c_int(K), C.c_int(G), _p(codes), _p(lut))
+    if rc:
+        raise ValueError(f"orc_nf3_export failed: {rc}")
+    return dict(codes=codes, lut=lut)
+
+
 def gemv_w2a16(words, lut_bits, x_f16_bits):
     """Weight-only GEMV by its definition. Returns dict(y float64 [M][N], labsx float64 [M][N], labs float64 [N])."""
     words = _c(words, np.uint32)

@@ -32,6 +32,10 @@
 // activations (exactly for elements within 2^-11 of the token's maximum, to half a unit otherwise)
 // and a hand-written case. Per-code sums of 8-bit planes: equal to the W2A4 oracle's S on int4 planes, a
 // pure-Python loop, sum_c S_c == sum_k a_k.
+// 3-bit weights: packing round trip and hand-written words; GEMV by a pure-Python loop; per-code form ==
+// direct form as exact integers; sum_c S_c == sum_k q_k; a grid with equal levels for codes c and c + 4
+// == the W2A4 oracle on the low two bits; planted index mistakes. NF3 export: hand-worked unit, zero-centred
+// symmetric case == nearest level of the table scaled by the absmax, levels at the range ends and the centre.
 // fp16 output y: the paper prints no worked numeric GEMV example, so y is pinned only by the
 // mathematical identities above, not by a printed value.
 #include <cstdint>
@@ -535,6 +539,188 @@ int orc_ldp_export(const uint16_t* w_f16, const float* sb, const float* sg, cons
           volatile float d = v - lo;
           volatile float x = d / h;
           code = (x >= t1) + (x >= t2) + (x >= t3);
+        }
+        codes[(size_t)n * K + (size_t)j * G + k] = (uint8_t)code;
+      }
+    }
+  return 0;
+}
+
+// ---------------------------------------------------------------------------------------
+// 3-bit weights (Section 4.3, paragraph "Application of LDP on NF3 format"; Table "memory", W3
+// column). The same look-up-table GEMV with eight levels per quantization unit instead of four.
+//
+// Packing. A code c in 0..7 is split into its low two bits, stored exactly like a 2-bit code
+// (words2 [N][K/16], code 16w+j in bits [2j, 2j+1]), and its top bit, stored in a bit plane of
+// its own: words1 [N][K/32], where word v covers the codes 32v .. 32v+31 and holds the top bit
+// of code 32v + i in bit 2i and of code 32v + 16 + i in bit 2i+1 (i = 0..15). Three bits per
+// code in all. (The paper prints no W3 layout; this one is this implementation's.)
+// ---------------------------------------------------------------------------------------
+int orc_pack_weights3(const uint8_t* codes, int N, int K, uint32_t* words2, uint32_t* words1) {
+  if (N < 1 || K < 32 || K % 32) return -1;
+  for (int n = 0; n < N; n++) {
+    for (int w = 0; w < K / 16; w++) {
+      uint32_t word = 0;
+      for (int j = 0; j < 16; j++) {
+        const uint8_t c = codes[(size_t)n * K + 16 * w + j];
+        if (c > 7) return -4;
+        word |= (uint32_t)(c & 3u) << (2 * j);
+      }
+      words2[(size_t)n * (K / 16) + w] = word;
+    }
+    for (int v = 0; v < K / 32; v++) {
+      uint32_t word = 0;
+      for (int i = 0; i < 16; i++) {
+        word |= (uint32_t)((codes[(size_t)n * K + 32 * v + i] >> 2) & 1u) << (2 * i);
+        word |= (uint32_t)((codes[(size_t)n * K + 32 * v + 16 + i] >> 2) & 1u) << (2 * i + 1);
+      }
+      words1[(size_t)n * (K / 32) + v] = word;
+    }
+  }
+  return 0;
+}
+
+// Inverse of the packing, written independently of it: code k of a row from its two words.
+void orc_unpack_weights3(const uint32_t* words2, const uint32_t* words1, int N, int K, uint8_t* codes) {
+  for (int n = 0; n < N; n++)
+    for (int k = 0; k < K; k++) {
+      const uint32_t lo2 = (words2[(size_t)n * (K / 16) + k / 16] >> (2 * (k % 16))) & 3u;
+      const int r = k % 32;                                  // place inside the 32 codes of a plane word
+      const int bit = (r < 16) ? 2 * r : 2 * (r - 16) + 1;
+      const uint32_t top = (words1[(size_t)n * (K / 32) + k / 32] >> bit) & 1u;
+      codes[(size_t)n * K + k] = (uint8_t)(lo2 | (top << 2));
+    }
+}
+
+// W3A4 look-up-table GEMV, one eight-entry grid per group of G weights of a row (G = K: one per row).
+//   S_c[m][n][j] = sum over k in group j with code[n][k] == c of q[m][k]          (exact integers)
+//   y_ref        = s_m * sum_j sum_c LUT[n][j][c] * S_c[m][n][j]                   (double)
+//   tol          = 2e-3 * ( s_m * sum_j sum_c |LUT[n][j][c]| * |S_c| ) + 1e-5
+// S int32 [M][N][K/G][8] (may be NULL). Returns 0; -1 bad shape.
+int orc_gemv_w3a4(const uint32_t* words2, const uint32_t* words1, const uint16_t* lut_f16, const uint8_t* xq,
+                  const uint16_t* scale_f16, int M, int N, int K, int G, int32_t* S, double* y_ref, double* tol) {
+  if (M < 1 || N < 1 || K < 32 || K % 32 || G < 1 || K % G) return -1;
+  const int NG = K / G;
+  uint8_t* codes = (uint8_t*)std::malloc((size_t)K);
+  int8_t* q = (int8_t*)std::malloc((size_t)M * K);
+  orc_unpack_act(xq, (size_t)M * (K / 2), q);
+  for (int n = 0; n < N; n++) {
+    orc_unpack_weights3(words2 + (size_t)n * (K / 16), words1 + (size_t)n * (K / 32), 1, K, codes);
+    for (int m = 0; m < M; m++) {
+      const double s = (double)orc_f16_to_f32(scale_f16[m]);
+      double acc = 0.0, mag = 0.0;
+      for (int j = 0; j < NG; j++) {
+        long long Sc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        for (int k = j * G; k < (j + 1) * G; k++) Sc[codes[k]] += (long long)q[(size_t)m * K + k];
+        for (int c = 0; c < 8; c++) {
+          const double L = (double)orc_f16_to_f32(lut_f16[((size_t)n * NG + j) * 8 + c]);
+          if (S) S[(((size_t)m * N + n) * NG + j) * 8 + c] = (int32_t)Sc[c];
+          acc += L * (double)Sc[c];
+          mag += std::fabs(L) * std::fabs((double)Sc[c]);
+        }
+      }
+      y_ref[(size_t)m * N + n] = s * acc;
+      if (tol) tol[(size_t)m * N + n] = 2e-3 * (s * mag) + 1e-5;
+    }
+  }
+  std::free(codes);
+  std::free(q);
+  return 0;
+}
+
+// Direct form of the same product with every fp16 level scaled by 2^24 (exact integers):
+// acc_int[m][n] = sum_k Lint[n][k / G][code[n][k]] * q[m][k]. For the check that the per-code form
+// and the direct form are the same number.
+int orc_gemv_w3a4_direct_int(const uint32_t* words2, const uint32_t* words1, const uint16_t* lut_f16,
+                             const uint8_t* xq, int M, int N, int K, int G, long long* acc_int) {
+  if (M < 1 || N < 1 || K < 32 || K % 32 || G < 1 || K % G) return -1;
+  const int NG = K / G;
+  uint8_t* codes = (uint8_t*)std::malloc((size_t)K);
+  int8_t* q = (int8_t*)std::malloc((size_t)M * K);
+  orc_unpack_act(xq, (size_t)M * (K / 2), q);
+  for (int n = 0; n < N; n++) {
+    orc_unpack_weights3(words2 + (size_t)n * (K / 16), words1 + (size_t)n * (K / 32), 1, K, codes);
+    for (int m = 0; m < M; m++) {
+      long long acc = 0;
+      for (int k = 0; k < K; k++) {
+        const double L = (double)orc_f16_to_f32(lut_f16[((size_t)n * NG + k / G) * 8 + codes[k]]);
+        acc += (long long)std::ldexp(L, 24) * (long long)q[(size_t)m * K + k];
+      }
+      acc_int[(size_t)m * N + n] = acc;
+    }
+  }
+  std::free(codes);
+  std::free(q);
+  return 0;
+}
+
+// Export of a 3-bit layer (paragraph "Application of LDP on NF3 format", Eq. "nf3scales", Eq. "nf3").
+// Per quantization unit (G consecutive weights of a row), fp32 arithmetic, one rounding per operation:
+//   lo = sigma(beta) min(W), hi = sigma(gamma) max(W), h = hi - lo, W clipped to [lo, hi]
+//   c  = lo + h sigma(s_1)                       the learnable centre
+//   s_neg = |c - lo|,  s_pos = |hi - c|          Eq. "nf3scales"
+//   v  = (W - c) / s_pos if W > c, else (W - c) / s_neg            in [-1, 1]
+//   code = index of the level of the format nearest to v, searched among the levels of v's side
+//   level_i = c + T_i * (s_pos if T_i > 0 else s_neg), rounded to fp16
+// The format is a table T of eight ascending normalized levels with T[zero_index] == 0 (three bits:
+// the asymmetric normal-float format has three negative levels, zero, four positive ones, its end levels
+// -1 and 1). Readings: Eq. "nf3" prints a round-to-nearest of the normalized weight and the text says the
+// result is multiplied by the scale and offset by c, so "rounding" is to the nearest representable level
+// of the format, not to an integer; the paper takes the level values from the format's own publication
+// and prints none, so the table is an argument here; a weight exactly between two levels takes the lower
+// one; a weight equal to c belongs to the negative side ("otherwise"); h <= 0 gives code zero_index and
+// eight levels equal to lo. Sigmoids are inputs, as for the 2-bit export.
+// codes u8 [N][K], lut fp16 bits [N][K/G][8]. Returns 0; -1 bad shape; -2 bad table.
+int orc_nf3_export(const uint16_t* w_f16, const float* sb, const float* sg, const float* s1, const float* table,
+                   int zero_index, int N, int K, int G, uint8_t* codes, uint16_t* lut_f16) {
+  if (N < 1 || K < 1 || G < 1 || K % G) return -1;
+  if (zero_index < 0 || zero_index > 7 || table[zero_index] != 0.0f) return -2;
+  for (int i = 1; i < 8; i++) if (!(table[i] > table[i - 1])) return -2;
+  const int NG = K / G;
+  for (int n = 0; n < N; n++)
+    for (int j = 0; j < NG; j++) {
+      const uint16_t* w = w_f16 + (size_t)n * K + (size_t)j * G;
+      const size_t u = (size_t)n * NG + j;
+      float wmin = orc_f16_to_f32(w[0]), wmax = wmin;
+      for (int k = 1; k < G; k++) {
+        float v = orc_f16_to_f32(w[k]);
+        if (v < wmin) wmin = v;
+        if (v > wmax) wmax = v;
+      }
+      volatile float lo = sb[u] * wmin;
+      volatile float hi = sg[u] * wmax;
+      volatile float h = hi - lo;
+      volatile float off = h * s1[u];
+      volatile float c = lo + off;
+      volatile float dn = c - lo;
+      volatile float dp = hi - c;
+      const float s_neg = std::fabs((float)dn), s_pos = std::fabs((float)dp);
+      const bool ok = h > 0.0f;
+      for (int i = 0; i < 8; i++) {
+        volatile float prod = table[i] * (i > zero_index ? s_pos : s_neg);
+        volatile float level = c + prod;
+        lut_f16[u * 8 + i] = orc_f32_to_f16(ok ? (float)level : (float)lo);
+      }
+      for (int k = 0; k < G; k++) {
+        int code = zero_index;
+        if (ok) {
+          float v = orc_f16_to_f32(w[k]);
+          if (v < lo) v = lo;
+          if (v > hi) v = hi;
+          volatile float d = v - c;
+          const bool pos = v > c;
+          const float sc = pos ? s_pos : s_neg;
+          if (sc > 0.0f) {
+            volatile float x = d / sc;
+            const int first = pos ? zero_index : 0, last = pos ? 7 : zero_index;
+            code = first;
+            float best = std::fabs((float)x - table[first]);
+            for (int i = first + 1; i <= last; i++) {
+              volatile float diff = (float)x - table[i];
+              const float dist = std::fabs((float)diff);
+              if (dist < best) { best = dist; code = i; }   // strict: a tie keeps the lower level
+            }
+          }
         }
         codes[(size_t)n * K + (size_t)j * G + k] = (uint8_t)code;
       }
