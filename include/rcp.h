@@ -129,6 +129,38 @@ int rcp_gemv_w2a16_checked(const uint32_t* words, const void* lut_f16, const voi
                            void* y_f16, int8_t* digits, float* unit, void* workspace, int32_t* S_dbg, void* stream);
 
 /*
+ * 3-bit weights (Section 4.3, paragraph "Application of LDP on NF3 format": the paper's other weight setting,
+ * W3 in Table "memory" and Table "main_result"): the same look-up-table GEMV with eight levels per quantization
+ * unit. The paper prints no storage layout for it; this library's is: the low two bits of a code stored exactly
+ * like a 2-bit code, the top bit in a bit plane of its own,
+ *   words2  uint32 [N][K/16]  bits [2j, 2j+1] of word w = low two bits of code 16w + j;
+ *   words1  uint32 [N][K/32]  word v covers codes 32v .. 32v+31: bit 2i = top bit of code 32v + i,
+ *                             bit 2i+1 = top bit of code 32v + 16 + i (i = 0..15),
+ * three bits per code in all.
+ *
+ * rcp_pack_weights3: codes uint8 [N][K], each in 0..7 -> words2, words1. K % 64 == 0. Offline, like
+ * rcp_pack_weights: synchronizes the stream to report RCP_ERR_CODE (a code above 7).
+ */
+int rcp_pack_weights3(const uint8_t* codes, int N, int K, uint32_t* words2, uint32_t* words1, void* stream);
+
+/*
+ * W3A4 look-up-table GEMV (Section 4.4 with eight levels):
+ *   S_c[m][n][j] = sum over k in group j with code[n][k] == c of q[m][k],  c = 0..7     (exact integers)
+ *   y[m][n]      = fp16( scale[m] * sum_j sum_c lut[n][j][c] * S_c[m][n][j] )           (fp32 arithmetic)
+ *   lut_f16   DEVICE fp16, 16-byte aligned: [N][8] with group == 0 (one grid per output row), [N][K/128][8] with
+ *             group == 128 (one grid per group of 128 weights, the paper's group size); other sizes:
+ *             RCP_ERR_SHAPE.
+ *   xq, scale_f16, y_f16, M, N, K as for rcp_gemv_w2a4.
+ *   S_dbg     NULL in production. Otherwise int32 [M][N][8] ([M][N][K/128][8]) receives S_c from the checked
+ *             instantiation of the same kernel.
+ * The integer sums are exact (seven sums of q over products of code bits plus the total, turned into the
+ * eight S_c by inclusion and exclusion). One token per launch, M launches. Never synchronizes.
+ */
+int rcp_gemv_w3a4(const uint32_t* words2, const uint32_t* words1, const void* lut_f16, int group,
+                  const uint8_t* xq, const void* scale_f16, int M, int N, int K, void* y_f16,
+                  int32_t* S_dbg, void* stream);
+
+/*
  * Bytes of caller-provided scratch rcp_gemv_w2a4 needs for this shape (0 on bad shapes). The scratch
  * holds a status word that a kernel sets if one of its bounded waits ever gives up (0 = fine). It
  * must be zero-filled once after allocation; every successful call leaves it zero-filled, so one

@@ -65,6 +65,10 @@ def lib():
         L.rcp_gemv_w2a4_static.argtypes = [vp, vp, vp, vp, i, i, i, vp, vp]
         L.rcp_gemv_w2a16.restype = i
         L.rcp_gemv_w2a16.argtypes = [vp, vp, vp, i, i, i, vp, vp, vp, vp, vp]
+        L.rcp_pack_weights3.restype = i
+        L.rcp_pack_weights3.argtypes = [vp, i, i, vp, vp, vp]
+        L.rcp_gemv_w3a4.restype = i
+        L.rcp_gemv_w3a4.argtypes = [vp, vp, vp, i, vp, vp, i, i, i, vp, vp, vp]
         L.rcp_gemv_w2a4_static_status.restype = i
         L.rcp_gemv_w2a4_static_status.argtypes = [vp, vp]
         L.rcp_selftest_wait_timeout.restype = i
@@ -234,6 +238,42 @@ def rcp_gemv_w2a16(words, lut, x, y=None, digits=None, unit=None, workspace=None
         _check("rcp_gemv_w2a16",
                lib().rcp_gemv_w2a16_checked(_ptr(words), _ptr(lut), _ptr(x), M, N, K, _ptr(y), _ptr(digits), _ptr(unit),
                                             _ptr(workspace), _ptr(S_dbg), _stream(words)))
+    return y
+
+
+def rcp_pack_weights3(codes: torch.Tensor):
+    """3-bit codes uint8 [N][K] in {0..7} -> (words2 int32 [N][K/16], words1 int32 [N][K/32])."""
+    _dev(codes, torch.uint8, "codes")
+    N, K = codes.shape
+    words2 = torch.empty((N, K // 16), dtype=torch.int32, device=codes.device)
+    words1 = torch.empty((N, K // 32), dtype=torch.int32, device=codes.device)
+    with _on(codes):
+        _check("rcp_pack_weights3",
+               lib().rcp_pack_weights3(_ptr(codes), N, K, _ptr(words2), _ptr(words1), _stream(codes)))
+    return words2, words1
+
+
+def rcp_gemv_w3a4(words2, words1, lut, xq, scale, group=0, y=None, S_dbg=None):
+    """W3A4 GEMV: words2 int32 [N][K/16], words1 int32 [N][K/32], lut fp16 [N][8] (group=0) or [N][K/128][8]
+    (group=128), xq uint8 [M][K/2], scale fp16 [M] -> y fp16 [M][N]."""
+    _dev(words2, torch.int32, "words2")
+    _dev(words1, torch.int32, "words1")
+    _dev(lut, torch.float16, "lut")
+    _dev(xq, torch.uint8, "xq")
+    _dev(scale, torch.float16, "scale")
+    N, W = words2.shape
+    K = W * 16
+    M = xq.shape[0]
+    group = int(group)
+    want = (N, 8) if group == 0 else (N, K // max(group, 1), 8)
+    if words1.shape != (N, K // 32) or xq.shape != (M, K // 2) or tuple(lut.shape) != want or scale.shape != (M,):
+        raise ValueError("shape mismatch between words2, words1, lut, group, xq and scale")
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.float16, device=words2.device)
+    with _on(words2):
+        _check("rcp_gemv_w3a4",
+               lib().rcp_gemv_w3a4(_ptr(words2), _ptr(words1), _ptr(lut), group, _ptr(xq), _ptr(scale), M, N, K, _ptr(y),
+                                   _ptr(S_dbg), _stream(words2)))
     return y
 
 

@@ -11,6 +11,7 @@
 #include "common.cuh"
 #include "gemv_simple.cuh"
 #include "gemv_stream.cuh"
+#include "gemv_w3.cuh"
 #include "ldp_export.cuh"
 #include "split_act16.cuh"
 #include "pack.cuh"
@@ -440,6 +441,26 @@ int static_scratch_address(void** out) {
   return RCP_OK;
 }
 
+template <bool GRP, bool SDBG>
+int launch_w3(const rcp::W3Params& wp, int grid, size_t smem, cudaStream_t st) {
+  static std::mutex mu;
+  static bool attr_set[kMaxDevices] = {};
+  auto kern = rcp::gemv_w3a4_kernel<GRP, SDBG>;
+  int dev = 0;
+  RCP_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return RCP_ERR_LIMIT;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (!attr_set[dev]) {
+      RCP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, rcp::kMaxK + 128));
+      attr_set[dev] = true;
+    }
+  }
+  kern<<<grid, rcp::kW3Threads, smem, st>>>(wp);
+  RCP_CUDA(cudaGetLastError());
+  return RCP_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -479,6 +500,55 @@ int rcp_pack_weights(const uint8_t* codes, int N, int K, uint32_t* words, void* 
   RCP_CUDA(cudaMemcpyAsync(&h_bad, bad, sizeof(int), cudaMemcpyDeviceToHost, st));
   RCP_CUDA(cudaStreamSynchronize(st));
   return h_bad ? RCP_ERR_CODE : RCP_OK;
+}
+
+int rcp_pack_weights3(const uint8_t* codes, int N, int K, uint32_t* words2, uint32_t* words1, void* stream) {
+  if (!codes || !words2 || !words1) return RCP_ERR_NULL;
+  if (N < 1 || !k_ok(K)) return RCP_ERR_SHAPE;
+  if (!aligned16(codes) || !aligned16(words2) || !aligned16(words1)) return RCP_ERR_ALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int* bad = nullptr;
+  RCP_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&bad), g_pack_bad));
+  bad += g_pack_next.fetch_add(1) % kPackSlots;
+  RCP_CUDA(cudaMemsetAsync(bad, 0, sizeof(int), st));
+  const size_t nplane = (size_t)N * (K / 32);
+  const int block = 256;
+  const int grid = (int)std::min<size_t>((nplane + block - 1) / block, (size_t)sm_count() * 32);
+  rcp::pack_weights3_kernel<<<grid, block, 0, st>>>(reinterpret_cast<const uint4*>(codes), nplane, words2, words1, bad);
+  RCP_CUDA(cudaGetLastError());
+  int h_bad = 0;
+  RCP_CUDA(cudaMemcpyAsync(&h_bad, bad, sizeof(int), cudaMemcpyDeviceToHost, st));
+  RCP_CUDA(cudaStreamSynchronize(st));
+  return h_bad ? RCP_ERR_CODE : RCP_OK;
+}
+
+int rcp_gemv_w3a4(const uint32_t* words2, const uint32_t* words1, const void* lut_f16, int group, const uint8_t* xq,
+                  const void* scale_f16, int M, int N, int K, void* y_f16, int32_t* S_dbg, void* stream) {
+  if (!words2 || !words1 || !lut_f16 || !xq || !scale_f16 || !y_f16) return RCP_ERR_NULL;
+  if (M < 1 || M > rcp::kMaxTokens || N < 1 || !k_ok(K)) return RCP_ERR_SHAPE;
+  if (group != 0 && (group != 128 || K % 128)) return RCP_ERR_SHAPE;
+  if (!aligned16(words2) || !aligned16(words1) || !aligned16(lut_f16) || !aligned16(xq) || !aligned16(S_dbg) ||
+      (reinterpret_cast<uintptr_t>(y_f16) & 1u) || (reinterpret_cast<uintptr_t>(scale_f16) & 1u))
+    return RCP_ERR_ALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int ngrp = group ? K / 128 : 1;
+  const int grid = std::min((N + rcp::kW3Threads / 32 - 1) / (rcp::kW3Threads / 32), sm_count() * 4);
+  const size_t smem = (size_t)((K / 64 + 1) / 2) * 8 * 16;   // expanded activations: eight 16-byte slots per pair of units
+  for (int m = 0; m < M; m++) {   // one token per launch: the variant is tuned for decoding one token
+    rcp::W3Params wp;
+    wp.words2 = words2; wp.words1 = words1;
+    wp.lut = static_cast<const uint4*>(lut_f16);
+    wp.xq = xq + (size_t)m * (K / 2);
+    wp.scale = static_cast<const __half*>(scale_f16) + m;
+    wp.y = static_cast<__half*>(y_f16) + (size_t)m * N;
+    wp.S_out = S_dbg ? S_dbg + (size_t)m * N * ngrp * 8 : nullptr;
+    wp.N = N; wp.K = K;
+    int rc;
+    if (group) rc = S_dbg ? launch_w3<true, true>(wp, grid, smem, st) : launch_w3<true, false>(wp, grid, smem, st);
+    else rc = S_dbg ? launch_w3<false, true>(wp, grid, smem, st) : launch_w3<false, false>(wp, grid, smem, st);
+    if (rc != RCP_OK) return rc;
+  }
+  return RCP_OK;
 }
 
 int rcp_ldp_export(const void* w_f16, const float* sig_beta, const float* sig_gamma, const float* sig_s1,
