@@ -26,8 +26,8 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2502_15779_b200 import configs as cfgs  # noqa: E402
-from paper_2502_15779_b200 import synth  # noqa: E402
+from gen import configs as cfgs  # noqa: E402
+from gen import synth  # noqa: E402
 
 METRIC = "w2a4_decode_layer_hbm_gbs"
 UNIT = "GB/s"
@@ -40,6 +40,36 @@ def measured_peaks():
     if os.path.exists(path):
         return json.load(open(path)), "measured"
     return {"hbm_gbs": 6650.0}, "fallback"
+
+
+def source_sha():
+    """Hash of the CUDA sources: counters taken from an older kernel are not reported."""
+    import hashlib
+    h = hashlib.sha1()
+    d = os.path.join(ROOT, "paper_2502_15779_b200", "csrc")
+    for name in sorted(os.listdir(d)):
+        h.update(name.encode())
+        h.update(open(os.path.join(d, name), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def profiled_counters(key):
+    """Per-launch counters of the streaming kernel for this workload, as the profiling helper
+    (python -m paper_2502_15779_b200.ncu_counters) wrote them from an ncu capture: DRAM bytes and warp
+    instructions per launch. None when there is no capture for the key or the kernel sources changed since."""
+    path = os.path.join(ROOT, "profiles", "counters.txt")
+    if not os.path.exists(path):
+        return None
+    for ln in open(path):
+        f = ln.split()
+        if len(f) >= 2 and f[0] == key:
+            d = dict(zip(f[1::2], f[2::2]))
+            if d.get("source_sha") != source_sha():
+                return None
+            return {"dram_bytes_per_launch": float(d["dram_bytes_per_launch"]),
+                    "warp_instructions_per_launch": float(d["warp_instructions_per_launch"]),
+                    "launches": int(d["launches"])}
+    return None
 
 
 def f16_bits(t):
@@ -322,6 +352,28 @@ def per_shape_table(cfg, Ms, device, rcp, stream, variant, reps=3):
                 row.update({"w2a16_bytes": nbytes_a, "w2a16_us_per_call": round(us_a, 3),
                             "w2a16_gbs": round(nbytes_a / us_a / 1e3, 1)})
                 del ga
+            if M == 1:
+                # the 3-bit variant on the same shape (random codes: the timing does not depend on them)
+                w2 = [torch.randint(-2 ** 31, 2 ** 31 - 1, (L.N, L.K // 16), dtype=torch.int32, device=device)
+                      for _ in range(copies)]
+                w1 = [torch.randint(-2 ** 31, 2 ** 31 - 1, (L.N, L.K // 32), dtype=torch.int32, device=device)
+                      for _ in range(copies)]
+                lut8 = torch.sort(torch.randn(L.N, 8, device=device) * 0.02, dim=1).values.half()
+
+                def body_3():
+                    for i in range(launches):
+                        rcp.rcp_gemv_w3a4(w2[i % copies], w1[i % copies], lut8, xq, scale, y=y)
+                with torch.cuda.stream(stream):
+                    body_3()
+                stream.synchronize()
+                g3 = capture(body_3, stream)
+                g3.replay()
+                stream.synchronize()
+                us_3 = min(time_graph_replays([g3], [0], stream) for _ in range(reps)) * 1e3 / launches
+                nbytes_3 = cfgs.gemv_w3a4_bytes(M, L.N, L.K)
+                row.update({"w3a4_bytes": nbytes_3, "w3a4_us_per_call": round(us_3, 3),
+                            "w3a4_gbs": round(nbytes_3 / us_3 / 1e3, 1)})
+                del g3, w2, w1
             rows.append(row)
         del words, luts, base, luts_g, lut_g
         torch.cuda.empty_cache()
@@ -440,6 +492,15 @@ def main():
     if args.impl == "reference":
         run_reference(args, cfg, M)
         return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as a plain script: start the N replicas (one process per GPU) the same way a launcher would
+        import socket
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        sys.exit(subprocess.call(cmd))
 
     import paper_2502_15779_b200 as rcp
     rank = int(os.environ.get("RANK", "0"))
@@ -532,22 +593,18 @@ def main():
                               "frac": round(p_ach / peaks["hbm_gbs"], 4),
                               "note": "rcp_gemv_w2a4 launches alone, activations quantized beforehand"}
     del pgraphs
-    # Second bound: the kernel needs 249 warp instructions per KB of packed weights at one token (instruction
-    # mix counted by ncu, profiles/gemv_stream_llama2_7b_M1_full.md) and an SM issues at most four per clock.
-    if M == 1 and args.variant in ("auto", "dp4a") and clocks and clocks.get("sm_mhz"):
+    # Second bound: instruction issue. An SM issues at most four warp instructions per clock; the count per KB of
+    # packed weights comes from the ncu capture of this workload (none, or taken from older sources: not reported).
+    counters = profiled_counters(f"{cfg.key}_M{M}_{args.variant}")
+    if counters and clocks and clocks.get("sm_mhz"):
         sms = torch.cuda.get_device_properties(device).multi_processor_count
-        issue_gbs = 4.0 * sms * clocks["sm_mhz"] * 1e6 / 249.0 * 1024.0 / 1e9
-        roofline["issue_bound"] = {"warp_instructions_per_kb": 249, "peak": round(issue_gbs, 1), "unit": "GB/s",
+        per_kb = counters["warp_instructions_per_launch"] / (layer.weight_bytes() * args.steps / g_launches / 1024.0)
+        issue_gbs = 4.0 * sms * clocks["sm_mhz"] * 1e6 / per_kb * 1024.0 / 1e9
+        roofline["issue_bound"] = {"warp_instructions_per_kb": round(per_kb, 1), "peak": round(issue_gbs, 1), "unit": "GB/s",
                                    "frac": round(achieved / issue_gbs, 4),
-                                   "plain_gemv_frac": round(p_ach / issue_gbs, 4),
-                                   "note": "4 warp instructions per clock per SM at the sampled SM clock"}
-    # DRAM bytes per launch from the committed ncu summary (null when there is none for this workload)
-    prof = os.path.join(ROOT, "profiles", "dram_traffic.txt")
-    if os.path.exists(prof):
-        for ln in open(prof):
-            parts = ln.split()
-            if len(parts) == 2 and parts[0] == f"{cfg.key}_M{M}_{args.variant}":
-                roofline["traffic"] = int(parts[1])
+                                   "note": "4 warp instructions per clock per SM at the sampled SM clock; count from ncu"}
+    if counters:
+        roofline["traffic"] = int(counters["dram_bytes_per_launch"])
 
     # ---- end to end through the C ABI with host buffers
     xh = [layer.x[li].cpu().pin_memory() for li in range(len(layer.layers))]

@@ -72,3 +72,8 @@ def quant_bytes(M: int, K: int) -> int:
 def gemv_w2a16_bytes(M: int, N: int, K: int) -> int:
     """Algorithmic bytes of one weight-only GEMV call: packed codes + per-row LUT + fp16 activations + fp16 output."""
     return N * K // 4 + 8 * N + 2 * M * K + 2 * M * N
+
+
+def gemv_w3a4_bytes(M: int, N: int, K: int) -> int:
+    """Algorithmic bytes of one W3A4 GEMV call: 3-bit codes + eight fp16 levels per row + int4 activations + fp16 output."""
+    return 3 * N * K // 8 + 16 * N + M * K // 2 + 2 * M * N

@@ -89,10 +89,15 @@ int rcp_quantize_act(const void* x_f16, int M, int K, int had_block, float clip_
  *                    else in launches of eight at most; for one or two tokens the b0*b1
  *                    plane is computed with dp4a beside the tensor cores.
  *   RCP_GEMV_MMA_ONLY  as RCP_GEMV_MMA with all three planes on the tensor cores for every M.
+ *   RCP_GEMV_MMA_STREAM  the tensor-core kernel with the expanded activations streamed beside the weights: each
+ *                    ring stage carries the int8 activations of the chunks of K its boxes cover, written by a
+ *                    warp of its own ahead of the consumers. Nothing is expanded up front, K never has to be
+ *                    gone through in parts, and one launch takes up to sixteen tokens whatever K is.
  * The streaming kernel: persistent CTAs, weights through a TMA/mbarrier shared-memory ring, 16-row
  * groups owned by warps, no exchange between CTAs.
  */
-enum { RCP_GEMV_AUTO = 0, RCP_GEMV_SIMPLE = 1, RCP_GEMV_DP4A = 2, RCP_GEMV_MMA = 3, RCP_GEMV_MMA_ONLY = 4 };
+enum { RCP_GEMV_AUTO = 0, RCP_GEMV_SIMPLE = 1, RCP_GEMV_DP4A = 2, RCP_GEMV_MMA = 3, RCP_GEMV_MMA_ONLY = 4,
+       RCP_GEMV_MMA_STREAM = 5 };
 
 /*
  * Weight-only form of the LUT GEMV (Section 5, the W2-only setting of Table "W2_inference": the codes
@@ -175,7 +180,9 @@ size_t rcp_gemv_workspace_bytes(int M, int N, int K);
  *   out[4] 128-byte chunks per row, out[5] number of phases, then per phase five ints:
  *   groups per CTA at most, first group, groups in the phase, CTAs taking part, repetitions;
  *   and one last int: the parts of K one launch goes through one after the other (1 unless several tokens
- *   meet a K so long that their expanded activations do not fit in shared memory at once).
+ *   meet a K so long that their expanded activations do not fit in shared memory at once; rcp_gemv_w2a4 then
+ *   runs the RCP_GEMV_MMA_STREAM form, one pass over K, where that form's ring fits, and the weight-only form
+ *   goes through K in parts).
  * (A group is 16 consecutive output rows; see the kernel's description.) Returns the number of
  * ints the full description has, or a negative status.
  */

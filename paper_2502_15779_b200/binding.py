@@ -14,8 +14,9 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 # RCP_W2A4_LIB names another build of the same library (the tests use it for the guarded build)
 LIB_PATH = os.environ.get("RCP_W2A4_LIB") or os.path.join(_HERE, "librcp_w2a4.so")
 
-GEMV_AUTO, GEMV_SIMPLE, GEMV_DP4A, GEMV_MMA, GEMV_MMA_ONLY = 0, 1, 2, 3, 4
-VARIANTS = {"auto": GEMV_AUTO, "simple": GEMV_SIMPLE, "dp4a": GEMV_DP4A, "mma": GEMV_MMA, "mma_only": GEMV_MMA_ONLY}
+GEMV_AUTO, GEMV_SIMPLE, GEMV_DP4A, GEMV_MMA, GEMV_MMA_ONLY, GEMV_MMA_STREAM = 0, 1, 2, 3, 4, 5
+VARIANTS = {"auto": GEMV_AUTO, "simple": GEMV_SIMPLE, "dp4a": GEMV_DP4A, "mma": GEMV_MMA, "mma_only": GEMV_MMA_ONLY,
+            "mma_stream": GEMV_MMA_STREAM}
 
 _lib = None
 

@@ -71,6 +71,7 @@ constexpr int kChunkWords = 32;                   // 128 bytes of K per row per 
 constexpr int kGroupBytes = 16 * kChunkWords * 4; // one group's rows in a box: 2 KB
 constexpr int kStageBytes = kTileRows * kChunkWords * 4;
 constexpr int kMaxStages = 8;
+constexpr int kExpWarps = 4;                      // SB: warps that expand the activations of the stages (one per scheduler)
 constexpr uint32_t kSpinLimit = 1u << 22;         // bounded waits: give up, flag the error and exit
 
 enum GemvMode { kModeMma = 0, kModeHybrid = 1, kModeDp4a = 2 };
@@ -118,6 +119,7 @@ struct GemvParams {
   int ramp_clk;         // clocks between the first `stages` requests of a CTA
   int off_bar, off_T0c, off_scale, off_red, off_bs;   // shared-memory byte offsets from the aligned base
   int bs_bytes, red_bytes, part_bytes;                // sizes of the areas at off_bs, off_red, off_part (guarded build)
+  int stage_stride;     // bytes from one ring stage to the next: kStageBytes, plus the stage's activation area (SB)
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -245,8 +247,15 @@ __global__ void wait_timeout_kernel(int32_t* status, uint32_t polls) {
 // SDBG  checked instantiation: the same kernel also stores the integer sums S_0..S_3 it finishes its rows
 //       from (p.S_out), so that a test can compare them with a reference bit for bit. The production
 //       instantiations (SDBG false) contain none of this.
-template <int MODE, int MTOK, bool GRP, bool FQ = false, bool A16 = false, bool SPLIT = false, bool SDBG = false>
-__global__ void __launch_bounds__(kGThreads, 1)
+// SB    activations streamed with the weights (tensor-core kernels of the per-row grid): nothing is expanded up
+//       front. Every ring stage carries, behind its boxes of weights, the expanded activations of the chunks
+//       those boxes cover (tokens x 512 bytes per chunk), written by one more warp that runs ahead of the
+//       consumers like the producer does. The token count and K then no longer meet in shared memory: no K in
+//       parts, up to sixteen tokens for any K, and the expansion (2 us at eight tokens of 8192) leaves the
+//       critical path. The host keeps (warps sharing a group) x tokens at 32 or less per stage.
+template <int MODE, int MTOK, bool GRP, bool FQ = false, bool A16 = false, bool SPLIT = false, bool SDBG = false,
+          bool SB = false>
+__global__ void __launch_bounds__(SB ? kGThreads + 32 * kExpWarps : kGThreads, 1)
 gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -265,6 +274,9 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   // A form of its own, so that the kernels that never need it keep their code.
   constexpr bool kSplit = SPLIT;
   static_assert(!SPLIT || (MODE == kModeMma && MTOK == 0 && !GRP && !FQ), "K in parts: eight-column tensor-core kernels, per-row grid");
+  static_assert(!SB || (MODE == kModeMma && !GRP && !FQ && !A16 && !SPLIT), "streamed activations: tensor-core kernels, per-row grid");
+  constexpr int kThreads = SB ? kGThreads + 32 * kExpWarps : kGThreads;   // consumers, producer warp, and the expander warps (SB)
+  const uint32_t stage_stride = SB ? (uint32_t)p.stage_stride : (uint32_t)kStageBytes;
   const int nsplit = kSplit ? p.nsplit : 1;
   const int ncol = M;
   const int stages = p.stages;
@@ -284,8 +296,8 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   auto ck_fail = [&](int site) { if (p.status) atomicMax(p.status, 16 + site); };
 #endif
   // areas of the layout (used by the guarded build's checks only)
-  const uint32_t ring_lo = base, ring_hi = base + (uint32_t)stages * kStageBytes;
-  const uint32_t bs_lo = base + (uint32_t)p.off_bs, bs_hi = bs_lo + (uint32_t)p.bs_bytes;
+  const uint32_t ring_lo = base, ring_hi = base + (uint32_t)stages * stage_stride;
+  const uint32_t bs_lo = SB ? ring_lo : base + (uint32_t)p.off_bs, bs_hi = SB ? ring_hi : bs_lo + (uint32_t)p.bs_bytes;
   (void)ring_lo; (void)ring_hi; (void)bs_lo; (void)bs_hi;
 
   const int b = blockIdx.x;
@@ -296,7 +308,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   // requests go out without waiting for anybody. The consumer warps wait for the announcement.
   if (warp != kCWarps) {
     if (tid < kMaxTokens) s_T0tot[tid] = 0;
-    asm volatile("bar.sync 3, %0;" ::"n"(kGThreads) : "memory");
+    asm volatile("bar.sync 3, %0;" ::"n"(kThreads) : "memory");
   }
 
   // ------------------------------------------------------------------ producer
@@ -305,11 +317,12 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   // other warps again.
   if (warp == kCWarps) {
     if (lane == 0) {
-      for (int s = 0; s < stages; s++) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, kCWarps); }
+      // a stage is full when its weights have landed (one arrival with the byte count) and, SB, the expander has arrived
+      for (int s = 0; s < stages; s++) { mbar_init(full0 + 8 * s, SB ? 1 + kExpWarps : 1); mbar_init(empty0 + 8 * s, kCWarps); }
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncwarp();
-    asm volatile("bar.arrive 3, %0;" ::"n"(kGThreads) : "memory");
+    asm volatile("bar.arrive 3, %0;" ::"n"(kThreads) : "memory");
     if (lane != 0) return;
     int slot = 0;
     uint32_t phase = 0;
@@ -342,7 +355,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
             const long long due = t_start + (long long)issued * p.ramp_clk;
             while (clock64() < due) { }
           }
-          const uint32_t bar = full0 + 8 * slot, dst = base + (uint32_t)slot * kStageBytes;
+          const uint32_t bar = full0 + 8 * slot, dst = base + (uint32_t)slot * stage_stride;
           const int nbox = kSplit ? max(0, min(KS, nch - s * KS)) : min(KS, nch - s * KS);   // a short last part can leave a stage empty
           mbar_expect_tx(bar, (uint32_t)nbox * box);
           for (int j = 0; j < nbox; j++) {
@@ -358,6 +371,97 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     }
     }
     return;
+  }
+
+  // ------------------------------------------------------------------ expander (SB)
+  // One warp walks the same sequence of stages as the producer and fills each stage's activation area:
+  // for every box of the stage (a chunk of K) and every token, the chunk's 512 int4 activations as int8 in the
+  // B-fragment order the consumers read. It waits for a slot to be released like the producer does.
+  if constexpr (SB) {
+    if (warp > kCWarps) {
+      const int ew = warp - (kCWarps + 1);   // which of the expander warps
+      asm volatile("griddepcontrol.wait;" ::: "memory");   // xq may belong to the kernel before this one
+      int slot = 0;
+      uint32_t phase = 0;
+      int issued = 0;
+      const int W = p.K / 16;
+      for (int pi = 0; pi < p.nphase; pi++) {
+        const GemvPhase ph = p.phase[pi];
+        if (b >= ph.ncta) continue;
+        const int KS = ph.ks, SA = ph.sa;
+        for (int rp = 0; rp < ph.reps; rp++) {
+          for (int s = 0; s < SA; s++) {
+            // The stage's work is (boxes x tokens x 16) units of two words, dealt to the lanes four at a time.
+            // The packed activations of a batch are fetched (global memory, L2) before the wait for the slot and
+            // before the previous batch is stored: the latency stays off the path.
+            const int nbox = min(KS, p.nchunk - s * KS);
+            const int per_box = M * 16, total = nbox * per_box;
+            const uint32_t inv_box = ((1u << 20) + per_box - 1) / per_box;   // v / per_box == (v * inv_box) >> 20 for v < 512
+            constexpr int kLaneStep = 32 * kExpWarps;
+            auto fetch = [&](int v0, uint4 (&x)[4]) {
+#pragma unroll
+              for (int r = 0; r < 4; r++) {
+                const int v = v0 + kLaneStep * r;
+                x[r] = make_uint4(0, 0, 0, 0);
+                if (v < total) {
+                  const int j = (int)(((uint32_t)v * inv_box) >> 20), w = v - j * per_box;
+                  const int col = w >> 4, lo = w & 3, hi = (w >> 2) & 3;
+                  const int wx = (s * KS + j) * kChunkWords + 8 * lo + 2 * hi;   // first of the unit's two words
+                  if (wx < W) x[r] = __ldg(reinterpret_cast<const uint4*>(p.xq + (size_t)col * (p.K / 2)) + (wx >> 1));
+                }
+              }
+            };
+            uint4 xa[4];
+            fetch(ew * 32 + lane, xa);
+            if (issued >= stages) {
+              if (!mbar_wait(empty0 + 8 * slot, phase ^ 1u)) {
+                if (lane == 0 && p.status) atomicExch(p.status, 4);
+                return;
+              }
+            }
+            uint8_t* const sb = gen + (size_t)slot * stage_stride + kStageBytes;
+            for (int v0 = ew * 32 + lane; v0 < total; v0 += 4 * kLaneStep) {
+              uint4 xn[4];
+              if (v0 + 4 * kLaneStep < total) fetch(v0 + 4 * kLaneStep, xn);
+#pragma unroll
+              for (int r = 0; r < 4; r++) {
+                const int v = v0 + kLaneStep * r;
+                if (v < total) {
+                  const int j = (int)(((uint32_t)v * inv_box) >> 20), w = v - j * per_box;
+                  const int col = w >> 4, lo = w & 3, hi = (w >> 2) & 3;
+                  const uint4 x = xa[r];
+                  uint32_t q[4][2];
+#pragma unroll
+                  for (int ww = 0; ww < 2; ww++) {
+                    const uint32_t lo32 = ww ? x.z : x.x, hi32 = ww ? x.w : x.y;
+                    uint32_t n4[4] = {lo32 & 0x0F0F0F0Fu, (lo32 >> 4) & 0x0F0F0F0Fu, hi32 & 0x0F0F0F0Fu, (hi32 >> 4) & 0x0F0F0F0Fu};
+#pragma unroll
+                    for (int h = 0; h < 4; h++) n4[h] |= (n4[h] & 0x08080808u) * 0x1Eu;   // sign-extend the nibbles
+                    const uint32_t e0 = __byte_perm(n4[0], n4[2], 0x6420), e2 = __byte_perm(n4[0], n4[2], 0x7531);
+                    q[0][ww] = (e0 << 2) & 0xFCFCFCFCu;
+                    q[1][ww] = __byte_perm(n4[1], n4[3], 0x6420);
+                    q[2][ww] = (e2 << 2) & 0xFCFCFCFCu;
+                    q[3][ww] = __byte_perm(n4[1], n4[3], 0x7531);
+                  }
+                  uint8_t* dst = sb + ((size_t)(((j * 4 + hi) * 2) * ncol + col)) * 64 + lo * 16;
+                  if (RCP_CK(dst >= gen && dst + (size_t)ncol * 64 + 16 <= gen + (size_t)(slot + 1) * stage_stride, 13)) {
+                    *reinterpret_cast<uint4*>(dst) = make_uint4(q[0][0], q[0][1], q[1][0], q[1][1]);
+                    *reinterpret_cast<uint4*>(dst + (size_t)ncol * 64) = make_uint4(q[2][0], q[2][1], q[3][0], q[3][1]);
+                  }
+                }
+              }
+#pragma unroll
+              for (int r = 0; r < 4; r++) xa[r] = xn[r];
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(full0 + 8 * slot);   // release: the stores above are visible to whoever sees the phase complete
+            issued++;
+            if (++slot == stages) { slot = 0; phase ^= 1u; }
+          }
+        }
+      }
+      return;
+    }
   }
 
   // The packed weights and the LUT are constants of the layer; everything else (xq, scale, y) may
@@ -434,6 +538,29 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     }
     if constexpr (!GRP)
       for (int i = tid; i < 2 * 8 * 16 * M * 3; i += kCWarps * 32) s_red[i] = 0;
+  } else if constexpr (SB) {
+    // Streamed activations: only the sum of q per token is needed up front (S_0 = T0 - S_1 - S_2 - S_3).
+    const int nvec = p.K / 32;   // 16-byte vectors of packed activations per token
+    for (int col = 0; col < M; col++) {
+      int tsum = 0;
+      for (int i = tid; i < nvec; i += kCWarps * 32) {
+        const uint4 x = __ldg(reinterpret_cast<const uint4*>(p.xq + (size_t)col * (p.K / 2)) + i);
+        const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int h = 0; h < 4; h++) {
+          uint32_t e = xs[h] & 0x0F0F0F0Fu, o = (xs[h] >> 4) & 0x0F0F0F0Fu;
+          e |= (e & 0x08080808u) * 0x1Eu;
+          o |= (o & 0x08080808u) * 0x1Eu;
+          tsum = __dp4a((int)e, 0x01010101, tsum);
+          tsum = __dp4a((int)o, 0x01010101, tsum);
+        }
+      }
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) tsum += __shfl_xor_sync(0xffffffffu, tsum, d);
+      if (lane == 0) atomicAdd(&s_T0tot[col], tsum);
+    }
+    if (tid < M) s_scale[tid] = __half2float(p.scale[tid]);
+    for (int i = tid; i < 2 * 8 * 16 * M * 3; i += kCWarps * 32) s_red[i] = 0;
   } else
   // ------------------------------------------------------------------ activations (consumer warps)
   // One unit = (column, chunk, i, pr, t) = two words. The 16 units of a (column, chunk) are 16
@@ -673,9 +800,8 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   for (int tok = 0; tok < NTD; tok++) bD_lane[tok] = (uint32_t)(tok * 64 + t * 16);
 
   // 16 rows x 128 bytes of weights at shared address a_grp against the activations of one chunk
-  auto compute_chunk = [&](uint32_t a_grp, uint32_t b_chunk) {
+  auto compute_chunk = [&](uint32_t a_grp, uint32_t b_ptr) {   // b_ptr: the chunk's expanded activations
     const uint32_t a_ptr = a_grp;                          // 32-bit shared-memory addresses throughout
-    const uint32_t b_ptr = base + (uint32_t)p.off_bs + b_chunk;
 #pragma unroll
     for (int i = 0; i < 2; i++) {
       const uint4 U = RCP_LDS128(a_ptr + a_chunk[i], ring_lo, ring_hi, 4);
@@ -1081,7 +1207,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
             if constexpr (kRelabel) {
               compute_chunk_grp_mma(a_grp, b_chunk, ch, lg_cur, row_first);
             } else {
-              compute_chunk(a_grp, b_chunk);
+              compute_chunk(a_grp, base + (uint32_t)p.off_bs + b_chunk);
               flush_grp_dp4a(ch, lg_cur, row_first);
             }
           }
@@ -1098,7 +1224,14 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
           if (lane == 0 && p.status) atomicExch(p.status, 3);
           return;
         }
-        if (active && ch < nch) compute_chunk(base + (uint32_t)slot * kStageBytes + a_off, b_chunk);
+        if (active && ch < nch) {
+          if constexpr (SB) {
+            const uint32_t st = base + (uint32_t)slot * stage_stride;
+            compute_chunk(st + a_off, st + kStageBytes + (uint32_t)ks * chunk_stride);
+          } else {
+            compute_chunk(base + (uint32_t)slot * kStageBytes + a_off, base + (uint32_t)p.off_bs + b_chunk);
+          }
+        }
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + 8 * slot);   // this warp is done with the slot
         if (++slot == stages) { slot = 0; phase ^= 1u; }

@@ -7,7 +7,7 @@ import numpy as np
 import torch
 
 import paper_2502_15779_b200 as rcp
-from paper_2502_15779_b200 import synth
+from gen import synth
 
 DEV = "cuda:0"
 

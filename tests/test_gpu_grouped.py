@@ -8,8 +8,8 @@ import torch
 
 import oracle
 import paper_2502_15779_b200 as rcp
-from paper_2502_15779_b200 import synth
-from paper_2502_15779_b200.configs import CONFIGS
+from gen import synth
+from gen.configs import CONFIGS
 from helpers import f16_bits
 
 pytestmark = pytest.mark.gpu

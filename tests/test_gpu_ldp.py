@@ -6,7 +6,7 @@ import torch
 
 import oracle
 import paper_2502_15779_b200 as rcp
-from paper_2502_15779_b200 import synth
+from gen import synth
 from helpers import f16_bits
 
 pytestmark = pytest.mark.gpu

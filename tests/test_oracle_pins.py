@@ -10,7 +10,7 @@ import scipy.linalg
 import torch
 
 import oracle
-from paper_2502_15779_b200 import synth
+from gen import synth
 from helpers import f16_bits
 
 GOLD = os.path.join(os.path.dirname(__file__), "golden")

@@ -7,7 +7,7 @@ import numpy as np
 import scipy.stats
 
 import oracle
-from paper_2502_15779_b200 import synth
+from gen import synth
 from helpers import f16_bits
 
 GOLD = os.path.join(os.path.dirname(__file__), "golden")

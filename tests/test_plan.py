@@ -5,7 +5,7 @@ import ctypes as C
 import pytest
 
 from paper_2502_15779_b200 import build
-from paper_2502_15779_b200.configs import CONFIGS
+from gen.configs import CONFIGS
 
 
 @pytest.fixture(scope="module")
