@@ -472,7 +472,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2_70b", choices=list(cfgs.BY_KEY))
     ap.add_argument("--tokens", type=int, default=1)
-    ap.add_argument("--variant", default="auto", choices=["auto", "simple", "dp4a", "mma", "mma_only", "w2a16"],
+    ap.add_argument("--variant", default="auto", choices=["auto", "simple", "dp4a", "mma", "mma_only", "mma_stream", "w2a16"],
                     help="kernel variant of the W2A4 GEMV; w2a16 (only with --profile) runs the layer in the "
                          "weight-only form instead, for the ncu summaries")
     ap.add_argument("--no-table", action="store_true", help="skip the per-shape table of the other configs")
