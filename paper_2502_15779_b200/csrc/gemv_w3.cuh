@@ -141,42 +141,65 @@ __global__ void __launch_bounds__(kW3Threads) gemv_w3a4_kernel(const W3Params p)
   const float s = __half2float(p.scale[0]);
   const int ngrp = p.K / 128;
   const int warps = gridDim.x * (kW3Threads / 32);
-  for (int row = blockIdx.x * (kW3Threads / 32) + warp; row < p.N; row += warps) {
-    const uint4* w2 = reinterpret_cast<const uint4*>(p.words2 + (size_t)row * W);
-    const uint2* w1 = reinterpret_cast<const uint2*>(p.words1 + (size_t)row * (W / 2));
+  // The weights of a lane step (two units: a 16-byte and an 8-byte load each) are fetched one step ahead, across
+  // the end of a row as well, so that the loads of the next step are in flight while this one is computed.
+  const int nit = (nunit + 63) / 64;                         // lane steps per row
+  const int row_first = blockIdx.x * (kW3Threads / 32) + warp;
+  auto fetch = [&](int row, int it, uint4 (&a)[2], uint2 (&z)[2]) {
+#pragma unroll
+    for (int h = 0; h < 2; h++) {
+      const int u = 2 * lane + 64 * it + h;
+      a[h] = make_uint4(0, 0, 0, 0);
+      z[h] = make_uint2(0, 0);
+      if (row < p.N && u < nunit) {
+        a[h] = __ldg(reinterpret_cast<const uint4*>(p.words2 + (size_t)row * W) + u);
+        z[h] = __ldg(reinterpret_cast<const uint2*>(p.words1 + (size_t)row * (W / 2)) + u);
+      }
+    }
+  };
+  uint4 an[2];
+  uint2 zn[2];
+  fetch(row_first, 0, an, zn);
+  for (int row = row_first; row < p.N; row += warps) {
     int acc[7][2];
 #pragma unroll
     for (int f = 0; f < 7; f++) { acc[f][0] = 0; acc[f][1] = 0; }
     float yacc = 0.f;
     // a lane takes units u = 2 (lane + 32 i), +1: 128 consecutive codes, one group of the group-wise grid
-    for (int u0 = 2 * lane; u0 < nunit; u0 += 64) {
+    for (int it = 0; it < nit; it++) {
+      const int u0 = 2 * lane + 64 * it;
+      uint4 ac[2] = {an[0], an[1]};
+      uint2 zc[2] = {zn[0], zn[1]};
+      if (it + 1 < nit) fetch(row, it + 1, an, zn); else fetch(row + warps, 0, an, zn);
+      if (u0 >= nunit) continue;   // (only in the last step of a row; the prefetch above has been issued)
 #pragma unroll
       for (int h = 0; h < 2; h++) {
         const int u = u0 + h;
         if (u < nunit) {
-          const uint4 a = __ldg(w2 + u);
-          const uint2 z = __ldg(w1 + u);
-          const uint32_t ww[4] = {a.x, a.y, a.z, a.w};
+          const uint32_t ww[4] = {ac[h].x, ac[h].y, ac[h].z, ac[h].w};
 #pragma unroll
           for (int i = 0; i < 4; i++) {
-            const uint32_t w = ww[i], hb = w >> 1;
-            const uint32_t zz = ((i & 1) ? ((i < 2 ? z.x : z.y) >> 1) : (i < 2 ? z.x : z.y)) & 0x55555555u;
-            // the seven planes, 16 single bits at the even bit positions
-            uint32_t P[7];
-            P[0] = w & 0x55555555u;           // b0
-            P[1] = hb & 0x55555555u;          // b1
-            P[2] = P[0] & hb;                 // b0 b1
-            P[3] = zz;                        // b2
-            P[4] = w & zz;                    // b0 b2
-            P[5] = hb & zz;                   // b1 b2
-            P[6] = P[2] & zz;                 // b0 b1 b2
+            const uint32_t w = ww[i], hb = w >> 1, whb = w & hb;
+            const uint32_t zsel = (i < 2) ? zc[h].x : zc[h].y;
+            const uint32_t zz = (i & 1) ? (zsel >> 1) : zsel;   // top bits lined up with the b0 bits (odd bits: the other half's)
             const uint4 q = s_act[(h * 4 + i) * npair + (u0 >> 1)];
             const uint32_t qq[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-            for (int f = 0; f < 7; f++)
+            for (int pp = 0; pp < 4; pp++) {
+              // the seven products of code bits at in-byte position pp: one logic operation each (the mask keeps
+              // the even bit of the position, so stray odd bits of hb and zz drop out)
+              const uint32_t m = 0x01010101u << (2 * pp);
+              uint32_t P[7];
+              P[0] = w & m;                   // b0
+              P[1] = hb & m;                  // b1
+              P[2] = whb & m;                 // b0 b1
+              P[3] = zz & m;                  // b2
+              asm("lop3.b32 %0, %1, %2, %3, 0x80;" : "=r"(P[4]) : "r"(w), "r"(zz), "r"(m));     // b0 b2
+              asm("lop3.b32 %0, %1, %2, %3, 0x80;" : "=r"(P[5]) : "r"(hb), "r"(zz), "r"(m));    // b1 b2
+              asm("lop3.b32 %0, %1, %2, %3, 0x80;" : "=r"(P[6]) : "r"(whb), "r"(zz), "r"(m));   // b0 b1 b2
 #pragma unroll
-              for (int pp = 0; pp < 4; pp++)
-                acc[f][pp >> 1] = __dp4a((int)(P[f] & (0x01010101u << (2 * pp))), (int)qq[pp], acc[f][pp >> 1]);
+              for (int f = 0; f < 7; f++) acc[f][pp >> 1] = __dp4a((int)P[f], (int)qq[pp], acc[f][pp >> 1]);
+            }
           }
         }
       }
