@@ -41,4 +41,7 @@ def build_checked(force: bool = False) -> str:
 
 
 if __name__ == "__main__":
+    import sys
     print(build(force=True, verbose=True))
+    if "--checked" in sys.argv[1:]:
+        print(build_checked(force=True))
