@@ -155,7 +155,7 @@ class LayerSet:
             self.y.append(torch.empty(M, L.N, dtype=torch.float16, device=device))
             self.ws.append(rcp.make_workspace(M, L.N, L.K, device))
         self.copies = copies
-        self.digits = self.unit = None
+        self.digits = self.unit = self.w3 = None
 
     def step_w2a16(self, copy):
         """The same layer in the weight-only form (fp16 activations): split kernel + GEMV per linear."""
@@ -166,10 +166,29 @@ class LayerSet:
             self.rcp.rcp_gemv_w2a16(self.words[li][copy], self.luts[li][copy], self.x[li], y=self.y[li],
                                     digits=self.digits[li], unit=self.unit[li], workspace=self.ws[li])
 
+    def step_w3a4(self, copy):
+        """The same layer with 3-bit weights (random codes: the timing does not depend on them): quantizer + GEMV."""
+        if self.w3 is None:
+            self.w3 = []
+            for L in self.layers:
+                per = []
+                for _ in range(self.copies):
+                    w2 = torch.randint(-2 ** 31, 2 ** 31 - 1, (L.N, L.K // 16), dtype=torch.int32, device=self.dev)
+                    w1 = torch.randint(-2 ** 31, 2 ** 31 - 1, (L.N, L.K // 32), dtype=torch.int32, device=self.dev)
+                    per.append((w2, w1))
+                lut8 = torch.sort(torch.randn(L.N, 8, device=self.dev) * 0.02, dim=1).values.half()
+                self.w3.append((per, lut8))
+        for li, L in enumerate(self.layers):
+            per, lut8 = self.w3[li]
+            self.rcp.rcp_quantize_act(self.x[li], L.had_block, 1.0, xq=self.xq[li], scale=self.scale[li])
+            self.rcp.rcp_gemv_w3a4(per[copy][0], per[copy][1], lut8, self.xq[li], self.scale[li], y=self.y[li])
+
     def step(self, copy, variant="auto"):
         r = self.rcp
         if variant == "w2a16":
             return self.step_w2a16(copy)
+        if variant == "w3a4":
+            return self.step_w3a4(copy)
         for li, L in enumerate(self.layers):
             if variant == "auto":
                 # the library's own chain: one kernel where that is faster, else quantizer + GEMV
@@ -472,9 +491,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2_70b", choices=list(cfgs.BY_KEY))
     ap.add_argument("--tokens", type=int, default=1)
-    ap.add_argument("--variant", default="auto", choices=["auto", "simple", "dp4a", "mma", "mma_only", "mma_stream", "w2a16"],
-                    help="kernel variant of the W2A4 GEMV; w2a16 (only with --profile) runs the layer in the "
-                         "weight-only form instead, for the ncu summaries")
+    ap.add_argument("--variant", default="auto", choices=["auto", "simple", "dp4a", "mma", "mma_only", "mma_stream", "w2a16", "w3a4"],
+                    help="kernel variant of the W2A4 GEMV; w2a16 and w3a4 (only with --profile) run the layer in the "
+                         "weight-only form and with 3-bit weights instead, for the ncu summaries")
     ap.add_argument("--no-table", action="store_true", help="skip the per-shape table of the other configs")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle leg")
     ap.add_argument("--sample-seconds", type=float, default=12.0,
@@ -487,8 +506,8 @@ def main():
     if args.warmup < 3:
         args.warmup = 3
 
-    if args.variant == "w2a16" and (not args.profile or args.impl == "reference"):
-        ap.error("--variant w2a16 is a profiling aid: use it with --profile")
+    if args.variant in ("w2a16", "w3a4") and (not args.profile or args.impl == "reference"):
+        ap.error(f"--variant {args.variant} is a profiling aid: use it with --profile")
     if args.impl == "reference":
         run_reference(args, cfg, M)
         return

@@ -166,6 +166,32 @@ int rcp_gemv_w3a4(const uint32_t* words2, const uint32_t* words1, const void* lu
                   int32_t* S_dbg, void* stream);
 
 /*
+ * Export of a 3-bit layer trained with a learnable centre to the inputs of rcp_gemv_w3a4 (Section 4.3, paragraph
+ * "Application of LDP on NF3 format", Eq. "nf3scales", Eq. "nf3"; clipping range of Section 4.2). Offline, like
+ * rcp_ldp_export. A unit is `group` consecutive weights of a row:
+ *   lo = sig_beta * min(W), hi = sig_gamma * max(W), h = hi - lo, W clipped to [lo, hi];
+ *   c = lo + h * sig_s1 (the centre), s_neg = |c - lo|, s_pos = |hi - c|;
+ *   v = (W - c) / s_pos if W > c, else (W - c) / s_neg;
+ *   code = index of the table level nearest to v among the levels of v's side (a tie takes the lower level; a
+ *          weight equal to c is on the negative side);
+ *   level_i = c + table[i] * (s_pos if i > zero_index else s_neg), rounded to fp16.
+ * fp32 arithmetic, one rounding per operation. A unit with h <= 0 gets code zero_index and eight levels lo.
+ * The paper takes the normalized levels of the format from that format's own publication and prints none, so
+ * they are an argument:
+ *   table8_host  HOST float [8], strictly ascending, table8_host[zero_index] == 0 (else RCP_ERR_SHAPE); read
+ *                during the call.
+ *   w_f16, sig_beta, sig_gamma, sig_s1   as for rcp_ldp_export (DEVICE; sigmoids evaluated by the caller).
+ *   group      a multiple of 32 dividing K (K for one grid per row).
+ *   words2, words1   DEVICE, the layout above; 16-byte aligned.
+ *   lut_f16    DEVICE fp16 [N][K/group][8], 16-byte aligned (the lut of rcp_gemv_w3a4 for group 128, or for
+ *              group == K with its group argument 0).
+ * Never synchronizes; ordering against the GEMV as for rcp_ldp_export.
+ */
+int rcp_nf3_export(const void* w_f16, const float* sig_beta, const float* sig_gamma, const float* sig_s1,
+                   const float* table8_host, int zero_index, int N, int K, int group, uint32_t* words2,
+                   uint32_t* words1, void* lut_f16, void* stream);
+
+/*
  * Bytes of caller-provided scratch rcp_gemv_w2a4 needs for this shape (0 on bad shapes). The scratch
  * holds a status word that a kernel sets if one of its bounded waits ever gives up (0 = fine). It
  * must be zero-filled once after allocation; every successful call leaves it zero-filled, so one

@@ -6,5 +6,5 @@ this package only marshals arguments. Importing it needs neither a GPU nor the b
 calling any entry point without the library raises.
 """
 from .binding import (RcpError, lib, make_workspace, rcp_gemv_w2a4, rcp_gemv_workspace_bytes,  # noqa: F401
-                      rcp_gemv_w2a4_grouped, rcp_gemv_w2a4_static, rcp_gemv_w2a16, rcp_ldp_export, rcp_linear_w2a4, rcp_linear_w2a4_host, rcp_linear_w2a4_launches, rcp_pack_weights, rcp_quantize_act,
+                      rcp_gemv_w2a4_grouped, rcp_gemv_w2a4_static, rcp_gemv_w2a16, rcp_ldp_export, rcp_nf3_export, rcp_linear_w2a4, rcp_linear_w2a4_host, rcp_linear_w2a4_launches, rcp_pack_weights, rcp_quantize_act,
                       rcp_pack_weights3, rcp_gemv_w3a4)

@@ -56,6 +56,8 @@ def lib():
         L.rcp_gemv_w2a4_grouped_variant.argtypes = [i, vp, vp, i, vp, vp, i, i, i, vp, vp, vp, vp]
         L.rcp_ldp_export.restype = i
         L.rcp_ldp_export.argtypes = [vp, vp, vp, vp, vp, i, i, i, vp, vp, vp]
+        L.rcp_nf3_export.restype = i
+        L.rcp_nf3_export.argtypes = [vp, vp, vp, vp, C.POINTER(C.c_float), i, i, i, i, vp, vp, vp, vp]
         L.rcp_linear_w2a4.restype = i
         L.rcp_linear_w2a4.argtypes = [vp, i, i, i, C.c_float, vp, vp, i, i, vp, vp, vp, vp, vp]
         L.rcp_linear_w2a4_launches.restype = i
@@ -140,6 +142,31 @@ def rcp_ldp_export(w, sig_beta, sig_gamma, sig_s1, sig_s2, group):
                lib().rcp_ldp_export(_ptr(w), _ptr(sig_beta), _ptr(sig_gamma), _ptr(sig_s1), _ptr(sig_s2), N, K, group,
                                     _ptr(words), _ptr(lut), _stream(w)))
     return words, lut
+
+
+def rcp_nf3_export(w, sig_beta, sig_gamma, sig_s1, table, zero_index, group):
+    """Rotated weights fp16 [N][K], the sigmoids of the clipping parameters and of the centre (float32
+    [N][K/group]) and the format's eight normalized levels (a sequence of floats, table[zero_index] == 0)
+    -> (words2 int32 [N][K/16], words1 int32 [N][K/32], lut fp16 [N][K/group][8])."""
+    _dev(w, torch.float16, "w")
+    N, K = w.shape
+    group = int(group)
+    for name, a in (("sig_beta", sig_beta), ("sig_gamma", sig_gamma), ("sig_s1", sig_s1)):
+        _dev(a, torch.float32, name)
+        if group < 1 or K % group or tuple(a.shape) != (N, K // group):
+            raise ValueError(f"{name}: expected shape [N][K/group]")
+    table = [float(t) for t in table]
+    if len(table) != 8:
+        raise ValueError("table: eight levels expected")
+    tab = (C.c_float * 8)(*table)
+    words2 = torch.empty((N, K // 16), dtype=torch.int32, device=w.device)
+    words1 = torch.empty((N, K // 32), dtype=torch.int32, device=w.device)
+    lut = torch.empty((N, K // group, 8), dtype=torch.float16, device=w.device)
+    with _on(w):
+        _check("rcp_nf3_export",
+               lib().rcp_nf3_export(_ptr(w), _ptr(sig_beta), _ptr(sig_gamma), _ptr(sig_s1), tab, int(zero_index), N, K,
+                                    group, _ptr(words2), _ptr(words1), _ptr(lut), _stream(w)))
+    return words2, words1, lut
 
 
 def rcp_quantize_act(x: torch.Tensor, had_block: int, clip_ratio: float = 1.0, xq=None, scale=None):

@@ -483,7 +483,7 @@ int static_scratch_address(void** out) {
 }
 
 template <bool GRP, bool SDBG>
-int launch_w3(const rcp::W3Params& wp, int grid, size_t smem, cudaStream_t st) {
+int launch_w3(const rcp::W3Params& wp, size_t smem, cudaStream_t st) {
   static std::mutex mu;
   static bool attr_set[kMaxDevices] = {};
   auto kern = rcp::gemv_w3a4_kernel<GRP, SDBG>;
@@ -497,6 +497,12 @@ int launch_w3(const rcp::W3Params& wp, int grid, size_t smem, cudaStream_t st) {
       attr_set[dev] = true;
     }
   }
+  // One wave of resident CTAs, rows dealt round-robin to their warps (measured: CTAs beyond the resident wave,
+  // and warps sharing a row along K, both cost more than the evener load returns).
+  int per_sm = 0;
+  RCP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, rcp::kW3Threads, smem));
+  const int warps_per_cta = rcp::kW3Threads / 32;
+  const int grid = std::min(sm_count() * std::max(per_sm, 1), (wp.N + warps_per_cta - 1) / warps_per_cta);
   kern<<<grid, rcp::kW3Threads, smem, st>>>(wp);
   RCP_CUDA(cudaGetLastError());
   return RCP_OK;
@@ -573,8 +579,7 @@ int rcp_gemv_w3a4(const uint32_t* words2, const uint32_t* words1, const void* lu
     return RCP_ERR_ALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int ngrp = group ? K / 128 : 1;
-  const int grid = std::min((N + rcp::kW3Threads / 32 - 1) / (rcp::kW3Threads / 32), sm_count() * 4);
-  const size_t smem = (size_t)((K / 64 + 1) / 2) * 8 * 16;   // expanded activations: eight 16-byte slots per pair of units
+  const size_t smem = (size_t)((K / 64 + 63) / 64) * 4096;   // expanded activations, K padded to whole lane steps of 4096 codes
   for (int m = 0; m < M; m++) {   // one token per launch: the variant is tuned for decoding one token
     rcp::W3Params wp;
     wp.words2 = words2; wp.words1 = words1;
@@ -585,10 +590,39 @@ int rcp_gemv_w3a4(const uint32_t* words2, const uint32_t* words1, const void* lu
     wp.S_out = S_dbg ? S_dbg + (size_t)m * N * ngrp * 8 : nullptr;
     wp.N = N; wp.K = K;
     int rc;
-    if (group) rc = S_dbg ? launch_w3<true, true>(wp, grid, smem, st) : launch_w3<true, false>(wp, grid, smem, st);
-    else rc = S_dbg ? launch_w3<false, true>(wp, grid, smem, st) : launch_w3<false, false>(wp, grid, smem, st);
+    if (group) rc = S_dbg ? launch_w3<true, true>(wp, smem, st) : launch_w3<true, false>(wp, smem, st);
+    else rc = S_dbg ? launch_w3<false, true>(wp, smem, st) : launch_w3<false, false>(wp, smem, st);
     if (rc != RCP_OK) return rc;
   }
+  return RCP_OK;
+}
+
+int rcp_nf3_export(const void* w_f16, const float* sig_beta, const float* sig_gamma, const float* sig_s1,
+                   const float* table8_host, int zero_index, int N, int K, int group, uint32_t* words2,
+                   uint32_t* words1, void* lut_f16, void* stream) {
+  if (!w_f16 || !sig_beta || !sig_gamma || !sig_s1 || !table8_host || !words2 || !words1 || !lut_f16) return RCP_ERR_NULL;
+  if (N < 1 || !k_ok(K) || group < 32 || group % 32 || K % group) return RCP_ERR_SHAPE;
+  if (zero_index < 0 || zero_index > 7 || table8_host[zero_index] != 0.0f) return RCP_ERR_SHAPE;
+  for (int i = 1; i < 8; i++)
+    if (!(table8_host[i] > table8_host[i - 1])) return RCP_ERR_SHAPE;   // ascending (and no NaN)
+  if (!aligned16(w_f16) || !aligned16(words2) || !aligned16(words1) || !aligned16(lut_f16) ||
+      (reinterpret_cast<uintptr_t>(sig_beta) & 3u) || (reinterpret_cast<uintptr_t>(sig_gamma) & 3u) ||
+      (reinterpret_cast<uintptr_t>(sig_s1) & 3u))
+    return RCP_ERR_ALIGN;
+  rcp::Nf3Params np;
+  np.w = static_cast<const __half*>(w_f16);
+  np.sb = sig_beta; np.sg = sig_gamma; np.s1 = sig_s1;
+  np.words2 = words2; np.words1 = words1;
+  np.lut = static_cast<uint4*>(lut_f16);
+  for (int i = 0; i < 8; i++) np.table[i] = table8_host[i];
+  np.zero = zero_index;
+  np.N = N; np.K = K; np.G = group;
+  np.units = (long long)N * (K / group);
+  const int block = 256;
+  const long long want = (np.units + (block / 32) - 1) / (block / 32);
+  const int grid = (int)std::min<long long>(want, (long long)sm_count() * 16);
+  rcp::nf3_export_kernel<<<grid, block, 0, static_cast<cudaStream_t>(stream)>>>(np);
+  RCP_CUDA(cudaGetLastError());
   return RCP_OK;
 }
 

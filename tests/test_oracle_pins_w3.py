@@ -4,27 +4,12 @@ fixture and a textbook special case. Nothing here compares the oracle with itsel
 import os
 
 import numpy as np
-import scipy.stats
 
 import oracle
 from gen import synth
-from helpers import f16_bits
+from helpers import f16_bits, normal_float_table
 
 GOLD = os.path.join(os.path.dirname(__file__), "golden")
-
-
-def normal_float_table(bits=3):
-    """Normalized levels of an asymmetric normal-float format, built from its published construction: equally
-    spaced probabilities between an offset and 1/2 are sent through the normal quantile function, 2^(bits-1) of
-    them on the positive side and 2^(bits-1) - 1 on the negative side, zero added, the lot divided by the
-    largest. Returns (table float32 [2^bits] ascending, index of zero)."""
-    half = 2 ** (bits - 1)
-    offset = 0.5 * ((1 - 1 / (2 * (2 * half - 1))) + (1 - 1 / (2 * 2 * half)))
-    pos = scipy.stats.norm.ppf(np.linspace(offset, 0.5, half + 1)[:-1])
-    neg = -scipy.stats.norm.ppf(np.linspace(offset, 0.5, half)[:-1])
-    t = np.sort(np.concatenate([neg, [0.0], pos]))
-    t = t / np.abs(t).max()
-    return t.astype(np.float32), int(np.argmin(np.abs(t)))
 
 
 # ----------------------------------------------------------------------------- packing
