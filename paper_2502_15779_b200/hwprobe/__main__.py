@@ -1,8 +1,8 @@
 """Micro-benchmarks behind the kernel design: what the B200's pipes do with the operations the W2A4 GEMV is made of.
 
-    python -m paper_2502_15779_b200.hwprobe [pipes] [umma_rate] [umma_pipeline] [sign_field_mix]
+    python -m paper_2502_15779_b200.hwprobe [pipes] [umma_rate] [umma_pipeline] [sign_field_mix] [bmma_rate]
 
-builds the named programs (all four by default) with nvcc for sm_100a next to their sources and runs them on the
+builds the named programs (all by default) with nvcc for sm_100a next to their sources and runs them on the
 current GPU; each prints its own table. They measure, they do not test anything: every wait in them is bounded.
 
   pipes           issue rates of LOP3, dp4a and int8 mma.sync alone and combined (other warps, same warp, with and
@@ -11,13 +11,14 @@ current GPU; each prints its own table. They measure, they do not test anything:
   umma_pipeline   the whole tcgen05 route for this GEMV: masked code words written to tensor memory by the threads,
                   int8 activations in shared memory, sums checked against the host, bytes of weights per clock
   sign_field_mix  the instruction mix of a formulation with fewer logic operations but more shifts and adds
+  bmma_rate       clocks per binary mma.sync (m16n8k256, and.popc) and a check of its fragment layout
 """
 import os
 import subprocess
 import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-PROGRAMS = {"pipes": [[]], "umma_rate": [[]], "sign_field_mix": [[]],
+PROGRAMS = {"pipes": [[]], "umma_rate": [[]], "sign_field_mix": [[]], "bmma_rate": [[]],
             "umma_pipeline": [["1", "4", "1", "0"], ["8", "8", "1", "0"], ["1", "2000", "148", "0"], ["8", "2000", "148", "0"],
                               ["1", "2000", "148", "1"], ["1", "2000", "148", "2"]]}
 
