@@ -155,7 +155,7 @@ class LayerSet:
             self.y.append(torch.empty(M, L.N, dtype=torch.float16, device=device))
             self.ws.append(rcp.make_workspace(M, L.N, L.K, device))
         self.copies = copies
-        self.digits = self.unit = self.w3 = None
+        self.digits = self.unit = self.w3 = self.glut = None
 
     def step_w2a16(self, copy):
         """The same layer in the weight-only form (fp16 activations): split kernel + GEMV per linear."""
@@ -183,10 +183,22 @@ class LayerSet:
             self.rcp.rcp_quantize_act(self.x[li], L.had_block, 1.0, xq=self.xq[li], scale=self.scale[li])
             self.rcp.rcp_gemv_w3a4(per[copy][0], per[copy][1], lut8, self.xq[li], self.scale[li], y=self.y[li])
 
+    def step_grouped(self, copy):
+        """The same layer with one grid per group of 128 weights (the paper's own granularity): the library's chain
+        with group=128 (one kernel where the quantizer goes inside, else quantizer + GEMV)."""
+        if self.glut is None:
+            self.glut = [synth.make_lut_grouped(L.N, L.K // 128, cfgs.BASE_SEED + 31 * li, self.dev)
+                         for li, L in enumerate(self.layers)]
+        for li, L in enumerate(self.layers):
+            self.rcp.rcp_linear_w2a4(self.x[li], L.had_block, 1.0, self.words[li][copy], self.glut[li], group=128,
+                                     y=self.y[li], xq=self.xq[li], scale=self.scale[li], workspace=self.ws[li])
+
     def step(self, copy, variant="auto"):
         r = self.rcp
         if variant == "w2a16":
             return self.step_w2a16(copy)
+        if variant == "grouped":
+            return self.step_grouped(copy)
         if variant == "w3a4":
             return self.step_w3a4(copy)
         for li, L in enumerate(self.layers):
@@ -491,9 +503,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2_70b", choices=list(cfgs.BY_KEY))
     ap.add_argument("--tokens", type=int, default=1)
-    ap.add_argument("--variant", default="auto", choices=["auto", "simple", "dp4a", "mma", "mma_only", "mma_stream", "w2a16", "w3a4"],
-                    help="kernel variant of the W2A4 GEMV; w2a16 and w3a4 (only with --profile) run the layer in the "
-                         "weight-only form and with 3-bit weights instead, for the ncu summaries")
+    ap.add_argument("--variant", default="auto", choices=["auto", "simple", "dp4a", "mma", "mma_only", "mma_stream", "w2a16", "w3a4", "grouped"],
+                    help="kernel variant of the W2A4 GEMV; w2a16, w3a4 and grouped (only with --profile) run the layer in "
+                         "the weight-only form, with 3-bit weights and with one grid per group of 128 weights "
+                         "instead, for the ncu summaries")
     ap.add_argument("--no-table", action="store_true", help="skip the per-shape table of the other configs")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle leg")
     ap.add_argument("--sample-seconds", type=float, default=12.0,
@@ -506,7 +519,7 @@ def main():
     if args.warmup < 3:
         args.warmup = 3
 
-    if args.variant in ("w2a16", "w3a4") and (not args.profile or args.impl == "reference"):
+    if args.variant in ("w2a16", "w3a4", "grouped") and (not args.profile or args.impl == "reference"):
         ap.error(f"--variant {args.variant} is a profiling aid: use it with --profile")
     if args.impl == "reference":
         run_reference(args, cfg, M)
