@@ -114,7 +114,7 @@ struct GemvParams {
   uint8_t* xq_out;      // optional [M][K/2]: the int4 activations, written by CTA 0
   __half* scale_out;    // optional [M]
   float inv_sqrt_b, clip_ratio;   // the rotation block is the whole token, K = 4096 or 8192
-  int off_qbuf;         // 4 K bytes of shared memory
+  int off_qbuf;         // the quantizer's scratch (rotate_scratch_bytes(K)) in shared memory
   int stages;           // ring depth
   int ramp_clk;         // clocks between the first `stages` requests of a CTA
   int off_bar, off_T0c, off_scale, off_red, off_bs;   // shared-memory byte offsets from the aligned base
@@ -481,7 +481,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     static_assert(!FQ || (MODE == kModeDp4a && MTOK == 1), "the fused quantizer serves the one-token kernels");
     constexpr int NT = kCWarps * 32;
     const int W = p.K / 16;                                           // 256 or 512 words: one per thread
-    float* const qbuf = reinterpret_cast<float*>(gen + p.off_qbuf);   // [16][W]
+    float* const qbuf = reinterpret_cast<float*>(gen + p.off_qbuf);   // rotate_scratch_bytes(K)
     float* const s_amax = s_scale + 16;                               // [16 warps] behind the scales
     float v[16];
     const float sc = rotate_token_words<NT>(p.x, W, p.inv_sqrt_b, p.clip_ratio, qbuf, s_amax, v);

@@ -193,16 +193,27 @@ __global__ void __launch_bounds__(1024) quantize_act_kernel(const QuantParams p)
 
 // ---------------------------------------------------------------------------------------------
 // One token of W = K / 16 words (256 or 512) under a single rotation block, by NT = 512 threads of one
-// CTA: thread tid holds word tid (16 consecutive activations). Strides 1..8 inside the word, 16..256
-// by lane exchanges, 512 and up through shared memory (thread (element tid >> 5, lane) takes the
-// R = W / 32 values of its column, 32 words apart), then the scale by 1/sqrt(K) and the token's
-// absmax. Same operations in the same order as quantize_act_kernel. Leaves the rotated, scaled
-// activations of the thread's word in v and returns the quantization scale (as rounded to fp16).
-// Uses named barrier 1 with NT threads; qbuf: 16 * W floats, s_amax: NT / 32 floats.
+// CTA: thread tid holds word tid (16 consecutive activations). Every butterfly stage runs in registers, the
+// data changing hands through shared memory in between, in ascending order of the strides (the order of
+// quantize_act_kernel: same operations on the same operands, bit-identical results):
+//   strides 1..8      inside the word;
+//   strides 16..128   after a transposition inside the warp (thread (h, e) of a warp, h = lane >> 4,
+//                     e = lane & 15, takes element e of the warp's words 16 h .. 16 h + 15);
+//   stride 256        one lane exchange (lane ^ 16);
+//   strides 512 ..    after a transposition across the warps (thread (warp = element, lane) takes the
+//                     R = W / 32 values of its column, 32 words apart);
+// then the scale by 1/sqrt(K) and the token's absmax. Leaves the rotated, scaled activations of the thread's
+// word in v and returns the quantization scale (as rounded to fp16). Uses named barrier 1 with NT threads;
+// qbuf: rotate_scratch_bytes(K) bytes, 16-byte aligned; s_amax: NT / 32 floats.
+__host__ __device__ constexpr size_t rotate_scratch_bytes(int K) { return (size_t)17 * (K / 16) * 4; }
+
 template <int NT>
 __device__ __forceinline__ float rotate_token_words(const __half* x, int W, float inv_sqrt_b, float clip_ratio,
                                                     float* qbuf, float* s_amax, float (&v)[16]) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int kPitch = 17;   // rows of the in-warp transposition: 16 floats and one of padding (no bank conflicts)
+  const int QP = W + 4;        // pitch of the cross-warp buffer [16 elements][W words]: the 16-byte stores of eight
+                               // lanes with different elements then fall into different banks
   if (tid < W) {
     const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)tid * 16);
     const uint4 r0 = __ldg(src), r1 = __ldg(src + 1);
@@ -217,34 +228,50 @@ __device__ __forceinline__ float rotate_token_words(const __half* x, int W, floa
 #pragma unroll
     for (int e = 0; e < 16; e++) v[e] = 0.f;
   }
+  // sixteen values in registers: the four stages that pair them
+  auto butterflies16 = [](float (&a)[16]) {
 #pragma unroll
-  for (int h = 1; h < 16; h *= 2) {
+    for (int h = 1; h < 16; h *= 2) {
 #pragma unroll
-    for (int e = 0; e < 16; e++) {
-      if ((e & h) == 0) {
-        const float u = v[e], w = v[e + h];
-        v[e] = __fadd_rn(u, w);
-        v[e + h] = __fsub_rn(u, w);
+      for (int e = 0; e < 16; e++) {
+        if ((e & h) == 0) {
+          const float u = a[e], w = a[e + h];
+          a[e] = __fadd_rn(u, w);
+          a[e + h] = __fsub_rn(u, w);
+        }
       }
     }
-  }
+  };
+  butterflies16(v);   // strides 1..8
+  const bool data_warp = warp * 32 < W;   // (W is a multiple of 256: a warp holds 32 words or none)
+  const int e1 = lane & 15, hi = lane & 16;
+  float u[16];
 #pragma unroll
-  for (int d = 1; d < 32; d *= 2) {   // element stride 16 d <-> lane distance d
-    const bool upper = (lane & d) != 0;
+  for (int j = 0; j < 16; j++) u[j] = 0.f;
+  if (data_warp) {
+    float* const wbuf = qbuf + warp * (32 * kPitch);
 #pragma unroll
-    for (int e = 0; e < 16; e++) {
-      const float other = __shfl_xor_sync(0xffffffffu, v[e], d);
-      v[e] = upper ? __fsub_rn(other, v[e]) : __fadd_rn(v[e], other);
+    for (int e = 0; e < 16; e++) wbuf[lane * kPitch + e] = v[e];
+    __syncwarp();
+#pragma unroll
+    for (int j = 0; j < 16; j++) u[j] = wbuf[(hi | j) * kPitch + e1];   // element e1 of the words hi + j
+    butterflies16(u);   // strides 16..128
+#pragma unroll
+    for (int j = 0; j < 16; j++) {   // stride 256
+      const float other = __shfl_xor_sync(0xffffffffu, u[j], 16);
+      u[j] = hi ? __fsub_rn(other, u[j]) : __fadd_rn(u[j], other);
     }
   }
-  if (tid < W) {
+  asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");   // every warp is done with its transposition area
+  if (data_warp) {   // u[j]: element e1 of word warp * 32 + hi + j
+    float4* const dst = reinterpret_cast<float4*>(qbuf + e1 * QP + warp * 32 + hi);
 #pragma unroll
-    for (int e = 0; e < 16; e++) qbuf[e * W + tid] = v[e];
+    for (int j = 0; j < 4; j++) dst[j] = make_float4(u[4 * j], u[4 * j + 1], u[4 * j + 2], u[4 * j + 3]);
   }
   asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");
   {
     const int R = W >> 5;   // 8 or 16 warps hold data
-    float* const colp = qbuf + warp * W + lane;
+    float* const colp = qbuf + warp * QP + lane;
     float tv[16];
 #pragma unroll
     for (int w = 0; w < 16; w++) tv[w] = (w < R) ? colp[w * 32] : 0.f;
@@ -254,9 +281,9 @@ __device__ __forceinline__ float rotate_token_words(const __half* x, int W, floa
 #pragma unroll
         for (int w = 0; w < 16; w++) {
           if ((w & h) == 0) {
-            const float u = tv[w], z = tv[w + h];
-            tv[w] = __fadd_rn(u, z);
-            tv[w + h] = __fsub_rn(u, z);
+            const float a = tv[w], z = tv[w + h];
+            tv[w] = __fadd_rn(a, z);
+            tv[w + h] = __fsub_rn(a, z);
           }
         }
       }
@@ -267,7 +294,7 @@ __device__ __forceinline__ float rotate_token_words(const __half* x, int W, floa
   asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");
   if (tid < W) {
 #pragma unroll
-    for (int e = 0; e < 16; e++) v[e] = qbuf[e * W + tid];
+    for (int e = 0; e < 16; e++) v[e] = qbuf[e * QP + tid];
   }
   float amax = 0.f;
 #pragma unroll
@@ -289,7 +316,7 @@ __device__ __forceinline__ float rotate_token_words(const __half* x, int W, floa
 // faster than the cluster form above for these shapes (no cluster launch, no passes through
 // distributed shared memory).
 __global__ void __launch_bounds__(512) quantize_act_wide_kernel(const QuantParams p) {
-  extern __shared__ float sbuf[];   // 16 * W floats
+  extern __shared__ __align__(16) float sbuf[];   // rotate_scratch_bytes(K)
   __shared__ float s_amax[16];
   const int m = blockIdx.x, tid = threadIdx.x;
   asm volatile("griddepcontrol.launch_dependents;");

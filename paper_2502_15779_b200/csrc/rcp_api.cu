@@ -321,7 +321,7 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   if (fa && (mode != rcp::kModeDp4a || !fused_ok(M, K, fa->B))) return RCP_ERR_VARIANT;
   EncodeTiledFn enc = encode_tiled_fn();
   if (!enc) return cuda_fail(cudaErrorNotSupported);
-  const StreamPlan pl = make_plan(M, N, K, sm_count(), grouped, fa ? (size_t)4 * K : (sa ? (size_t)M * K : 0), nsplit,
+  const StreamPlan pl = make_plan(M, N, K, sm_count(), grouped, fa ? rcp::rotate_scratch_bytes(K) : (sa ? (size_t)M * K : 0), nsplit,
                                   stream_act);
   if (pl.stages < 2 || pl.smem > kSmemMax) return RCP_ERR_SHAPE;
   // Tensor maps of the phases in use (the others repeat the first). Encoding one costs the host about a
@@ -672,7 +672,7 @@ int rcp_quantize_act(const void* x_f16, int M, int K, int had_block, float clip_
   if (B == K && (K == 4096 || K == 8192)) {
     // one rotation block over a long token: one CTA of 512 threads per token (measured faster than a cluster)
     qp.unit = K; qp.nunits = 1; qp.lg_local = qp.lgB;
-    RCP_CUDA(launch_overlapped(rcp::quantize_act_wide_kernel, dim3((unsigned)M), dim3(512), (size_t)4 * K, st, qp));
+    RCP_CUDA(launch_overlapped(rcp::quantize_act_wide_kernel, dim3((unsigned)M), dim3(512), rcp::rotate_scratch_bytes(K), st, qp));
     return RCP_OK;
   }
   // whole rotation blocks per CTA (a block is at most 2048 elements here: longer single blocks went above,
