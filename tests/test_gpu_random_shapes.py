@@ -185,3 +185,60 @@ def test_many_launches_repeat_bit_for_bit(N, K, M, variant, grouped):
             assert torch.equal(ys[1].view(torch.int16), ref.view(torch.int16))
     torch.cuda.synchronize()
     assert int(ws.abs().max()) == 0
+
+
+def test_packed_weights_beyond_four_gibibytes():
+    """270 000 rows of 65 536 weights: 17.7 G codes, 4.4 GB of packed words, so every byte offset and element
+    index past 2^32 is exercised (packing, the one-token and the eight-token kernel, the plain kernel's integer
+    sums, the group-wise grid, the 3-bit kernel), on sampled rows against the oracle."""
+    if torch.cuda.get_device_properties(0).total_memory < 60 << 30:
+        pytest.skip("needs about 35 GB of device memory")
+    N, K, B = 270000, 65536, 128
+    g = torch.Generator(device=DEV)
+    g.manual_seed(270000)
+    codes = torch.randint(0, 4, (N, K), dtype=torch.uint8, device=DEV, generator=g)
+    words = rcp.rcp_pack_weights(codes)
+    rows = np.unique(np.concatenate([np.arange(24), np.arange(N - 24, N), [65535, 65536, 65537, 131071, 131072],
+                                     np.random.default_rng(7).integers(0, N, size=48)]))
+    rows_t = torch.from_numpy(rows).to(DEV)
+    w_ref = oracle.pack_weights(codes[rows_t].cpu().numpy())
+    del codes
+    torch.cuda.empty_cache()
+    assert np.array_equal(words[rows_t].cpu().numpy().view(np.uint32), w_ref)
+    lut = synth.make_lut(N, 11, device=DEV)
+    for M, variant in ((1, "auto"), (8, "mma_only"), (1, "simple")):
+        x = synth.make_activations(M, K, 3 + M, device=DEV)
+        xq, scale = rcp.rcp_quantize_act(x, B, 1.0)
+        qa = oracle.quantize_act(f16_bits(x), B, 1.0)
+        assert np.array_equal(xq.cpu().numpy(), qa["xq"]) and np.array_equal(f16_bits(scale), qa["scale"])
+        ws = rcp.make_workspace(M, N, K, DEV)
+        S = torch.zeros(M, N, 4, dtype=torch.int32, device=DEV) if variant == "simple" else None
+        y = rcp.rcp_gemv_w2a4(words, lut, xq, scale, workspace=ws, variant=variant, S_dbg=S)
+        torch.cuda.synchronize()
+        assert int(ws.abs().max()) == 0
+        ref = oracle.gemv_w2a4(w_ref, np.ascontiguousarray(f16_bits(lut[rows_t])), qa["xq"], qa["scale"])
+        got = y[:, rows_t].float().cpu().numpy().astype(np.float64)
+        assert np.all(np.isfinite(got)) and np.all(np.abs(got - ref["y"]) <= ref["tol"]), (M, variant)
+        if S is not None:
+            assert np.array_equal(S[:, rows_t].cpu().numpy(), ref["S"])
+    # one token: group-wise grid and the 3-bit kernel on the same words (a random plane of top bits)
+    x = synth.make_activations(1, K, 5, device=DEV)
+    xq, scale = rcp.rcp_quantize_act(x, B, 1.0)
+    qa = oracle.quantize_act(f16_bits(x), B, 1.0)
+    ws = rcp.make_workspace(1, N, K, DEV)
+    glut = synth.make_lut_grouped(N, K // 128, 13, device=DEV)
+    y = rcp.rcp_gemv_w2a4_grouped(words, glut, xq, scale, group=128, workspace=ws)
+    torch.cuda.synchronize()
+    ref = oracle.gemv_w2a4_grouped(w_ref, np.ascontiguousarray(f16_bits(glut[rows_t])), qa["xq"], qa["scale"], 128)
+    got = y[:, rows_t].float().cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(got - ref["y"]) <= ref["tol"])
+    del glut
+    torch.cuda.empty_cache()
+    w1 = torch.randint(-2 ** 31, 2 ** 31 - 1, (N, K // 32), dtype=torch.int32, device=DEV, generator=g)
+    lut8 = torch.sort(torch.randn(N, 8, device=DEV, generator=g) * 0.02, dim=1).values.half()
+    y = rcp.rcp_gemv_w3a4(words, w1, lut8, xq, scale)
+    torch.cuda.synchronize()
+    ref = oracle.gemv_w3a4(w_ref, w1[rows_t].cpu().numpy().view(np.uint32), np.ascontiguousarray(f16_bits(lut8[rows_t])),
+                           qa["xq"], qa["scale"])
+    got = y[:, rows_t].float().cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(got - ref["y"]) <= ref["tol"])
