@@ -962,48 +962,58 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
         const uint4 x = RCP_LDS128(b_ptr, bs_lo, bs_hi, 9);
         const uint4 y = RCP_LDS128(b_ptr + half_stride, bs_lo, bs_hi, 9);
         const uint32_t bM[4][2] = {{x.x, x.y}, {x.z, x.w}, {y.x, y.y}, {y.z, y.w}};
-        const uint32_t u0 = U.x, u1 = U.y, v0 = V.x, v1 = V.y;
-        const uint32_t u0s = u0 + u0, u1s = u1 + u1, v0s = v0 + v0, v1s = v1 + v1;
+        // Positions 2 and 3 are moved down onto the bits of 0 and 1 first, so that all four positions add into one
+        // set of accumulators: the finish below then converts three sums per entry, not six halves.
+        const uint32_t wu[2][2] = {{U.x, U.y}, {U.x >> 4, U.y >> 4}}, wv[2][2] = {{V.x, V.y}, {V.x >> 4, V.y >> 4}};
+        uint32_t su[2][2], sv[2][2];   // b0 moved onto b1's bit
+#pragma unroll
+        for (int d = 0; d < 2; d++)
+#pragma unroll
+          for (int w = 0; w < 2; w++) { su[d][w] = wu[d][w] + wu[d][w]; sv[d][w] = wv[d][w] + wv[d][w]; }
 #pragma unroll
         for (int po = 0; po < 4; po++) {
-          const int pp = ((po & 1) << 1) | (po >> 1);
-          const uint32_t m0 = 0x01010101u << (2 * pp), m1 = m0 << 1;
-          const uint32_t au0[3] = {u0 & m0, u0 & m1, and3(u0, u0s, m1)};
-          const uint32_t au1[3] = {u1 & m0, u1 & m1, and3(u1, u1s, m1)};
-          const uint32_t av0[3] = {v0 & m0, v0 & m1, and3(v0, v0s, m1)};
-          const uint32_t av1[3] = {v1 & m0, v1 & m1, and3(v1, v1s, m1)};
+          const int pp = ((po & 1) << 1) | (po >> 1);   // positions in the order 0, 2, 1, 3
+          const int d = pp >> 1;
+          const uint32_t m0 = 0x01010101u << (2 * (pp & 1)), m1 = m0 << 1;
+          const uint32_t au0[3] = {wu[d][0] & m0, wu[d][0] & m1, and3(wu[d][0], su[d][0], m1)};
+          const uint32_t au1[3] = {wu[d][1] & m0, wu[d][1] & m1, and3(wu[d][1], su[d][1], m1)};
+          const uint32_t av0[3] = {wv[d][0] & m0, wv[d][0] & m1, and3(wv[d][0], sv[d][0], m1)};
+          const uint32_t av1[3] = {wv[d][1] & m0, wv[d][1] & m1, and3(wv[d][1], sv[d][1], m1)};
 #pragma unroll
           for (int f = 0; f < 3; f++) {
-            if (po < 2) mma_u8s8_zero(accM[f][pp >> 1], au0[f], av0[f], au1[f], av1[f], bM[pp][0], bM[pp][1]);
-            else mma_u8s8(accM[f][pp >> 1], au0[f], av0[f], au1[f], av1[f], bM[pp][0], bM[pp][1]);
+            if (po == 0) mma_u8s8_zero(accM[f][0], au0[f], av0[f], au1[f], av1[f], bM[pp][0], bM[pp][1]);
+            else mma_u8s8(accM[f][0], au0[f], av0[f], au1[f], av1[f], bM[pp][0], bM[pp][1]);
           }
         }
-        // The accumulators hold 4 T1 and 64 T1 (positions {0,1} and {2,3}), 8 and 128 times T2 and T3.
-        // Everything below works on 8 x the sums, in fp32 (small integers: exact); the 1/8 goes into
-        // the final scale.
+        // The accumulators hold 4 T1, 8 T2 and 8 T3. Everything below works on 8 x the sums, in fp32 (small
+        // integers: exact); the 1/8 goes into the final scale. With the levels L0..L3 of the (row, group),
+        //   8 y = L0 (8 T0) + 2 (L1 - L0) (4 T1) + (L2 - L0) (8 T2) + ((L3 - L1) - (L2 - L0)) (8 T3):
+        // the coefficients are made once per row and serve all its tokens.
         const int gi = ch * 4 + j;
         const float2 t0 = *reinterpret_cast<const float2*>(s_T0f + gi * Mp + tok2);
-        uint2 lgj[2];
+        float cf[2][4];
 #pragma unroll
         for (int rr = 0; rr < 2; rr++) {
-          lgj[rr].x = __shfl_sync(0xffffffffu, lg[0][rr].x, (lane & ~3) | j);
-          lgj[rr].y = __shfl_sync(0xffffffffu, lg[0][rr].y, (lane & ~3) | j);
+          const uint32_t lx = __shfl_sync(0xffffffffu, lg[0][rr].x, (lane & ~3) | j);
+          const uint32_t ly = __shfl_sync(0xffffffffu, lg[0][rr].y, (lane & ~3) | j);
+          const float2 l01 = __half22float2(*reinterpret_cast<const __half2*>(&lx));
+          const float2 l23 = __half22float2(*reinterpret_cast<const __half2*>(&ly));
+          const float d1 = l01.y - l01.x, d2 = l23.x - l01.x;
+          cf[rr][0] = l01.x;
+          cf[rr][1] = d1 + d1;
+          cf[rr][2] = d2;
+          cf[rr][3] = (l23.y - l01.y) - d2;
         }
 #pragma unroll
         for (int r = 0; r < 4; r++) {
-          const float F1 = small_int_to_float(accM[0][0][r] + (accM[0][1][r] >> 4));   // 4 T1
-          const float F2 = small_int_to_float(accM[1][0][r] + (accM[1][1][r] >> 4));   // 8 T2
-          const float F3 = small_int_to_float(accM[2][0][r] + (accM[2][1][r] >> 4));   // 8 T3 = 8 S3
-          const float S1 = fmaf(2.f, F1, -F3), S2 = F2 - F3;
-          const float S0 = (((r & 1) ? t0.y : t0.x) - S1) - (S2 + F3);
-          const float2 l01 = __half22float2(*reinterpret_cast<const __half2*>(&lgj[r >> 1].x));
-          const float2 l23 = __half22float2(*reinterpret_cast<const __half2*>(&lgj[r >> 1].y));
-          yacc[r] = fmaf(l01.x, S0, fmaf(l01.y, S1, fmaf(l23.x, S2, fmaf(l23.y, F3, yacc[r]))));
+          const float F1 = small_int_to_float(accM[0][0][r]);   // 4 T1
+          const float F2 = small_int_to_float(accM[1][0][r]);   // 8 T2
+          const float F3 = small_int_to_float(accM[2][0][r]);   // 8 T3
+          const float (&c)[4] = cf[r >> 1];
+          yacc[r] = fmaf(c[0], (r & 1) ? t0.y : t0.x, fmaf(c[1], F1, fmaf(c[2], F2, fmaf(c[3], F3, yacc[r]))));
           if constexpr (SDBG) {
-            // the same sums as integers: the accumulators hold 4 T1, 8 T2, 8 T3 (and 16 times that)
-            const int I1 = (accM[0][0][r] + (accM[0][1][r] >> 4)) >> 2;
-            const int I2 = (accM[1][0][r] + (accM[1][1][r] >> 4)) >> 3;
-            const int I3 = (accM[2][0][r] + (accM[2][1][r] >> 4)) >> 3;
+            // the same sums as integers
+            const int I1 = accM[0][0][r] >> 2, I2 = accM[1][0][r] >> 3, I3 = accM[2][0][r] >> 3;
             const int tok = 2 * t + (r & 1), row = row_first + grow + 8 * (r >> 1);
             if (tok < M && row < p.N && gi < p.ngrp) {
               const int I0 = __float2int_rn(0.125f * ((r & 1) ? t0.y : t0.x)) - (I1 - I3) - (I2 - I3) - I3;
