@@ -230,7 +230,7 @@ __global__ void wait_timeout_kernel(int32_t* status, uint32_t polls) {
 
 // MODE  kModeMma: all three planes on the tensor cores; kModeHybrid: b0 and b1 planes on the tensor
 //       cores, the b0*b1 plane on dp4a; kModeDp4a: everything on dp4a (CUDA cores only)
-// MTOK  tokens, fixed at compile time for the dp4a modes (1 or 2); kModeMma: 0 = run-time, up to 8
+// MTOK  tokens, fixed at compile time for the dp4a modes (1 or 2); kModeMma: 0 = run-time, up to 8; 8 = exactly eight
 //       (one MMA column tile), 16 = run-time, 9 to 16 (two column tiles fed from the same masks)
 // GRP   one grid per group of 128 weights instead of one per row (kModeHybrid has no such form)
 // FQ    one token of 4096 or 8192 activations under one rotation block: the activations arrive as
@@ -263,7 +263,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   uint8_t* const gen = smem_raw + (base - raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t = lane & 3;
-  const int M = (MTOK > 0 && MODE != kModeMma) ? MTOK : p.M;
+  const int M = (MTOK > 0 && MTOK != 16) ? MTOK : p.M;   // (kModeMma with MTOK 8: exactly eight tokens, known at compile time)
   constexpr bool kTwoTiles = (MODE == kModeMma && MTOK == 16);   // tokens 8..15 in a second set of accumulators
   static_assert(!(kTwoTiles && (GRP || FQ)), "two column tiles: per-row grid, quantized activations only");
   static_assert(!A16 || (MODE == kModeMma && !GRP && !FQ), "digit columns: tensor-core mode, per-row grid");

@@ -409,6 +409,7 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
     if (mode == rcp::kModeDp4a)
       return M == 1 ? launch_stream_t<rcp::kModeDp4a, 1, true>(maps, gp, pl, st)
                     : launch_stream_t<rcp::kModeDp4a, 2, true>(maps, gp, pl, st);
+    if (M == 8 && !gp.S_out) return launch_stream_s<rcp::kModeMma, 8, true, false, false, false, false>(maps, gp, pl, st);
     return launch_stream_t<rcp::kModeMma, 0, true>(maps, gp, pl, st);
   }
   if (mode == rcp::kModeHybrid)
@@ -417,8 +418,12 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
   if (mode == rcp::kModeDp4a)
     return M == 1 ? launch_stream_t<rcp::kModeDp4a, 1>(maps, gp, pl, st)
                   : launch_stream_t<rcp::kModeDp4a, 2>(maps, gp, pl, st);
-  if (stream_act) return M > 8 ? launch_stream_sb<16>(maps, gp, pl, st) : launch_stream_sb<0>(maps, gp, pl, st);
+  if (stream_act) {
+    if (M == 8 && !gp.S_out) return launch_stream_sb<8>(maps, gp, pl, st);
+    return M > 8 ? launch_stream_sb<16>(maps, gp, pl, st) : launch_stream_sb<0>(maps, gp, pl, st);
+  }
   if (pl.nsplit > 1) return launch_stream_t<rcp::kModeMma, 0, false, false, false, true>(maps, gp, pl, st);
+  if (M == 8 && !gp.S_out) return launch_stream_s<rcp::kModeMma, 8, false, false, false, false, false>(maps, gp, pl, st);   // token count known at compile time
   return M > 8 ? launch_stream_t<rcp::kModeMma, 16>(maps, gp, pl, st) : launch_stream_t<rcp::kModeMma, 0>(maps, gp, pl, st);
 }
 
