@@ -278,8 +278,10 @@ int rcp_ldp_export(const void* w_f16, const float* sig_beta, const float* sig_ga
  *   y[m][n]      = fp16( scale[m] * sum_j sum_c lut[n][j][c] * S_c[m][n][j] )   (fp32 arithmetic;
  *                  the order of the fp32 sum over groups is fixed for a shape, so results repeat)
  *   lut_f16    DEVICE fp16 [N][K/group][4], 8-byte aligned. A constant of the layer like `words`.
- *   group      a multiple of 16 that divides K. group == 128 runs the streaming kernels; any
- *              other size runs the plain kernel (correct, not tuned).
+ *   group      a multiple of 16 that divides K. group == 128 runs the streaming kernels (up to eight tokens per
+ *              launch; where K is so long that their expanded activations do not fit in shared memory, the form
+ *              that streams the activations beside the weights); any other size runs the plain kernel
+ *              (correct, not tuned).
  *   S_dbg      NULL in production. Otherwise int32 [M][N][K/group][4] receives S_c (plain kernel; through
  *              rcp_gemv_w2a4_grouped_variant with RCP_GEMV_DP4A or RCP_GEMV_MMA_ONLY: the checked
  *              instantiation of that streaming kernel).

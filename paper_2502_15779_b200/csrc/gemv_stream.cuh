@@ -274,7 +274,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   // A form of its own, so that the kernels that never need it keep their code.
   constexpr bool kSplit = SPLIT;
   static_assert(!SPLIT || (MODE == kModeMma && MTOK == 0 && !GRP && !FQ), "K in parts: eight-column tensor-core kernels, per-row grid");
-  static_assert(!SB || (MODE == kModeMma && !GRP && !FQ && !A16 && !SPLIT), "streamed activations: tensor-core kernels, per-row grid");
+  static_assert(!SB || (MODE == kModeMma && !FQ && !A16 && !SPLIT), "streamed activations: tensor-core kernels");
   constexpr int kThreads = SB ? kGThreads + 32 * kExpWarps : kGThreads;   // consumers, producer warp, and the expander warps (SB)
   const uint32_t stage_stride = SB ? (uint32_t)p.stage_stride : (uint32_t)kStageBytes;
   const int nsplit = kSplit ? p.nsplit : 1;
@@ -406,7 +406,7 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
                 if (v < total) {
                   const int j = (int)(((uint32_t)v * inv_box) >> 20), w = v - j * per_box;
                   const int col = w >> 4, lo = w & 3, hi = (w >> 2) & 3;
-                  const int wx = (s * KS + j) * kChunkWords + 8 * lo + 2 * hi;   // first of the unit's two words
+                  const int wx = (s * KS + j) * kChunkWords + (kRelabel ? 8 * hi + 2 * lo : 8 * lo + 2 * hi);   // first of the unit's two words
                   if (wx < W) x[r] = __ldg(reinterpret_cast<const uint4*>(p.xq + (size_t)col * (p.K / 2)) + (wx >> 1));
                 }
               }
@@ -538,6 +538,31 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
     }
     if constexpr (!GRP)
       for (int i = tid; i < 2 * 8 * 16 * M * 3; i += kCWarps * 32) s_red[i] = 0;
+  } else if constexpr (SB && GRP) {
+    // Streamed activations, group-wise grid: the sum of q of every (token, group of 128) is needed up front, as
+    // 8 x the sum in fp32 (what the finish works with). A group is 64 bytes of packed activations.
+    // (the last chunk may reach beyond K: its missing groups get a sum of zero, they meet a grid of zeros)
+    const int ngroups = p.K / 128;
+    for (int i = tid; i < M * ng4; i += kCWarps * 32) {
+      const int col = i / ng4, gi = i - col * ng4;
+      const uint4* src = reinterpret_cast<const uint4*>(p.xq + (size_t)col * (p.K / 2) + (size_t)gi * 64);
+      int tsum = 0;
+#pragma unroll
+      for (int v4 = 0; v4 < 4; v4++) {
+        const uint4 x = gi < ngroups ? __ldg(src + v4) : make_uint4(0, 0, 0, 0);
+        const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int h = 0; h < 4; h++) {
+          uint32_t e = xs[h] & 0x0F0F0F0Fu, o = (xs[h] >> 4) & 0x0F0F0F0Fu;
+          e |= (e & 0x08080808u) * 0x1Eu;
+          o |= (o & 0x08080808u) * 0x1Eu;
+          tsum = __dp4a((int)e, 0x01010101, tsum);
+          tsum = __dp4a((int)o, 0x01010101, tsum);
+        }
+      }
+      s_T0f[gi * Mp + col] = (float)(8 * tsum);
+    }
+    if (tid < M) s_scale[tid] = __half2float(p.scale[tid]);
   } else if constexpr (SB) {
     // Streamed activations: only the sum of q per token is needed up front (S_0 = T0 - S_1 - S_2 - S_3).
     const int nvec = p.K / 32;   // 16-byte vectors of packed activations per token
@@ -949,10 +974,10 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
   };
   // Tensor-core mode: one chunk = four groups, each read by the whole quad, finished after its
   // twelve MMAs.
-  auto compute_chunk_grp_mma = [&](uint32_t a_grp, uint32_t b_chunk, int ch, const uint2 (&lg)[NLG][2], int row_first) {
+  auto compute_chunk_grp_mma = [&](uint32_t a_grp, uint32_t b_abs, int ch, const uint2 (&lg)[NLG][2], int row_first) {   // b_abs: the chunk's expanded activations
     if constexpr (kRelabel) {
       const uint32_t a_row = a_grp + (uint32_t)(grow * 128 + ((t & 1) << 3));
-      const uint32_t b_grp = base + (uint32_t)p.off_bs + b_chunk + bM_lane;
+      const uint32_t b_grp = b_abs + bM_lane;
 #pragma unroll
       for (int j = 0; j < 4; j++) {
         const uint32_t a_sw = (uint32_t)(((2 * j + (t >> 1)) ^ (grow & 7)) << 4);
@@ -1213,9 +1238,11 @@ gemv_stream_kernel(const __grid_constant__ GemvMaps maps, const GemvParams p) {
             return;
           }
           if (active && ch < p.nchunk) {
-            const uint32_t a_grp = base + (uint32_t)slot * kStageBytes + a_off;
+            const uint32_t st = base + (uint32_t)slot * stage_stride;   // (stage_stride == kStageBytes unless SB)
+            const uint32_t a_grp = st + a_off;
             if constexpr (kRelabel) {
-              compute_chunk_grp_mma(a_grp, b_chunk, ch, lg_cur, row_first);
+              compute_chunk_grp_mma(a_grp, SB ? st + kStageBytes + (uint32_t)ks * chunk_stride : base + (uint32_t)p.off_bs + b_chunk,
+                                    ch, lg_cur, row_first);
             } else {
               compute_chunk(a_grp, base + (uint32_t)p.off_bs + b_chunk);
               flush_grp_dp4a(ch, lg_cur, row_first);

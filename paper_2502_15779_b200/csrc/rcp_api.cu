@@ -310,7 +310,7 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
                   int M, int N, int K, void* y_f16, void* workspace, cudaStream_t st, bool grouped = false,
                   const FusedAct* fa = nullptr, const float* unit = nullptr, int nsplit = 1,
                   const SplitAct* sa = nullptr, int32_t* S_out = nullptr, bool stream_act = false) {
-  if (stream_act && (mode != rcp::kModeMma || grouped || fa || unit || sa || nsplit > 1)) return RCP_ERR_VARIANT;
+  if (stream_act && (mode != rcp::kModeMma || fa || unit || sa || nsplit > 1 || M > (grouped ? 8 : rcp::kMaxTokens))) return RCP_ERR_VARIANT;
   if (nsplit > 1 && (mode != rcp::kModeMma || grouped || fa || M > 8)) return RCP_ERR_VARIANT;
   if (sa && (mode != rcp::kModeMma || grouped || fa || unit || nsplit > 1 || M != 4 || K > 16384)) return RCP_ERR_VARIANT;
   // unit: weight-only form; xq then holds M digit columns of K signed bytes (four per token), scale_f16 is unused
@@ -409,6 +409,9 @@ int launch_stream(int mode, const uint32_t* words, const void* lut_f16, const ui
     if (mode == rcp::kModeDp4a)
       return M == 1 ? launch_stream_t<rcp::kModeDp4a, 1, true>(maps, gp, pl, st)
                     : launch_stream_t<rcp::kModeDp4a, 2, true>(maps, gp, pl, st);
+    if (stream_act)
+      return gp.S_out ? launch_stream_s<rcp::kModeMma, 0, true, false, false, false, true, true>(maps, gp, pl, st)
+                      : launch_stream_s<rcp::kModeMma, 0, true, false, false, false, false, true>(maps, gp, pl, st);
     if (M == 8 && !gp.S_out) return launch_stream_s<rcp::kModeMma, 8, true, false, false, false, false>(maps, gp, pl, st);
     return launch_stream_t<rcp::kModeMma, 0, true>(maps, gp, pl, st);
   }
@@ -445,6 +448,24 @@ int launch_stream_passes(int mode, int cap, const uint32_t* words, const void* l
                                      static_cast<const __half*>(scale_f16) + m0, mm, N, K,
                                      static_cast<__half*>(y_f16) + (size_t)m0 * N, workspace, st, false, nullptr, nullptr, 1,
                                      nullptr, S_out ? S_out + (size_t)m0 * N * 4 : nullptr, true);
+        if (rc != RCP_OK) return rc;
+      }
+      return RCP_OK;
+    }
+  }
+  // Group-wise grid on the tensor cores, a K so long that not even eight tokens' expanded activations fit: the form
+  // with the activations streamed beside the weights takes up to eight tokens in one pass over the weights
+  // (8192 x 28672 at eight tokens: one launch instead of two of four tokens).
+  if (mode == rcp::kModeMma && grouped && mp < std::min(M, 8)) {
+    const int m8 = std::min(M, 8);
+    const StreamPlan sp = make_plan(m8, N, K, sm_count(), true, 0, 1, true);
+    if (sp.stages >= 3 && sp.smem <= kSmemMax) {
+      for (int m0 = 0; m0 < M; m0 += m8) {
+        const int mm = std::min(m8, M - m0);
+        const int rc = launch_stream(mode, words, lut_f16, xq + (size_t)m0 * (K / 2),
+                                     static_cast<const __half*>(scale_f16) + m0, mm, N, K,
+                                     static_cast<__half*>(y_f16) + (size_t)m0 * N, workspace, st, true, nullptr, nullptr, 1,
+                                     nullptr, S_out ? S_out + (size_t)m0 * N * 4 * (K / 128) : nullptr, true);
         if (rc != RCP_OK) return rc;
       }
       return RCP_OK;

@@ -24,6 +24,7 @@ CASES = [
     (64, 28672, 128, 1, "dp4a", True), (300, 2048, 128, 1, "w2a16", False), (2369, 5120, 128, 4, "w2a16", False),
     (40, 65536, 128, 2, "w2a16", False), (300000, 64, 64, 1, "dp4a", False), (150000, 128, 128, 3, "mma_only", True),
     (10240, 8192, 8192, 1, "dp4a", False), (8192, 8192, 8192, 8, "mma_only", False),
+    (300, 28672, 128, 8, "mma_only", True), (2400, 16512, 128, 6, "mma_only", True),   # group-wise grid, activations streamed
 ]
 
 

@@ -61,6 +61,9 @@ SMALL = [
     (127, 1024, 128, 16), (300, 2048, 2048, 1), (256, 4096, 4096, 4), (130, 11008, 128, 1), (64, 28672, 128, 1),
     (40, 14336, 128, 16), (33, 8192, 8192, 8), (2048, 2048, 2048, 1), (513, 1152, 128, 5), (1000, 2560, 128, 7),
     (4800, 1024, 128, 2), (2500, 512, 128, 8),
+    # K so long that eight tokens' expanded activations do not fit: the form with the activations streamed beside
+    # the weights (five to eight tokens in one launch, sixteen as two)
+    (64, 28672, 128, 8), (200, 20480, 128, 5), (33, 65536, 128, 7), (2400, 16512, 128, 8), (40, 28672, 128, 16),
 ]
 
 
