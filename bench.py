@@ -323,11 +323,13 @@ def per_shape_table(cfg, Ms, device, rcp, stream, variant, reps=3):
             best = min(time_graph_replays([g], [0], stream) for _ in range(reps))
             us = best * 1e3 / launches
             nbytes = cfgs.gemv_bytes(M, L.N, L.K)
-            # isolated single launch (includes launch latency)
+            # isolated single launch: no neighbour to overlap with. Queued behind a spin of about 100 us, so that the
+            # two event records and the launch are all waiting when the spin ends and no host latency is inside.
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             iso = []
             for c in range(min(copies, 5)):
                 with torch.cuda.stream(stream):
+                    torch.cuda._sleep(200000)
                     e0.record(stream)
                     rcp.rcp_gemv_w2a4(words[c], luts[c], xq, scale, y=y, workspace=ws, variant=variant)
                     e1.record(stream)
