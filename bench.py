@@ -669,6 +669,21 @@ def main():
                        "stores y into it directly (no staging copy); the host waits for the stream after every step",
            "h2d_bytes_per_step": sum(2 * M * L.K for L in layer.layers),
            "d2h_bytes_per_step": sum(2 * M * L.N for L in layer.layers)}
+    # The same step from a C++ host program through the C ABI (no interpreter in the loop), one token: what the
+    # binding and the interpreter add to the figure above. Rank 0 of a single-GPU run only; reported beside it.
+    if rank == 0 and world == 1 and M == 1:
+        try:
+            from paper_2502_15779_b200 import build as _b
+            drv = _b.build_driver()
+            cmd = [drv, str(e2e_steps), "5"] + [str(v) for L in layer.layers for v in (L.N, L.K, L.had_block)]
+            env = dict(os.environ, CUDA_VISIBLE_DEVICES=os.environ.get("CUDA_VISIBLE_DEVICES", str(local_rank)))
+            out = subprocess.run(cmd, capture_output=True, text=True, timeout=300, env=env)
+            d = json.loads(out.stdout.strip().splitlines()[-1])
+            e2e["c_driver"] = {"value": round(d["gbs"], 2), "unit": UNIT, "ms_per_step": round(d["us_per_step"] / 1e3, 4),
+                               "note": "e2e_driver.cu: rcp_linear_w2a4_host per linear on pinned buffers, "
+                                       "cudaStreamSynchronize after every step, host wall clock"}
+        except Exception as ex:   # noqa: BLE001  (the driver is an extra: never fail the benchmark for it)
+            e2e["c_driver"] = {"unavailable": repr(ex)[:200]}
 
     if rank != 0:
         if dist is not None:

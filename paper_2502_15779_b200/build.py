@@ -6,6 +6,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librcp_w2a4.so")
 LIB_CHECKED = os.path.join(HERE, "librcp_w2a4_checked.so")   # the guarded build (-DRCP_CHECKED), for tests
+DRIVER = os.path.join(HERE, "e2e_driver")                     # host program: a decode step through the C ABI
 SOURCES = ["rcp_api.cu"]
 
 
@@ -40,8 +41,21 @@ def build_checked(force: bool = False) -> str:
     return _compile(LIB_CHECKED, defines=("RCP_CHECKED",))
 
 
+def build_driver(force: bool = False) -> str:
+    """The end-to-end driver (e2e_driver.cu): a C++ host program linked against the library, run by bench.py."""
+    build()
+    src = os.path.join(HERE, "e2e_driver.cu")
+    if not force and os.path.exists(DRIVER) and os.path.getmtime(DRIVER) >= max(os.path.getmtime(src), os.path.getmtime(LIB)):
+        return DRIVER
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O2", "-std=c++17", "-o", DRIVER, src,
+                           "-L" + HERE, "-lrcp_w2a4", "-Xlinker", "-rpath", "-Xlinker", "$ORIGIN"])
+    return DRIVER
+
+
 if __name__ == "__main__":
     import sys
     print(build(force=True, verbose=True))
+    print(build_driver(force=True))
     if "--checked" in sys.argv[1:]:
         print(build_checked(force=True))
