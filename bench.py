@@ -329,7 +329,8 @@ def per_shape_table(cfg, Ms, device, rcp, stream, variant, reps=3):
             iso = []
             for c in range(min(copies, 5)):
                 with torch.cuda.stream(stream):
-                    torch.cuda._sleep(200000)
+                    if hasattr(torch.cuda, "_sleep"):
+                        torch.cuda._sleep(200000)
                     e0.record(stream)
                     rcp.rcp_gemv_w2a4(words[c], luts[c], xq, scale, y=y, workspace=ws, variant=variant)
                     e1.record(stream)
