@@ -55,7 +55,7 @@ def test_random_shape(N, K, M, variant, grouped, i):
     torch.cuda.synchronize()
     assert int(ws.abs().max()) == 0
     rows = np.arange(N) if N * K * M <= 1 << 24 else np.unique(np.concatenate(
-        [np.arange(64), np.arange(N - 64, N), np.random.default_rng(i).integers(0, N, size=256)]))
+        [np.arange(min(N, 64)), np.arange(max(N - 64, 0), N), np.random.default_rng(i).integers(0, N, size=256)]))
     qa = oracle.quantize_act(f16_bits(x), B, 1.0)
     assert np.array_equal(xq.cpu().numpy(), qa["xq"]) and np.array_equal(f16_bits(scale), qa["scale"])
     w_ref = oracle.pack_weights(codes.cpu().numpy()[rows])
@@ -99,7 +99,7 @@ def test_random_shape_weight_only(N, K, M, variant, grouped, i):
     assert np.array_equal(digits.cpu().numpy(), sp["digits"])
     assert np.array_equal(unit.cpu().numpy().astype(np.float64), sp["unit"])
     rows = np.arange(N) if N * K * M <= 1 << 24 else np.unique(np.concatenate(
-        [np.arange(64), np.arange(N - 64, N), np.random.default_rng(i).integers(0, N, size=256)]))
+        [np.arange(min(N, 64)), np.arange(max(N - 64, 0), N), np.random.default_rng(i).integers(0, N, size=256)]))
     ref = oracle.gemv_w2a16(oracle.pack_weights(codes.cpu().numpy()[rows]), np.ascontiguousarray(f16_bits(lut)[rows]),
                             f16_bits(x))
     tol = (0.5 * sp["unit"][:, :1] * ref["labs"][None, :] + 2.0 ** -20 * ref["labsx"]
@@ -132,7 +132,7 @@ def test_extreme_shapes(N, K, M, grouped):
     torch.cuda.synchronize()
     assert int(ws.abs().max()) == 0
     rows = np.arange(N) if N <= 4096 else np.unique(np.concatenate(
-        [np.arange(64), np.arange(N - 64, N), np.random.default_rng(seed).integers(0, N, size=512)]))
+        [np.arange(min(N, 64)), np.arange(max(N - 64, 0), N), np.random.default_rng(seed).integers(0, N, size=512)]))
     qa = oracle.quantize_act(f16_bits(x), B, 1.0)
     assert np.array_equal(xq.cpu().numpy(), qa["xq"]) and np.array_equal(f16_bits(scale), qa["scale"])
     w_ref = oracle.pack_weights(codes.cpu().numpy()[rows])

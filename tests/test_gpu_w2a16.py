@@ -110,7 +110,7 @@ def test_w2a16_matches_w2a4_on_int4_activations():
 
 def test_w2a16_full_size_sampled_rows():
     N, K = 28672, 4096
-    rows = np.unique(np.concatenate([np.arange(64), np.arange(N - 64, N), np.random.default_rng(0).integers(0, N, 256)]))
+    rows = np.unique(np.concatenate([np.arange(min(N, 64)), np.arange(max(N - 64, 0), N), np.random.default_rng(0).integers(0, N, 256)]))
     _check(N, K, 1, seed=11, rows=rows)
     N, K = 8192, 28672
     rows = np.unique(np.concatenate([np.arange(32), np.arange(N - 32, N), np.random.default_rng(1).integers(0, N, 64)]))
