@@ -242,3 +242,11 @@ def test_packed_weights_beyond_four_gibibytes():
                            qa["xq"], qa["scale"])
     got = y[:, rows_t].float().cpu().numpy().astype(np.float64)
     assert np.all(np.abs(got - ref["y"]) <= ref["tol"])
+
+
+def test_random_shapes_other_seeds():
+    """The sweep above over six more seeds (288 cases) in one test: shapes the fixed list never meets."""
+    for seed in (101, 202, 303, 404, 505, 606):
+        for c in _cases(48, seed):
+            N, K, M, variant, grouped, i = c.values
+            test_random_shape(N, K, M, variant, grouped, i)
